@@ -1,0 +1,305 @@
+"""Pins for the float64 checker: everything here is fixed by the paper's equations or by
+mathematics, not by the checker itself (hand-worked values, an independent scalar-loop
+transcription, closed forms, invariants, library routines for special cases)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ficoco_oracle as fo
+from paper_2411_17686_b200 import synth
+from tests import brute_force as bf
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def tiny_v(seed, n_side=4, dim=8, heads=3, keep=10, dtype="fp32"):
+    return synth.make_v_batch(seed, 1, n_side, n_side, dim, heads, keep, dtype, True, 1.0, corr_len=1.5)
+
+
+# ---------------------------------------------------------------------------
+# hand-worked example (Eq. 1, Eq. 2)
+# ---------------------------------------------------------------------------
+
+def test_hand_worked_example():
+    g = json.load(open(os.path.join(HERE, "golden", "hand_example.json")))
+    P = np.array(g["patches"], dtype=np.float32)
+    attn = np.array(g["cls_attention"], dtype=np.float32)
+    for case in g["cases"]:
+        p = fo.Params(lam=g["lambda"], eps=case["eps"], local_penalty=False)
+        r = fo.ficoco_v_reduce(P, attn, None, (2, 2), g["keep"], has_cls=False, p=p)
+        # float32 storage of 0.1 / 0.4 attention limits the agreement to ~1e-8
+        np.testing.assert_allclose(r.v, g["vision_redundancy"], atol=1e-12)
+        np.testing.assert_allclose(r.score, g["score"], atol=1e-8)
+        assert sorted(r.S.tolist()) == g["S"] and r.T.tolist() == g["T"]
+        order = np.argsort(r.S)
+        C = r.C[order]
+        np.testing.assert_allclose(C, g["C"], atol=1e-12)
+        for k, si in enumerate(order):
+            assert r.J[si].tolist() == case["J"][k]
+            np.testing.assert_allclose(r.alpha[si], case["alpha"][k], atol=1e-12)
+        np.testing.assert_allclose(r.out.astype(np.float64), case["merged"], rtol=1e-6)
+        assert r.kept_idx.tolist() == g["T"]
+
+
+# ---------------------------------------------------------------------------
+# independent scalar-loop transcription on tiny inputs
+# ---------------------------------------------------------------------------
+
+def _compare_with_brute(r, b, P64):
+    np.testing.assert_allclose(r.score_raw, b["s_raw"], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(r.score, b["s"], rtol=0, atol=1e-12)
+    assert r.S.tolist() == b["S"]
+    assert r.T.tolist() == b["T"]
+    Tl = r.T.tolist()
+    for k, i in enumerate(r.S.tolist()):
+        assert [Tl[j] for j in r.J[k].tolist()] == b["J"][i]
+        for jj, a in zip(r.J[k].tolist(), r.alpha[k].tolist()):
+            assert abs(a - b["alpha"][(i, Tl[jj])]) < 1e-12
+        for jj, j in enumerate(Tl):
+            assert abs(r.C[k, jj] - b["C"][(i, j)]) < 1e-12
+    return Tl
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+@pytest.mark.parametrize("penalty", [True, False])
+@pytest.mark.parametrize("eps", [0.998, 0.7])
+def test_v_matches_brute_force(seed, penalty, eps):
+    batch = tiny_v(seed)
+    # knock out some grid cells so that padding of discarded positions is exercised
+    alive = np.sort(synth.rng_for(seed, 9).permutation(16)[:13]).astype(np.int32)
+    tok = np.concatenate([batch.tokens[0][:1], batch.tokens[0][1:][alive]])
+    attn = batch.attn[0][:, alive]
+    p = fo.Params(eps=eps, local_penalty=penalty)
+    r = fo.ficoco_v_reduce(tok, attn, alive, (4, 4), 8, True, p)
+    P = tok[1:].astype(np.float64)
+    b = bf.reduce_v(P.tolist(), attn.astype(np.float64).tolist(), alive.tolist(), 4, 4, 8,
+                    eps=eps, penalty=penalty)
+    Tl = _compare_with_brute(r, b, P)
+    for jj, j in enumerate(Tl):
+        np.testing.assert_allclose(r.out[1 + jj].astype(np.float64), b["merged"][j], rtol=2e-7, atol=1e-7)
+    assert r.kept_idx.tolist() == [0] + [1 + j for j in Tl]
+    assert r.pos_out.tolist() == [int(alive[j]) for j in Tl]
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+@pytest.mark.parametrize("eps", [0.998, 0.6])
+def test_l_matches_brute_force(seed, eps):
+    lb = synth.make_l_batch(seed, 1, 14, 5, 8, 3, 6, "fp32", scale=1.0)
+    p = fo.Params(eps=eps)
+    r = fo.ficoco_l_reduce(lb.tokens[0], lb.attn_t2v[0], 14, 6, p)
+    P = lb.tokens[0][:14].astype(np.float64)
+    b = bf.reduce_l(P.tolist(), lb.attn_t2v[0].astype(np.float64).tolist(), 6, eps=eps)
+    Tl = _compare_with_brute(r, b, P)
+    for jj, j in enumerate(Tl):
+        np.testing.assert_allclose(r.out[jj].astype(np.float64), b["merged"][j], rtol=2e-7, atol=1e-7)
+    # text rows pass through untouched after the preserved vision rows
+    assert np.array_equal(r.out[len(Tl):], lb.tokens[0][14:])
+    assert r.kept_idx.tolist() == Tl + list(range(14, 19))
+
+
+def test_planted_mistakes_are_caught(monkeypatch):
+    """Each plausible slip in the checker must break agreement with the scalar transcription."""
+    batch = tiny_v(5)
+    tok, attn = batch.tokens[0], batch.attn[0]
+    P = tok[1:].astype(np.float64)
+    b = bf.reduce_v(P.tolist(), attn.astype(np.float64).tolist(), list(range(16)), 4, 4, 10, eps=0.6)
+
+    def disagree():
+        r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 10, True, fo.Params(eps=0.6))
+        try:
+            Tl = _compare_with_brute(r, b, P)
+            for jj, j in enumerate(Tl):
+                np.testing.assert_allclose(r.out[1 + jj].astype(np.float64), b["merged"][j],
+                                           rtol=2e-7, atol=1e-7)
+        except AssertionError:
+            return True
+        return False
+
+    assert not disagree()
+    mistakes = {
+        "score_v": lambda v, a, lam: lam * v + (1 - lam) * a,                       # wrong sign
+        "vision_redundancy": lambda R: (R.sum(axis=1) - 1.0) / R.shape[0],          # dropped j = i
+        "correlation_v": lambda R, S, T: R[np.ix_(T, S)].T[::-1],                   # wrong index
+        "head_mean": lambda attn: attn.astype(np.float64).sum(axis=0),              # no 1/H
+        "quantile_threshold": lambda row, eps: float(np.sort(row)[int(eps * (len(row) - 1))]),  # no interpolation
+    }
+    for name, wrong in mistakes.items():
+        with monkeypatch.context() as m:
+            m.setattr(fo, name, wrong)
+            assert disagree(), f"planted mistake in {name} went unnoticed"
+
+
+# ---------------------------------------------------------------------------
+# closed forms and invariants
+# ---------------------------------------------------------------------------
+
+def test_relation_properties_and_closed_form_row_mean():
+    batch = synth.make_v_batch(21, 1, 6, 6, 32, 2, 20, "fp32")
+    P = batch.tokens[0][1:].astype(np.float64)
+    R = fo.cosine_relation(P)
+    assert np.allclose(np.diag(R), 1.0, atol=1e-14)
+    assert np.allclose(R, R.T, atol=1e-15)
+    assert np.abs(R).max() <= 1.0 + 1e-14
+    Ph = P / np.linalg.norm(P, axis=1, keepdims=True)
+    closed = Ph @ Ph.mean(axis=0)           # (1/N) sum_j R_ij = x_hat_i . mean_j x_hat_j
+    np.testing.assert_allclose(fo.vision_redundancy(R), closed, atol=1e-14)
+    # against torch's cosine similarity routine
+    tP = torch.from_numpy(P)
+    Rt = torch.nn.functional.cosine_similarity(tP[:, None, :], tP[None, :, :], dim=-1).numpy()
+    np.testing.assert_allclose(R, Rt, atol=1e-12)
+
+
+def test_lambda_extremes():
+    batch = synth.make_v_batch(22, 1, 6, 6, 32, 2, 20, "fp32")
+    tok, attn = batch.tokens[0], batch.attn[0]
+    r1 = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(lam=1.0, local_penalty=False))
+    assert set(r1.S.tolist()) == set(np.argsort(-r1.v, kind="stable")[:16].tolist())
+    r0 = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(lam=0.0, local_penalty=False))
+    a = attn.astype(np.float64).mean(axis=0)
+    assert set(r0.S.tolist()) == set(np.argsort(a, kind="stable")[:16].tolist())  # lowest CLS attention
+
+
+def test_local_penalty_special_cases():
+    batch = synth.make_v_batch(23, 1, 6, 6, 32, 2, 20, "fp32")
+    tok, attn = batch.tokens[0], batch.attn[0]
+    off = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(local_penalty=False))
+    one = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(penalty_coef=1.0))
+    assert np.array_equal(off.score, one.score) and np.array_equal(off.out, one.out)
+    w1 = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(window=1))
+    np.testing.assert_allclose(w1.score, 2.0 * w1.score_raw, rtol=0, atol=0)
+    # default: exactly one token per 2x2 window is doubled, and it is the window maximum
+    d = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True)
+    changed = np.nonzero(d.score != d.score_raw)[0]
+    assert changed.shape[0] == 9
+    grid = d.score_raw.reshape(3, 2, 3, 2).transpose(0, 2, 1, 3).reshape(9, 4)
+    np.testing.assert_allclose(np.sort(d.score[changed]), np.sort(2.0 * grid.max(axis=1)))
+    # odd grid: edge windows are smaller, discarded cells are padding
+    s = np.array([0.3, -0.2, 0.1, 0.5, -0.4, -0.1], dtype=np.float64)
+    pos = np.array([0, 1, 2, 3, 5, 8])
+    out = fo.local_penalty(s, pos, (3, 3), 2, 2.0)
+    # windows: {0,1,3,(4 dead)} -> max 0.5 at pos 3 ; {2,5} -> 0.1 ; {(6,7 dead)} none ; {8} -> -0.1
+    np.testing.assert_allclose(out, [0.3, -0.2, 0.2, 1.0, -0.4, -0.2])
+
+
+def test_selection_invariants_and_permutation_equivariance():
+    batch = synth.make_v_batch(24, 1, 6, 6, 32, 2, 20, "fp32")
+    tok, attn = batch.tokens[0], batch.attn[0]
+    p = fo.Params(local_penalty=False)
+    r = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, p)
+    assert r.out.shape[0] == 1 + 20 and r.kept_idx[0] == 0
+    assert np.array_equal(r.out[0], tok[0])
+    S, T = set(r.S.tolist()), set(r.T.tolist())
+    assert not (S & T) and (S | T) == set(range(36)) and len(S) == 16
+    assert np.all(np.diff(r.T) > 0)
+    perm = synth.rng_for(24, 5).permutation(36)
+    tok2 = np.concatenate([tok[:1], tok[1:][perm]])
+    r2 = fo.ficoco_v_reduce(tok2, attn[:, perm], None, (6, 6), 20, True, p)
+    assert set(perm[r2.S].tolist()) == S
+    # same merged rows, in the permuted order
+    inv = {int(perm[j]): k for k, j in enumerate(r2.T.tolist())}
+    for k, j in enumerate(r.T.tolist()):
+        np.testing.assert_allclose(r.out[1 + k], r2.out[1 + inv[j]], rtol=1e-6)
+
+
+def test_quantile_matches_library_and_eps_one():
+    rng = synth.rng_for(25)
+    for n in (2, 3, 17, 288, 512, 1440):
+        row = rng.standard_normal(n)
+        for eps in (0.998, 0.5, 0.0, 1.0, 0.9731):
+            assert abs(fo.quantile_threshold(row, eps) - float(np.quantile(row, eps))) < 1e-12
+            tq = float(torch.quantile(torch.from_numpy(row), eps))
+            assert abs(fo.quantile_threshold(row, eps) - tq) < 1e-12
+    C = rng.standard_normal((5, 40))
+    J, A, tau = fo.targets_and_weights(C, fo.Params(eps=1.0))
+    for i in range(5):
+        assert J[i].tolist() == [int(np.argmax(C[i]))] or C[i].max() <= 0
+        if J[i].size:
+            assert A[i].tolist() == [1.0]
+
+
+def test_number_of_targets_follows_the_quantile_level():
+    rng = synth.rng_for(26)
+    for n, k in ((288, 1), (144, 1), (64, 1), (512, 2), (720, 2), (1440, 3)):
+        C = np.abs(rng.standard_normal((3, n))) + 0.01
+        J, A, _ = fo.targets_and_weights(C, fo.Params())
+        for i in range(3):
+            assert J[i].shape[0] == k == n - 1 - int(np.floor(0.998 * (n - 1)))
+            assert abs(A[i].sum() - 1.0) < 1e-14
+            assert set(J[i].tolist()) == set(np.argsort(-C[i])[:k].tolist())
+
+
+def test_merge_invariants():
+    batch = synth.make_v_batch(27, 1, 8, 8, 16, 2, 24, "fp32")
+    tok, attn = batch.tokens[0], batch.attn[0]
+    p = fo.Params(eps=0.9)
+    r = fo.ficoco_v_reduce(tok, attn, None, (8, 8), 24, True, p)
+    P = tok[1:].astype(np.float64)
+    # total-mass identity: sum_j (1 + w_j) out_j = sum_{j in T} x_j + sum_{i in S, J_i != {}} x_i
+    merged, wsum = fo.compress(P, r.S, r.T, r.J, r.alpha)
+    lhs = ((1.0 + wsum)[:, None] * merged).sum(axis=0)
+    used = [int(i) for k, i in enumerate(r.S) if r.J[k].size]
+    rhs = P[r.T].sum(axis=0) + P[used].sum(axis=0)
+    np.testing.assert_allclose(lhs, rhs, atol=1e-10)
+    # a target with a single source keeps at least half of itself
+    for jj in range(len(r.T)):
+        srcs = [k for k in range(len(r.S)) if jj in r.J[k].tolist()]
+        if len(srcs) == 1:
+            assert 1.0 / (1.0 + wsum[jj]) >= 0.5
+    # K = 0 is plain pruning: the output is a gather of the input rows
+    r0 = fo.ficoco_v_reduce(tok, attn, None, (8, 8), 24, True, fo.Params(max_targets=0))
+    assert np.array_equal(r0.out, tok[r0.kept_idx])
+    assert np.array_equal(r0.T, r.T)
+    # identical tokens merge to themselves
+    same = np.repeat(tok[1:2], 65, axis=0)
+    rs = fo.ficoco_v_reduce(same, attn, None, (8, 8), 24, True, p)
+    np.testing.assert_allclose(rs.out, same[:25], rtol=1e-6)
+
+
+def test_untouched_rows_keep_their_bits_and_bf16_rounding():
+    batch = synth.make_v_batch(28, 2, 8, 8, 64, 2, 40, "bf16")
+    for b in range(2):
+        r = fo.ficoco_v_reduce(batch.tokens[b], batch.attn[b], None, (8, 8), 40, True)
+        untouched = np.nonzero(r.wsum == 0)[0]
+        assert untouched.size > 0
+        assert np.array_equal(r.out[1 + untouched], batch.tokens[b][1 + r.T[untouched]])
+    # the float64 -> bf16 rounding against torch's own conversion, incl. exact halfway cases
+    rng = synth.rng_for(28, 1)
+    x = rng.standard_normal(20000) * np.exp(rng.uniform(-20, 20, 20000))
+    half = (np.arange(1, 200, dtype=np.float64) * 2 + 1) / 512.0   # 9 significant bits: ties
+    x = np.concatenate([x, half, -half, [0.0, 1.0, -1.0, 3.0 + 2.0 ** -8, 3.0 + 2.0 ** -7]])
+    mine = fo.round_to_bf16_bits(x)
+    ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(mine, ref)
+    assert np.array_equal(fo.widen(mine), synth.bf16_bits_to_f32(mine).astype(np.float64))
+
+
+def test_ficoco_l_special_cases():
+    lb = synth.make_l_batch(29, 1, 40, 6, 32, 3, 12, "fp32", scale=1.0)
+    tok, att = lb.tokens[0], lb.attn_t2v[0]
+    t = fo.head_mean(att)
+    P = tok[:40].astype(np.float64)
+    R = fo.cosine_relation(P)
+    r = fo.ficoco_l_reduce(tok, att, 40, 12, fo.Params(gamma=1.0))
+    np.testing.assert_allclose(r.C, R[np.ix_(r.S, r.T)], atol=0)
+    rb = fo.ficoco_l_reduce(tok, att, 40, 12, fo.Params(beta=1.0))
+    np.testing.assert_allclose(rb.score, fo.vision_redundancy(R), atol=0)
+    G = t.T @ t / t.shape[0]
+    assert np.allclose(G, G.T) and np.linalg.eigvalsh(G).min() > -1e-12
+    full = fo.ficoco_l_reduce(tok, att, 40, 12)
+    expect = 0.6 * R[np.ix_(full.S, full.T)] + 0.4 * G[np.ix_(full.S, full.T)]
+    np.testing.assert_allclose(full.C, expect, atol=1e-15)
+    assert full.out.shape[0] == 12 + 6
+
+
+def test_edge_counts():
+    batch = synth.make_v_batch(30, 1, 4, 4, 8, 2, 16, "fp32")
+    tok, attn = batch.tokens[0], batch.attn[0]
+    r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 16, True)      # discard nothing
+    assert np.array_equal(r.out, tok) and r.S.size == 0
+    r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 0, True)       # discard everything
+    assert r.out.shape[0] == 1 and np.array_equal(r.out[0], tok[0])
+    r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 1, True)       # one target takes it all
+    assert r.out.shape[0] == 2 and all(j.tolist() == [0] for j in r.J if j.size)
