@@ -1,0 +1,214 @@
+/*
+ * libficoco -- the FiCoCo token-reduction step (filter, correlate, compress, compact)
+ * as CUDA kernels for sm_100a behind a C ABI.
+ *
+ * What one call computes, per image (or per sequence), following the paper
+ * "Filter, Correlate, Compress: Training-Free Token Reduction for MLLM Acceleration":
+ *
+ *   filter    Eq. 1:  s_i = lambda * (1/N) sum_j A_ij - (1 - lambda) * a_i, followed by the
+ *             local penalty (2x2 windows on the patch grid, window maximum times 2; Sec.
+ *             "Redundancy-based Token Discard") and a top-N^S selection of the tokens to
+ *             discard (set S); the rest is the target set T.
+ *   correlate Sec. "Correlation-based Information Recycling": C_ij = A_ij for i in S,
+ *             j in T; tau_i = eps-quantile of row i; J_i = { j : C_ij >= tau_i }.
+ *   compress  Eq. 2:  X_j <- (X_j + sum_{i in I_j} alpha_ij X_i) / (1 + sum_{i in I_j} alpha_ij),
+ *             alpha_ij = C_ij / sum_{j in J_i} C_ij.
+ *   compact   Algorithm 1, last step: the rows of S are removed, order preserved.
+ *
+ * The token-to-token relation A_ij between two vision tokens is the cosine similarity of
+ * the token features; the attention-derived term a_i is supplied by the caller (CLS->patch
+ * attention per head for FiCoCo-V, text->vision attention per head for FiCoCo-L) and is
+ * averaged over heads.  FiCoCo-L (Sec. "Task-Aware Improvements for FiCoCo-L") uses
+ * s_i = beta * v_i - (1 - beta) * (1/M) sum_k t_ki, no local penalty, and
+ * C_ij = gamma * A_ij + (1 - gamma) * (1/M) sum_k t_ki t_kj with t the head-mean
+ * text->vision attention.
+ *
+ * General rules
+ *   - "device" pointers are CUDA device memory on the context's device; "host" pointers
+ *     are ordinary host memory read during the call.
+ *   - The caller owns every input and output buffer.  A context owns only scratch memory.
+ *   - ficoco_v_reduce / ficoco_l_reduce enqueue work on the given stream and return without
+ *     synchronising.  A context must be used from one stream at a time.
+ *   - The first call with a new combination of shapes builds and uploads a small plan
+ *     (per-image descriptors); that first call may synchronise the stream and must happen
+ *     outside stream capture.  Up to 8 plans are cached per context.
+ *   - Every function returns FICOCO_OK (0) or a negative ficoco_error; nothing is launched
+ *     when argument validation fails.  Problems only the device can see (a `pos` entry
+ *     outside the grid) set bits in a status word read by ficoco_status.
+ *   - Token rows must be 16-byte aligned: dim % 8 == 0 for bf16, dim % 4 == 0 for fp32.
+ *     A token row of all zeros has no direction; its cosine is taken as 0.
+ *   - At most 8192 vision tokens per image; the top list needed for tau_i,
+ *     n - floor(eps * (n - 1)) entries for n preserved tokens, must not exceed 16.
+ */
+#ifndef FICOCO_H_
+#define FICOCO_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ficoco_ctx ficoco_ctx;
+
+enum ficoco_dtype { FICOCO_FP32 = 0, FICOCO_BF16 = 1 };
+
+enum ficoco_error {
+  FICOCO_OK = 0,
+  FICOCO_ERR_INVALID_ARG = -1,   /* NULL pointer, non-positive size, misaligned pointer */
+  FICOCO_ERR_UNSUPPORTED = -2,   /* dtype / dim / per-image size / quantile level outside the supported range */
+  FICOCO_ERR_KEEP_RANGE = -3,    /* keep count < 0 or > number of alive vision tokens */
+  FICOCO_ERR_WORKSPACE = -4,     /* problem larger than the sizes given to ficoco_create */
+  FICOCO_ERR_CUDA = -5,          /* a CUDA runtime call failed (see ficoco_last_cuda_error) */
+  FICOCO_ERR_TIMEOUT = -6,       /* a bounded device-side wait ran out */
+  FICOCO_ERR_CAPTURE = -7,       /* a new plan would have to be uploaded during stream capture */
+  FICOCO_ERR_GRID = -8           /* grid_h * grid_w smaller than the number of alive patches */
+};
+
+enum ficoco_flags {
+  FICOCO_HAS_CLS = 1u,           /* row 0 of every image is a CLS token: never scored, always kept */
+  FICOCO_LOCAL_PENALTY = 2u      /* apply the local penalty (FiCoCo-V default) */
+};
+
+/* Hyper-parameters; defaults are the paper's (Sec. "Implementation Details"):
+ * lambda 0.35, beta 0.6, gamma 0.6, eps 0.998, penalty coefficient 2, window 2. */
+typedef struct ficoco_params {
+  double lambda_;       /* Eq. 1 balance (FiCoCo-V) */
+  double beta;          /* score balance (FiCoCo-L) */
+  double gamma;         /* direct / text-bridged balance in C^l (FiCoCo-L) */
+  double eps;           /* quantile level of the token-wise threshold tau_i, in [0, 1] */
+  double penalty_coef;  /* local-penalty scaling coefficient */
+  int window;           /* local-penalty window side, >= 1 */
+  int max_targets;      /* < 0: token-adaptive K (the paper's method); 0: pruning only;
+                           k > 0: every discarded token goes to its k most correlated targets */
+  unsigned flags;       /* ficoco_flags */
+  int reserved;
+} ficoco_params;
+
+/* Fill *p with the paper's defaults and flags = HAS_CLS | LOCAL_PENALTY. */
+void ficoco_default_params(ficoco_params* p);
+
+/* Create a context on `device` with scratch sized for
+ *   max_tokens : upper bound on the total number of token rows in one call (all images),
+ *   max_dim    : upper bound on the hidden size,
+ *   max_batch  : upper bound on the number of images / sequences per call,
+ *   max_text   : upper bound on text tokens per sequence (0 if ficoco_l_reduce is not used).
+ * Allocates device memory once; no later device-pointer call allocates.  *out receives the
+ * context. */
+int ficoco_create(ficoco_ctx** out, int device, long long max_tokens, int max_dim,
+                  int max_batch, int max_text);
+int ficoco_destroy(ficoco_ctx* ctx);
+
+const char* ficoco_strerror(int code);
+/* The CUDA error code behind the last FICOCO_ERR_CUDA of this context (0 if none). */
+int ficoco_last_cuda_error(const ficoco_ctx* ctx);
+
+/*
+ * FiCoCo-V reduce step (Algorithm 1) for a batch of images.
+ *
+ * Packing.  Image b has c (0 or 1, from FICOCO_HAS_CLS) CLS rows followed by Np_b alive
+ * patch rows.  Uniform batches give n_tokens = c + Np for all images; ragged batches give
+ * `seqlens` (host, B entries, each c + Np_b) and n_tokens is ignored.  In both cases rows
+ * are packed back to back: image b starts at row sum_{b'<b} (c + Np_b').
+ * Per-patch arrays (pos, scores_out) are packed the same way without the CLS rows.
+ * attn holds, per image, an [H, Np_b] row-major block; blocks are back to back, so image b
+ * starts at float offset H * sum_{b'<b} Np_b' (for a uniform batch this is [B, H, Np]).
+ */
+typedef struct ficoco_v_args {
+  const void* tokens;      /* device, dtype elements, [rows, dim] row-major */
+  const int* seqlens;      /* host int32[B] rows per image incl. CLS, or NULL for uniform */
+  const float* attn;       /* device fp32, CLS->patch attention weights per head */
+  const int* grid_h;       /* host int32[n_grid]: rows of the original patch grid */
+  const int* grid_w;       /* host int32[n_grid]: columns of the original patch grid */
+  const int* pos;          /* device int32 per patch: linear index r * grid_w + c on the
+                              original grid (used by the local penalty); NULL means
+                              pos = 0..Np-1 (nothing discarded yet) */
+  const int* keep;         /* host int32[n_keep]: N^T, patch tokens preserved per image */
+  void* out_tokens;        /* device, dtype, packed [sum_b (c + keep_b), dim] */
+  int* kept_idx;           /* device int32, packed like out_tokens rows: for every output
+                              row the row index inside its image's input (CLS = 0) */
+  int* pos_out;            /* device int32 packed [sum_b keep_b]: pos of the preserved
+                              patches (input to the next step), or NULL */
+  float* scores_out;       /* device fp32 packed per patch: redundancy score after the
+                              local penalty, or NULL */
+  int dtype;               /* ficoco_dtype */
+  int batch;               /* B >= 1 */
+  int n_tokens;            /* rows per image incl. CLS (uniform batches) */
+  int dim;                 /* D */
+  int heads;               /* H >= 1 */
+  int n_grid;              /* 1 (same grid for all images) or B */
+  int n_keep;              /* 1 or B */
+  int reserved;
+} ficoco_v_args;
+
+int ficoco_v_reduce(ficoco_ctx* ctx, const ficoco_v_args* args, const ficoco_params* params,
+                    void* cuda_stream);
+
+/*
+ * FiCoCo-L reduce step (Algorithm 2) for a batch of decoder sequences of equal shape.
+ * Each sequence has n_vision vision rows followed by n_text text rows.  Vision rows are
+ * reduced to `keep`; text rows pass through unchanged after them.
+ */
+typedef struct ficoco_l_args {
+  const void* tokens;      /* device, [B, n_vision + n_text, dim] */
+  const float* attn_t2v;   /* device fp32 [B, H, M, N]: attention of text row k to vision token i */
+  const int* keep;         /* host int32[n_keep]: vision tokens preserved */
+  void* out_tokens;        /* device, packed [sum_b (keep_b + M), dim] */
+  int* kept_idx;           /* device int32 packed like out_tokens rows (text rows: N..N+M-1) */
+  float* scores_out;       /* device fp32 [B, N] redundancy score s^l, or NULL */
+  int dtype;
+  int batch;
+  int n_vision;            /* N */
+  int n_text;              /* M >= 1 */
+  int dim;
+  int heads;
+  int n_keep;              /* 1 or B */
+  int reserved;
+} ficoco_l_args;
+
+int ficoco_l_reduce(ficoco_ctx* ctx, const ficoco_l_args* args, const ficoco_params* params,
+                    void* cuda_stream);
+
+/*
+ * Host-buffer variants: every pointer of the args struct that is documented "device" is a
+ * HOST pointer here.  The call copies the inputs to the device, runs the same kernels,
+ * copies the outputs back and returns after the results are in host memory.  Staging
+ * buffers are allocated inside the context on the first host call (sized by the maxima
+ * given to ficoco_create) and reused.
+ */
+int ficoco_v_reduce_host(ficoco_ctx* ctx, const ficoco_v_args* host_args,
+                         const ficoco_params* params);
+int ficoco_l_reduce_host(ficoco_ctx* ctx, const ficoco_l_args* host_args,
+                         const ficoco_params* params);
+
+/* Synchronise `cuda_stream`, read and clear the device status word into *device_status
+ * (0 = clean; bit 0: a pos entry outside grid_h*grid_w was ignored by the local penalty). */
+int ficoco_status(ficoco_ctx* ctx, void* cuda_stream, int* device_status);
+
+/*
+ * Inspection of the intermediate results of the most recent reduce call on this context
+ * (for tests and debugging).  Synchronises the device, then copies up to `bytes` bytes of
+ * the selected array to `host_dst`; *bytes_avail (optional) receives the array's size.
+ * Arrays are packed over images in call order.
+ */
+enum ficoco_inspect_what {
+  FICOCO_INSPECT_RNORM = 0,      /* fp32 per patch: 1 / ||x_i|| */
+  FICOCO_INSPECT_SCORE_RAW = 1,  /* fp32 per patch: score before the local penalty */
+  FICOCO_INSPECT_SCORE = 2,      /* fp32 per patch: score after the local penalty */
+  FICOCO_INSPECT_SRC_IDX = 3,    /* int32 per discarded token: patch index, ascending */
+  FICOCO_INSPECT_TGT_IDX = 4,    /* int32 per preserved token: patch index, ascending */
+  FICOCO_INSPECT_CORR_CNT = 5,   /* int32 per discarded token: |J_i| */
+  FICOCO_INSPECT_CORR_TGT = 6,   /* int32 [discarded, 16]: positions in T of the targets */
+  FICOCO_INSPECT_CORR_W = 7,     /* fp32  [discarded, 16]: alpha_ij */
+  FICOCO_INSPECT_CORR_C = 8,     /* fp32  [discarded, 16]: C_ij of the top list, descending */
+  FICOCO_INSPECT_TAU = 9         /* fp32 per discarded token: tau_i */
+};
+int ficoco_inspect(ficoco_ctx* ctx, int what, void* host_dst, size_t bytes, size_t* bytes_avail);
+
+/* Number of kernels the most recent reduce call launched (for launch accounting). */
+int ficoco_last_launch_count(const ficoco_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FICOCO_H_ */
