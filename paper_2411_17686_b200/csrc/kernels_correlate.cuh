@@ -1,0 +1,291 @@
+// Correlate stage: C_ij for i in S, j in T, per-row top list, tau_i, J_i, alpha_ij, and the
+// inversion of the per-source target lists into per-target source lists.
+#pragma once
+#include <limits.h>
+#include <math_constants.h>
+#include "common.cuh"
+
+namespace ficoco {
+
+constexpr int CBM = 64;   // source rows per CTA
+constexpr int CBN = 64;   // target columns per tile
+constexpr int CKC = 16;   // reduction chunk
+
+// ---------------------------------------------------------------------------------------
+// fp32 SIMT correlate (the path for fp32 tokens, where 1e-5 relative accuracy rules out
+// bf16 tensor-core products).  One CTA owns up to 64 discarded tokens of one image and one
+// column split of that image's preserved tokens; it walks the split in 64-column tiles,
+// forms C = gamma * rn_i rn_j (x_i . x_j) [+ (1-gamma)/M * sum_k t_ki t_kj] in registers
+// (4x4 per thread) and keeps, per row, the L largest entries (value, position in T).
+// The N^S x N^T matrix never leaves the SM.
+// ---------------------------------------------------------------------------------------
+template <class T>
+__global__ void __launch_bounds__(256) k_correlate_simt(
+    const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
+    const WorkItem* __restrict__ work, const float* __restrict__ rn,
+    const int* __restrict__ S_idx, const int* __restrict__ T_idx,
+    const float* __restrict__ tmean, int M, float gamma,
+    float* __restrict__ part_val, int* __restrict__ part_idx) {
+  __shared__ __align__(16) float As[CKC][CBM + 4];
+  __shared__ __align__(16) float Bs[CKC][CBN + 4];
+  __shared__ float Cs[CBM][CBN + 1];
+  __shared__ float lv[CBM][KCAP];
+  __shared__ int li[CBM][KCAP];
+  __shared__ int rowS[CBM], rowT[CBN];
+  __shared__ float rnS[CBM], rnT[CBN];
+
+  const WorkItem w = work[blockIdx.x];
+  const ImgDesc d = desc[w.img];
+  const int L = d.list_len;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+
+  for (int i = tid; i < CBM * KCAP; i += 256) {
+    (&lv[0][0])[i] = -CUDART_INF_F;
+    (&li[0][0])[i] = INT_MAX;
+  }
+  if (tid < CBM) {
+    const bool ok = tid < w.nrows;
+    const int p = ok ? S_idx[d.src0 + w.r0 + tid] : -1;
+    rowS[tid] = p;
+    rnS[tid] = ok ? rn[d.patch0 + p] : 0.f;
+  }
+  const int col_begin = w.aux * d.cols_per_split;
+  const int col_end = min(d.n_tgt, col_begin + d.cols_per_split);
+  const size_t tok0 = (size_t)(d.row0 + d.n_cls);
+  const int N = d.np;
+
+  for (int c0 = col_begin; c0 < col_end; c0 += CBN) {
+    __syncthreads();
+    if (tid < CBN) {
+      const int c = c0 + tid;
+      const bool ok = c < col_end;
+      const int p = ok ? T_idx[d.tgt0 + c] : -1;
+      rowT[tid] = p;
+      rnT[tid] = ok ? rn[d.patch0 + p] : 0.f;
+    }
+    __syncthreads();
+
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    const int lr = tid >> 2, lq = tid & 3;
+    for (int k0 = 0; k0 < D; k0 += CKC) {
+      {
+        float fa[4] = {0.f, 0.f, 0.f, 0.f}, fb[4] = {0.f, 0.f, 0.f, 0.f};
+        const int kk = k0 + lq * 4;
+        if (kk < D) {
+          const int pa = rowS[lr], pb = rowT[lr];
+          if (sizeof(T) == 4) {
+            if (pa >= 0) {
+              float4 v = __ldg(reinterpret_cast<const float4*>(tokens + (tok0 + pa) * D + kk));
+              fa[0] = v.x; fa[1] = v.y; fa[2] = v.z; fa[3] = v.w;
+            }
+            if (pb >= 0) {
+              float4 v = __ldg(reinterpret_cast<const float4*>(tokens + (tok0 + pb) * D + kk));
+              fb[0] = v.x; fb[1] = v.y; fb[2] = v.z; fb[3] = v.w;
+            }
+          } else {
+            if (pa >= 0) {
+              uint2 v = __ldg(reinterpret_cast<const uint2*>(tokens + (tok0 + pa) * D + kk));
+              fa[0] = __uint_as_float(v.x << 16); fa[1] = __uint_as_float(v.x & 0xFFFF0000u);
+              fa[2] = __uint_as_float(v.y << 16); fa[3] = __uint_as_float(v.y & 0xFFFF0000u);
+            }
+            if (pb >= 0) {
+              uint2 v = __ldg(reinterpret_cast<const uint2*>(tokens + (tok0 + pb) * D + kk));
+              fb[0] = __uint_as_float(v.x << 16); fb[1] = __uint_as_float(v.x & 0xFFFF0000u);
+              fb[2] = __uint_as_float(v.y << 16); fb[3] = __uint_as_float(v.y & 0xFFFF0000u);
+            }
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          As[lq * 4 + e][lr] = fa[e];
+          Bs[lq * 4 + e][lr] = fb[e];
+        }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kk = 0; kk < CKC; ++kk) {
+        const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+        const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+      }
+      __syncthreads();
+    }
+
+    float cval[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) cval[i][j] = gamma * (rnS[ty * 4 + i] * rnT[tx * 4 + j]) * acc[i][j];
+
+    if (tmean != nullptr) {
+      // text-bridged term: (1-gamma)/M * sum_k t[k, i] t[k, j]
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+      const float* tb = tmean + (size_t)w.img * M * N;
+      for (int k0 = 0; k0 < M; k0 += CKC) {
+        for (int idx = tid; idx < CKC * CBM; idx += 256) {
+          const int kk = idx / CBM, r = idx % CBM;
+          const bool kin = k0 + kk < M;
+          const int pa = rowS[r], pb = rowT[r];
+          As[kk][r] = (kin && pa >= 0) ? __ldg(tb + (size_t)(k0 + kk) * N + pa) : 0.f;
+          Bs[kk][r] = (kin && pb >= 0) ? __ldg(tb + (size_t)(k0 + kk) * N + pb) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < CKC; ++kk) {
+          const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+          const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+          const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+      }
+      const float sc = (1.0f - gamma) / (float)M;
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cval[i][j] = fmaf(sc, acc[i][j], cval[i][j]);
+    }
+
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Cs[ty * 4 + i][tx * 4 + j] = cval[i][j];
+    __syncthreads();
+
+    if (tid < w.nrows) {
+      const int ncol = min(CBN, col_end - c0);
+      for (int c = 0; c < ncol; ++c) {
+        const float val = Cs[tid][c];
+        const int idx = c0 + c;
+        if (toplist_better(val, idx, lv[tid][L - 1], li[tid][L - 1]))
+          toplist_insert(lv[tid], li[tid], L, val, idx);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < w.nrows * L; i += 256) {
+    const int r = i / L, k = i % L;
+    const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + r) * d.nsplit + w.aux) * L + k;
+    part_val[o] = lv[r][k];
+    part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Per image: merge the column splits' partial top lists, take the quantile threshold
+//   tau_i = v[L-1] + frac * (v[L-2] - v[L-1])   (v descending: the two order statistics
+//   around eps*(n-1)), J_i = { entries >= tau_i }, alpha_ij = C+_ij / sum_{J_i} C+  (Eq. 2),
+// then invert source->targets into per-target segments sorted by source, which fixes the
+// accumulation order of the merge.
+// One CTA (256 threads) per image; dynamic smem: 2 * n_tgt ints.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_finalize(
+    const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
+    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, int* __restrict__ corr_tgt,
+    float* __restrict__ corr_w, float* __restrict__ corr_c, float* __restrict__ tau_out,
+    int* __restrict__ seg_off, int* __restrict__ seg_src, float* __restrict__ seg_w) {
+  extern __shared__ int smi[];
+  __shared__ int warp_tot[33];
+  const ImgDesc d = desc[blockIdx.x];
+  const int img = blockIdx.x;
+  const int L = d.list_len;
+  const int tid = threadIdx.x;
+  int* cnt = smi;
+  int* cur = smi + d.n_tgt;
+
+  for (int j = tid; j < d.n_tgt; j += 256) cnt[j] = 0;
+  __syncthreads();
+
+  for (int s = tid; s < d.n_src; s += 256) {
+    const size_t o = (size_t)(d.src0 + s);
+    if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; continue; }
+    float v[KCAP];
+    int ix[KCAP];
+#pragma unroll
+    for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
+    for (int e = 0; e < d.nsplit * L; ++e) {
+      const int id = part_idx[pbase + e];
+      const float val = part_val[pbase + e];
+      if (id >= 0 && toplist_better(val, id, v[L - 1], ix[L - 1])) toplist_insert(v, ix, L, val, id);
+    }
+    const float tau = (L >= 2) ? v[L - 1] + d.frac * (v[L - 2] - v[L - 1]) : v[0];
+    int nj = 0;
+    float den = 0.f;
+    for (int k = 0; k < L; ++k) {
+      if (ix[k] != INT_MAX && v[k] >= tau) { ++nj; den += fmaxf(v[k], 0.f); } else break;
+    }
+    if (!(den > 1e-12f)) nj = 0;
+    corr_cnt[o] = nj;
+    tau_out[o] = tau;
+    for (int k = 0; k < KCAP; ++k) {
+      corr_tgt[o * KCAP + k] = k < nj ? ix[k] : -1;
+      corr_w[o * KCAP + k] = k < nj ? fmaxf(v[k], 0.f) / den : 0.f;
+      corr_c[o * KCAP + k] = k < L ? v[k] : 0.f;
+    }
+    for (int k = 0; k < nj; ++k) atomicAdd(&cnt[ix[k]], 1);
+  }
+  __syncthreads();
+
+  int base = 0;
+  for (int j0 = 0; j0 < d.n_tgt; j0 += 256) {
+    const int j = j0 + tid;
+    const int c = j < d.n_tgt ? cnt[j] : 0;
+    int tot;
+    const int ex = base + block_exclusive_scan(c, warp_tot, &tot);
+    if (j < d.n_tgt) {
+      cur[j] = ex;
+      seg_off[d.tgt0 + img + j] = d.ent0 + ex;
+    }
+    base += tot;
+  }
+  if (tid == 0) seg_off[d.tgt0 + img + d.n_tgt] = d.ent0 + base;
+  __syncthreads();
+
+  for (int s = tid; s < d.n_src; s += 256) {
+    const size_t o = (size_t)(d.src0 + s);
+    const int nj = corr_cnt[o];
+    for (int k = 0; k < nj; ++k) {
+      const int j = corr_tgt[o * KCAP + k];
+      const int slot = atomicAdd(&cur[j], 1);
+      seg_src[d.ent0 + slot] = s;
+      seg_w[d.ent0 + slot] = corr_w[o * KCAP + k];
+    }
+  }
+  __syncthreads();
+
+  // ascending source order inside every segment (sources ascend with the token index)
+  for (int j = tid; j < d.n_tgt; j += 256) {
+    const int e1 = d.ent0 + cur[j];
+    const int e0 = e1 - cnt[j];
+    for (int a = e0 + 1; a < e1; ++a) {
+      const int ks = seg_src[a];
+      const float kw = seg_w[a];
+      int b = a - 1;
+      while (b >= e0 && seg_src[b] > ks) {
+        seg_src[b + 1] = seg_src[b];
+        seg_w[b + 1] = seg_w[b];
+        --b;
+      }
+      seg_src[b + 1] = ks;
+      seg_w[b + 1] = kw;
+    }
+  }
+}
+
+}  // namespace ficoco
