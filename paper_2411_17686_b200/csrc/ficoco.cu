@@ -1,0 +1,690 @@
+// C ABI of libficoco: context, plans, argument validation and kernel launches.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/ficoco.h"
+#include "common.cuh"
+#include "kernels_correlate.cuh"
+#include "kernels_filter.cuh"
+#include "kernels_merge.cuh"
+
+using namespace ficoco;
+
+namespace {
+
+constexpr int N_PLANS = 8;
+constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
+constexpr int OUT_ROWS_PER_CTA = 32;
+constexpr int NSPLIT_MAX = 8;
+constexpr int TARGET_CTAS = 2 * 148;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct PlanKey {
+  int mode;  // 0 = V, 1 = L
+  int dtype, batch, dim, n_text, has_cls, max_targets;
+  double eps;
+  std::vector<int> ntok, keep, gh, gw;
+  bool operator==(const PlanKey& o) const {
+    return mode == o.mode && dtype == o.dtype && batch == o.batch && dim == o.dim &&
+           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets &&
+           eps == o.eps && ntok == o.ntok && keep == o.keep && gh == o.gh && gw == o.gw;
+  }
+};
+
+struct Plan {
+  bool valid = false;
+  unsigned long long stamp = 0;
+  PlanKey key;
+  // device tables (inside the slot)
+  ImgDesc* d_desc = nullptr;
+  WorkItem* d_rows = nullptr;
+  WorkItem* d_corr = nullptr;
+  WorkItem* d_out = nullptr;
+  int n_rows = 0, n_corr = 0, n_out = 0;
+  // totals and maxima used to size launches and inspection copies
+  int tot_patch = 0, tot_src = 0, tot_tgt = 0, tot_out_rows = 0;
+  int max_np = 0, max_tgt = 0, max_rc = 0, max_nwin_cells = 0;
+  std::vector<ImgDesc> h_desc;
+};
+
+}  // namespace
+
+struct ficoco_ctx {
+  int device = 0;
+  long long max_tokens = 0;
+  int max_dim = 0, max_batch = 0, max_text = 0;
+  int last_cuda = 0;
+  int launches = 0;
+  unsigned long long clock = 0;
+
+  char* d_base = nullptr;
+  size_t d_bytes = 0;
+  // scratch arrays
+  float* rn = nullptr;
+  float* partial = nullptr;
+  float* s_raw = nullptr;
+  float* s_pen = nullptr;
+  int* S_idx = nullptr;
+  int* T_idx = nullptr;
+  float* part_val = nullptr;
+  int* part_idx = nullptr;
+  int* corr_cnt = nullptr;
+  int* corr_tgt = nullptr;
+  float* corr_w = nullptr;
+  float* corr_c = nullptr;
+  float* tau = nullptr;
+  int* seg_off = nullptr;
+  int* seg_src = nullptr;
+  float* seg_w = nullptr;
+  float* tmean = nullptr;
+  unsigned* status = nullptr;
+  char* plan_slots = nullptr;
+  size_t slot_bytes = 0;
+  size_t off_rows = 0, off_corr = 0, off_out = 0;
+  int cap_rows = 0, cap_corr = 0, cap_out = 0;
+  long long cap_part = 0;
+
+  char* h_stage = nullptr;  // pinned, slot_bytes
+  Plan plans[N_PLANS];
+  Plan* last_plan = nullptr;
+
+  // grow-only staging for the host-buffer entry points
+  char* hs_dev = nullptr;
+  size_t hs_dev_bytes = 0;
+  cudaStream_t hs_stream = nullptr;
+};
+
+#define CUDA_TRY(ctx, expr)                                  \
+  do {                                                       \
+    cudaError_t e__ = (expr);                                \
+    if (e__ != cudaSuccess) {                                \
+      (ctx)->last_cuda = (int)e__;                           \
+      return FICOCO_ERR_CUDA;                                \
+    }                                                        \
+  } while (0)
+
+extern "C" const char* ficoco_strerror(int code) {
+  switch (code) {
+    case FICOCO_OK: return "ok";
+    case FICOCO_ERR_INVALID_ARG: return "invalid argument";
+    case FICOCO_ERR_UNSUPPORTED: return "unsupported dtype, size or quantile level";
+    case FICOCO_ERR_KEEP_RANGE: return "keep count out of range";
+    case FICOCO_ERR_WORKSPACE: return "problem exceeds the sizes given to ficoco_create";
+    case FICOCO_ERR_CUDA: return "CUDA runtime error";
+    case FICOCO_ERR_TIMEOUT: return "device-side wait timed out";
+    case FICOCO_ERR_CAPTURE: return "a new plan cannot be uploaded during stream capture";
+    case FICOCO_ERR_GRID: return "grid smaller than the number of alive patches";
+    default: return "unknown error";
+  }
+}
+
+extern "C" void ficoco_default_params(ficoco_params* p) {
+  if (!p) return;
+  p->lambda_ = 0.35;
+  p->beta = 0.6;
+  p->gamma = 0.6;
+  p->eps = 0.998;
+  p->penalty_coef = 2.0;
+  p->window = 2;
+  p->max_targets = -1;
+  p->flags = FICOCO_HAS_CLS | FICOCO_LOCAL_PENALTY;
+  p->reserved = 0;
+}
+
+extern "C" int ficoco_last_cuda_error(const ficoco_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+extern "C" int ficoco_last_launch_count(const ficoco_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens, int max_dim,
+                             int max_batch, int max_text) {
+  if (!out || max_tokens <= 0 || max_dim <= 0 || max_batch <= 0 || max_text < 0 || device < 0)
+    return FICOCO_ERR_INVALID_ARG;
+  if (max_tokens > (1ll << 26) || max_dim > 16384) return FICOCO_ERR_UNSUPPORTED;
+  ficoco_ctx* c = new (std::nothrow) ficoco_ctx();
+  if (!c) return FICOCO_ERR_INVALID_ARG;
+  c->device = device;
+  c->max_tokens = max_tokens;
+  c->max_dim = max_dim;
+  c->max_batch = max_batch;
+  c->max_text = max_text;
+  cudaError_t e = cudaSetDevice(device);
+  if (e != cudaSuccess) { delete c; return FICOCO_ERR_CUDA; }
+
+  const size_t T = (size_t)max_tokens, B = (size_t)max_batch;
+  c->cap_rows = (int)(MAX_CHUNKS * B);
+  c->cap_corr = (int)(2 * (T / CBM + B) + 2048);
+  c->cap_out = (int)(T / OUT_ROWS_PER_CTA + B);
+  c->cap_part = (long long)T * PART_PER_TOKEN;
+  c->off_rows = align_up(B * sizeof(ImgDesc), 256);
+  c->off_corr = c->off_rows + align_up((size_t)c->cap_rows * sizeof(WorkItem), 256);
+  c->off_out = c->off_corr + align_up((size_t)c->cap_corr * sizeof(WorkItem), 256);
+  c->slot_bytes = c->off_out + align_up((size_t)c->cap_out * sizeof(WorkItem), 256);
+
+  size_t off = 0;
+  auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
+  const size_t o_rn = carve(T * 4), o_partial = carve((size_t)MAX_CHUNKS * B * max_dim * 4);
+  const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
+  const size_t o_S = carve(T * 4), o_T = carve(T * 4);
+  const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
+  const size_t o_cc = carve(T * 4), o_ct = carve(T * KCAP * 4), o_cw = carve(T * KCAP * 4);
+  const size_t o_c = carve(T * KCAP * 4), o_tau = carve(T * 4);
+  const size_t o_so = carve((T + B + 1) * 4), o_ss = carve(T * KCAP * 4), o_sw = carve(T * KCAP * 4);
+  const size_t o_tm = carve(max_text > 0 ? T * (size_t)max_text * 4 : 256);
+  const size_t o_st = carve(256);
+  const size_t o_pl = carve(c->slot_bytes * N_PLANS);
+  c->d_bytes = off;
+  e = cudaMalloc((void**)&c->d_base, c->d_bytes);
+  if (e != cudaSuccess) { c->last_cuda = (int)e; delete c; return FICOCO_ERR_CUDA; }
+  e = cudaMemset(c->d_base, 0, c->d_bytes);
+  if (e == cudaSuccess) e = cudaMallocHost((void**)&c->h_stage, c->slot_bytes);
+  if (e != cudaSuccess) { cudaFree(c->d_base); delete c; return FICOCO_ERR_CUDA; }
+  char* b = c->d_base;
+  c->rn = (float*)(b + o_rn); c->partial = (float*)(b + o_partial);
+  c->s_raw = (float*)(b + o_sraw); c->s_pen = (float*)(b + o_spen);
+  c->S_idx = (int*)(b + o_S); c->T_idx = (int*)(b + o_T);
+  c->part_val = (float*)(b + o_pv); c->part_idx = (int*)(b + o_pi);
+  c->corr_cnt = (int*)(b + o_cc); c->corr_tgt = (int*)(b + o_ct); c->corr_w = (float*)(b + o_cw);
+  c->corr_c = (float*)(b + o_c); c->tau = (float*)(b + o_tau);
+  c->seg_off = (int*)(b + o_so); c->seg_src = (int*)(b + o_ss); c->seg_w = (float*)(b + o_sw);
+  c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
+  c->plan_slots = b + o_pl;
+
+  // kernels that may need more than 48 KB of dynamic shared memory
+  cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaFuncSetAttribute(k_finalize, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024);
+  cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+  cudaGetLastError();
+  *out = c;
+  return FICOCO_OK;
+}
+
+extern "C" int ficoco_destroy(ficoco_ctx* c) {
+  if (!c) return FICOCO_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  if (c->d_base) cudaFree(c->d_base);
+  if (c->h_stage) cudaFreeHost(c->h_stage);
+  if (c->hs_dev) cudaFree(c->hs_dev);
+  if (c->hs_stream) cudaStreamDestroy(c->hs_stream);
+  delete c;
+  return FICOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Plans
+// ---------------------------------------------------------------------------------------
+namespace {
+
+int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
+  const int B = key.batch;
+  const int cls = key.mode == 0 ? key.has_cls : 0;
+  const int tail = key.mode == 1 ? key.n_text : 0;
+  p->h_desc.assign(B, ImgDesc());
+  std::vector<WorkItem> rows, corr, outw;
+  long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
+  p->max_np = p->max_tgt = p->max_rc = p->max_nwin_cells = 0;
+
+  // first pass: sizes
+  long long base_strips = 0;
+  for (int b = 0; b < B; ++b) {
+    ImgDesc& d = p->h_desc[b];
+    const int ntok = key.ntok[b];
+    const int np = ntok - cls - tail;
+    if (np < 1) return FICOCO_ERR_INVALID_ARG;
+    if (np > MAX_IMG_TOKENS) return FICOCO_ERR_UNSUPPORTED;
+    const int keep = key.keep[b];
+    if (keep < 0 || keep > np) return FICOCO_ERR_KEEP_RANGE;
+    d.n_cls = cls; d.np = np; d.n_tgt = keep; d.n_src = np - keep; d.n_tail = tail;
+    d.gh = key.gh[b]; d.gw = key.gw[b];
+    if (key.mode == 0) {
+      if (d.gh < 1 || d.gw < 1) return FICOCO_ERR_INVALID_ARG;
+      if ((long long)d.gh * d.gw < np) return FICOCO_ERR_GRID;
+      if ((long long)d.gh * d.gw > 20000) return FICOCO_ERR_UNSUPPORTED;
+    }
+    int L = 0;
+    float frac = 0.f;
+    if (key.max_targets != 0 && d.n_src > 0 && d.n_tgt > 0) {
+      if (key.max_targets > 0) {
+        L = key.max_targets < d.n_tgt ? key.max_targets : d.n_tgt;
+      } else {
+        const double q = key.eps * (double)(d.n_tgt - 1);
+        const double lo = floor(q);
+        L = d.n_tgt - (int)lo;
+        frac = (float)(q - lo);
+      }
+      if (L > KCAP) return FICOCO_ERR_UNSUPPORTED;
+    }
+    d.list_len = L;
+    d.frac = frac;
+    if (L > 0) base_strips += (d.n_src + CBM - 1) / CBM;
+  }
+  int want_split = 1;
+  if (base_strips > 0) {
+    want_split = (int)((TARGET_CTAS + base_strips - 1) / base_strips);
+    if (want_split < 1) want_split = 1;
+    if (want_split > NSPLIT_MAX) want_split = NSPLIT_MAX;
+  }
+
+  for (int b = 0; b < B; ++b) {
+    ImgDesc& d = p->h_desc[b];
+    d.row0 = (int)row0; d.patch0 = (int)patch0; d.out_row0 = (int)out0;
+    d.src0 = (int)src0; d.tgt0 = (int)tgt0; d.ent0 = (int)ent0; d.part0 = (int)part0;
+    d.attn0 = 0;  // set by the caller-specific code below
+    // row chunks
+    int rc = (d.np + MAX_CHUNKS - 1) / MAX_CHUNKS;
+    rc = (rc + 7) / 8 * 8;
+    if (rc < 64) rc = 64;
+    d.n_chunks = (d.np + rc - 1) / rc;
+    d.chunk0 = (int)chunk0;
+    for (int k = 0; k < d.n_chunks; ++k) {
+      WorkItem w; w.img = b; w.r0 = k * rc; w.nrows = (d.np - w.r0 < rc) ? d.np - w.r0 : rc; w.aux = k;
+      rows.push_back(w);
+    }
+    if (rc > p->max_rc) p->max_rc = rc;
+    // correlate
+    d.nsplit = 1; d.cols_per_split = d.n_tgt > 0 ? d.n_tgt : 1;
+    if (d.list_len > 0) {
+      int ns = want_split;
+      const int max_by_cols = (d.n_tgt + CBN - 1) / CBN;
+      if (ns > max_by_cols) ns = max_by_cols;
+      int cps = (d.n_tgt + ns - 1) / ns;
+      cps = (cps + CBN - 1) / CBN * CBN;
+      ns = (d.n_tgt + cps - 1) / cps;
+      d.nsplit = ns; d.cols_per_split = cps;
+      for (int s0 = 0; s0 < d.n_src; s0 += CBM)
+        for (int sp = 0; sp < ns; ++sp) {
+          WorkItem w; w.img = b; w.r0 = s0; w.nrows = (d.n_src - s0 < CBM) ? d.n_src - s0 : CBM; w.aux = sp;
+          corr.push_back(w);
+        }
+      part0 += (long long)d.n_src * ns * d.list_len;
+      ent0 += (long long)d.n_src * d.list_len;
+    }
+    // output rows
+    const int orows = d.n_cls + d.n_tgt + d.n_tail;
+    for (int r0 = 0; r0 < orows; r0 += OUT_ROWS_PER_CTA) {
+      WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < OUT_ROWS_PER_CTA) ? orows - r0 : OUT_ROWS_PER_CTA; w.aux = 0;
+      outw.push_back(w);
+    }
+    row0 += key.ntok[b]; patch0 += d.np; out0 += orows; src0 += d.n_src; tgt0 += d.n_tgt;
+    chunk0 += d.n_chunks;
+    if (d.np > p->max_np) p->max_np = d.np;
+    if (d.n_tgt > p->max_tgt) p->max_tgt = d.n_tgt;
+    if (key.mode == 0 && d.gh * d.gw > p->max_nwin_cells) p->max_nwin_cells = d.gh * d.gw;
+  }
+  if (row0 > c->max_tokens || B > c->max_batch || key.dim > c->max_dim || tail > c->max_text)
+    return FICOCO_ERR_WORKSPACE;
+  if ((int)rows.size() > c->cap_rows || (int)corr.size() > c->cap_corr || (int)outw.size() > c->cap_out ||
+      part0 > c->cap_part)
+    return FICOCO_ERR_WORKSPACE;
+  p->tot_patch = (int)patch0; p->tot_src = (int)src0; p->tot_tgt = (int)tgt0; p->tot_out_rows = (int)out0;
+  p->n_rows = (int)rows.size(); p->n_corr = (int)corr.size(); p->n_out = (int)outw.size();
+
+  char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
+  p->d_desc = (ImgDesc*)slot_dev;
+  p->d_rows = (WorkItem*)(slot_dev + c->off_rows);
+  p->d_corr = (WorkItem*)(slot_dev + c->off_corr);
+  p->d_out = (WorkItem*)(slot_dev + c->off_out);
+  p->key = key;
+  memcpy(c->h_stage + c->off_rows, rows.data(), rows.size() * sizeof(WorkItem));
+  memcpy(c->h_stage + c->off_corr, corr.data(), corr.size() * sizeof(WorkItem));
+  memcpy(c->h_stage + c->off_out, outw.data(), outw.size() * sizeof(WorkItem));
+  return FICOCO_OK;
+}
+
+// Finds or builds the plan for `key`.  heads_or_text scales the attention block offsets:
+// V: image b's block starts at H * patch0 floats; L: at M * b * N floats of the head-mean
+// block t.
+int get_plan(ficoco_ctx* c, const PlanKey& key, long long attn_rows, cudaStream_t stream, Plan** out) {
+  ++c->clock;
+  for (int i = 0; i < N_PLANS; ++i)
+    if (c->plans[i].valid && c->plans[i].key == key) {
+      // attention offsets depend on the head count, which is not part of the key
+      bool same = true;
+      for (int b = 0; b < key.batch && same; ++b)
+        same = c->plans[i].h_desc[b].attn0 == attn_rows * c->plans[i].h_desc[b].patch0;
+      if (same) {
+        c->plans[i].stamp = c->clock;
+        *out = &c->plans[i];
+        return FICOCO_OK;
+      }
+      c->plans[i].valid = false;
+    }
+  cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+  CUDA_TRY(c, cudaStreamIsCapturing(stream, &cs));
+  if (cs != cudaStreamCaptureStatusNone) return FICOCO_ERR_CAPTURE;
+  int slot = 0;
+  for (int i = 0; i < N_PLANS; ++i) {
+    if (!c->plans[i].valid) { slot = i; break; }
+    if (c->plans[i].stamp < c->plans[slot].stamp) slot = i;
+  }
+  // the staging buffer and the slot may still be read by work enqueued earlier
+  CUDA_TRY(c, cudaStreamSynchronize(stream));
+  Plan* p = &c->plans[slot];
+  p->valid = false;
+  int rc = build_plan(c, p, key, slot);
+  if (rc != FICOCO_OK) return rc;
+  for (int b = 0; b < key.batch; ++b) p->h_desc[b].attn0 = attn_rows * p->h_desc[b].patch0;
+  memcpy(c->h_stage, p->h_desc.data(), key.batch * sizeof(ImgDesc));
+  CUDA_TRY(c, cudaMemcpyAsync(c->plan_slots + (size_t)slot * c->slot_bytes, c->h_stage, c->slot_bytes,
+                              cudaMemcpyHostToDevice, stream));
+  CUDA_TRY(c, cudaStreamSynchronize(stream));
+  p->valid = true;
+  p->stamp = c->clock;
+  *out = p;
+  return FICOCO_OK;
+}
+
+template <class T, int VPL>
+void launch_colsum_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, cudaStream_t st) {
+  constexpr int E = VecTraits<T>::E;
+  k_colsum<T, VPL, true><<<dim3(p->n_rows, 1), 256, VPL * 32 * E * sizeof(float), st>>>(
+      tok, D, p->d_desc, p->d_rows, c->rn, c->partial);
+}
+
+// Runs the whole reduce step for tokens of type T.  `attn` is the per-head CLS attention
+// (V) or the head-mean text->vision block (L); `attn_rows` its number of rows per image.
+template <class T>
+int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn, int attn_rows,
+             float cA, const int* pos, int window, float coef, int penalty, const float* tmean, int M,
+             float gamma, T* out_tokens, int* kept_idx, int* pos_out, float* scores_out,
+             cudaStream_t st) {
+  constexpr int E = VecTraits<T>::E;
+  const int nvec = D / E;
+  const int vpl = (nvec + 31) / 32;
+  if (vpl <= 8) {
+    if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
+    else if (vpl <= 2) launch_colsum_fused<T, 2>(c, p, tok, D, st);
+    else if (vpl <= 4) launch_colsum_fused<T, 4>(c, p, tok, D, st);
+    else if (vpl <= 5) launch_colsum_fused<T, 5>(c, p, tok, D, st);
+    else launch_colsum_fused<T, 8>(c, p, tok, D, st);
+    c->launches += 1;
+  } else {
+    k_rownorm<T><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn);
+    const int slabs = (nvec + 255) / 256;
+    k_colsum<T, 8, false><<<dim3(p->n_rows, slabs), 256, 8 * 32 * E * sizeof(float), st>>>(
+        tok, D, p->d_desc, p->d_rows, c->rn, c->partial);
+    c->launches += 2;
+  }
+  k_score<T><<<p->n_rows, 256, (size_t)(D + p->max_rc) * sizeof(float), st>>>(
+      tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
+  const size_t sel_smem = align_up((size_t)p->max_np * 4, 8) + (size_t)(penalty ? p->max_nwin_cells : 0) * 8 + 16;
+  k_select<<<p->key.batch, 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
+                                                  c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
+                                                  pos_out, c->status);
+  c->launches += 2;
+  if (p->n_corr > 0) {
+    k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
+                                                   c->T_idx, tmean, M, gamma, c->part_val, c->part_idx);
+    c->launches += 1;
+  }
+  k_finalize<<<p->key.batch, 256, (size_t)(2 * p->max_tgt + 2) * sizeof(int), st>>>(
+      p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->corr_tgt, c->corr_w, c->corr_c, c->tau,
+      c->seg_off, c->seg_src, c->seg_w);
+  k_merge_compact<T><<<p->n_out, 256, 0, st>>>(tok, D, p->d_desc, p->d_out, c->S_idx, c->T_idx,
+                                               c->seg_off, c->seg_src, c->seg_w, out_tokens);
+  c->launches += 2;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { c->last_cuda = (int)e; return FICOCO_ERR_CUDA; }
+  return FICOCO_OK;
+}
+
+int check_common(const ficoco_params* prm, int dtype, int batch, int dim, int heads, const void* tokens,
+                 const void* out_tokens) {
+  if (!prm || !tokens || !out_tokens) return FICOCO_ERR_INVALID_ARG;
+  if (batch < 1 || dim < 1 || heads < 1) return FICOCO_ERR_INVALID_ARG;
+  if (dtype != FICOCO_FP32 && dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
+  const int e = dtype == FICOCO_BF16 ? 8 : 4;
+  if (dim % e != 0) return FICOCO_ERR_UNSUPPORTED;
+  if (((uintptr_t)tokens & 15) || ((uintptr_t)out_tokens & 15)) return FICOCO_ERR_INVALID_ARG;
+  if (!(prm->eps >= 0.0 && prm->eps <= 1.0) || prm->window < 1) return FICOCO_ERR_INVALID_ARG;
+  return FICOCO_OK;
+}
+
+}  // namespace
+
+extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm,
+                               void* cuda_stream) {
+  if (!c || !a) return FICOCO_ERR_INVALID_ARG;
+  int rc = check_common(prm, a->dtype, a->batch, a->dim, a->heads, a->tokens, a->out_tokens);
+  if (rc) return rc;
+  if (!a->attn || !a->grid_h || !a->grid_w || !a->keep || !a->kept_idx) return FICOCO_ERR_INVALID_ARG;
+  if ((a->n_grid != 1 && a->n_grid != a->batch) || (a->n_keep != 1 && a->n_keep != a->batch))
+    return FICOCO_ERR_INVALID_ARG;
+  if (!a->seqlens && a->n_tokens < 1) return FICOCO_ERR_INVALID_ARG;
+  if (a->batch > c->max_batch) return FICOCO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+
+  PlanKey key;
+  key.mode = 0; key.dtype = a->dtype; key.batch = a->batch; key.dim = a->dim; key.n_text = 0;
+  key.has_cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
+  key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
+  key.eps = prm->eps;
+  key.ntok.resize(a->batch); key.keep.resize(a->batch); key.gh.resize(a->batch); key.gw.resize(a->batch);
+  for (int b = 0; b < a->batch; ++b) {
+    key.ntok[b] = a->seqlens ? a->seqlens[b] : a->n_tokens;
+    key.keep[b] = a->keep[a->n_keep == 1 ? 0 : b];
+    key.gh[b] = a->grid_h[a->n_grid == 1 ? 0 : b];
+    key.gw[b] = a->grid_w[a->n_grid == 1 ? 0 : b];
+  }
+  Plan* p = nullptr;
+  rc = get_plan(c, key, a->heads, st, &p);
+  if (rc) return rc;
+  c->last_plan = p;
+  c->launches = 0;
+  const int penalty = (prm->flags & FICOCO_LOCAL_PENALTY) ? 1 : 0;
+  if (a->dtype == FICOCO_BF16)
+    return run_step<__nv_bfloat16>(c, p, (const __nv_bfloat16*)a->tokens, a->dim, a->attn, a->heads,
+                                   (float)prm->lambda_, a->pos, prm->window, (float)prm->penalty_coef,
+                                   penalty, nullptr, 0, 1.0f, (__nv_bfloat16*)a->out_tokens, a->kept_idx,
+                                   a->pos_out, a->scores_out, st);
+  return run_step<float>(c, p, (const float*)a->tokens, a->dim, a->attn, a->heads, (float)prm->lambda_,
+                         a->pos, prm->window, (float)prm->penalty_coef, penalty, nullptr, 0, 1.0f,
+                         (float*)a->out_tokens, a->kept_idx, a->pos_out, a->scores_out, st);
+}
+
+extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const ficoco_params* prm,
+                               void* cuda_stream) {
+  if (!c || !a) return FICOCO_ERR_INVALID_ARG;
+  int rc = check_common(prm, a->dtype, a->batch, a->dim, a->heads, a->tokens, a->out_tokens);
+  if (rc) return rc;
+  if (!a->attn_t2v || !a->keep || !a->kept_idx) return FICOCO_ERR_INVALID_ARG;
+  if (a->n_vision < 1 || a->n_text < 1) return FICOCO_ERR_INVALID_ARG;
+  if (a->n_keep != 1 && a->n_keep != a->batch) return FICOCO_ERR_INVALID_ARG;
+  if (a->batch > c->max_batch || a->n_text > c->max_text) return FICOCO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+
+  PlanKey key;
+  key.mode = 1; key.dtype = a->dtype; key.batch = a->batch; key.dim = a->dim; key.n_text = a->n_text;
+  key.has_cls = 0;
+  key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
+  key.eps = prm->eps;
+  key.ntok.assign(a->batch, a->n_vision + a->n_text);
+  key.keep.resize(a->batch);
+  key.gh.assign(a->batch, 1); key.gw.assign(a->batch, a->n_vision);
+  for (int b = 0; b < a->batch; ++b) key.keep[b] = a->keep[a->n_keep == 1 ? 0 : b];
+  Plan* p = nullptr;
+  rc = get_plan(c, key, a->n_text, st, &p);
+  if (rc) return rc;
+  c->last_plan = p;
+  c->launches = 0;
+  k_head_mean<<<a->batch * a->n_text, 256, 0, st>>>(a->attn_t2v, a->heads, a->n_text, a->n_vision, c->tmean);
+  c->launches += 1;
+  if (a->dtype == FICOCO_BF16)
+    return run_step<__nv_bfloat16>(c, p, (const __nv_bfloat16*)a->tokens, a->dim, c->tmean, a->n_text,
+                                   (float)prm->beta, nullptr, 1, 1.0f, 0, c->tmean, a->n_text,
+                                   (float)prm->gamma, (__nv_bfloat16*)a->out_tokens, a->kept_idx, nullptr,
+                                   a->scores_out, st);
+  return run_step<float>(c, p, (const float*)a->tokens, a->dim, c->tmean, a->n_text, (float)prm->beta,
+                         nullptr, 1, 1.0f, 0, c->tmean, a->n_text, (float)prm->gamma,
+                         (float*)a->out_tokens, a->kept_idx, nullptr, a->scores_out, st);
+}
+
+extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_status) {
+  if (!c || !device_status) return FICOCO_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+  unsigned v = 0;
+  CUDA_TRY(c, cudaMemcpyAsync(&v, c->status, 4, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaMemsetAsync(c->status, 0, 4, st));
+  CUDA_TRY(c, cudaStreamSynchronize(st));
+  *device_status = (int)v;
+  return FICOCO_OK;
+}
+
+extern "C" int ficoco_inspect(ficoco_ctx* c, int what, void* host_dst, size_t bytes, size_t* bytes_avail) {
+  if (!c || !c->last_plan) return FICOCO_ERR_INVALID_ARG;
+  const Plan* p = c->last_plan;
+  const void* src = nullptr;
+  size_t n = 0;
+  switch (what) {
+    case FICOCO_INSPECT_RNORM: src = c->rn; n = (size_t)p->tot_patch * 4; break;
+    case FICOCO_INSPECT_SCORE_RAW: src = c->s_raw; n = (size_t)p->tot_patch * 4; break;
+    case FICOCO_INSPECT_SCORE: src = c->s_pen; n = (size_t)p->tot_patch * 4; break;
+    case FICOCO_INSPECT_SRC_IDX: src = c->S_idx; n = (size_t)p->tot_src * 4; break;
+    case FICOCO_INSPECT_TGT_IDX: src = c->T_idx; n = (size_t)p->tot_tgt * 4; break;
+    case FICOCO_INSPECT_CORR_CNT: src = c->corr_cnt; n = (size_t)p->tot_src * 4; break;
+    case FICOCO_INSPECT_CORR_TGT: src = c->corr_tgt; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_CORR_W: src = c->corr_w; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_CORR_C: src = c->corr_c; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_TAU: src = c->tau; n = (size_t)p->tot_src * 4; break;
+    default: return FICOCO_ERR_INVALID_ARG;
+  }
+  if (bytes_avail) *bytes_avail = n;
+  if (!host_dst || bytes == 0) return FICOCO_OK;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+  CUDA_TRY(c, cudaDeviceSynchronize());
+  CUDA_TRY(c, cudaMemcpy(host_dst, src, bytes < n ? bytes : n, cudaMemcpyDeviceToHost));
+  return FICOCO_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Host-buffer entry points
+// ---------------------------------------------------------------------------------------
+namespace {
+
+int ensure_staging(ficoco_ctx* c, size_t dev_bytes) {
+  if (!c->hs_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->hs_stream, cudaStreamNonBlocking));
+  if (dev_bytes > c->hs_dev_bytes) {
+    if (c->hs_dev) { CUDA_TRY(c, cudaDeviceSynchronize()); cudaFree(c->hs_dev); c->hs_dev = nullptr; }
+    CUDA_TRY(c, cudaMalloc((void**)&c->hs_dev, dev_bytes));
+    c->hs_dev_bytes = dev_bytes;
+  }
+  return FICOCO_OK;
+}
+
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(char* b) : base(b) {}
+  template <class U> U* take(size_t bytes) { U* p = (U*)(base + off); off += align_up(bytes, 256); return p; }
+};
+
+}  // namespace
+
+extern "C" int ficoco_v_reduce_host(ficoco_ctx* c, const ficoco_v_args* h, const ficoco_params* prm) {
+  if (!c || !h || !prm) return FICOCO_ERR_INVALID_ARG;
+  if (!h->tokens || !h->attn || !h->keep || !h->out_tokens || !h->kept_idx || h->batch < 1 || h->dim < 1 ||
+      h->heads < 1 || (h->n_keep != 1 && h->n_keep != h->batch))
+    return FICOCO_ERR_INVALID_ARG;
+  if (h->dtype != FICOCO_FP32 && h->dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
+  const int cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
+  const size_t es = h->dtype == FICOCO_BF16 ? 2 : 4;
+  long long rows = 0, patches = 0, orows = 0, kept = 0;
+  for (int b = 0; b < h->batch; ++b) {
+    const int n = h->seqlens ? h->seqlens[b] : h->n_tokens;
+    const int k = h->keep[h->n_keep == 1 ? 0 : b];
+    if (n < cls + 1 || k < 0 || k > n - cls) return FICOCO_ERR_KEEP_RANGE;
+    rows += n; patches += n - cls; orows += cls + k; kept += k;
+  }
+  if (rows > c->max_tokens) return FICOCO_ERR_WORKSPACE;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+  const size_t b_tok = (size_t)rows * h->dim * es, b_attn = (size_t)patches * h->heads * 4;
+  const size_t b_pos = h->pos ? (size_t)patches * 4 : 0;
+  const size_t b_out = (size_t)orows * h->dim * es, b_kidx = (size_t)orows * 4;
+  const size_t b_posout = h->pos_out ? (size_t)kept * 4 : 0, b_sc = h->scores_out ? (size_t)patches * 4 : 0;
+  const size_t total = align_up(b_tok, 256) + align_up(b_attn, 256) + align_up(b_pos, 256) +
+                       align_up(b_out, 256) + align_up(b_kidx, 256) + align_up(b_posout, 256) +
+                       align_up(b_sc, 256) + 256;
+  int rc = ensure_staging(c, total);
+  if (rc) return rc;
+  Carver dv(c->hs_dev);
+  ficoco_v_args a = *h;
+  char* d_tok = dv.take<char>(b_tok);
+  char* d_attn = dv.take<char>(b_attn);
+  char* d_pos = dv.take<char>(b_pos);
+  char* d_out = dv.take<char>(b_out);
+  char* d_kidx = dv.take<char>(b_kidx);
+  char* d_po = dv.take<char>(b_posout);
+  char* d_sc = dv.take<char>(b_sc);
+  cudaStream_t st = c->hs_stream;
+  CUDA_TRY(c, cudaMemcpyAsync(d_tok, h->tokens, b_tok, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(c, cudaMemcpyAsync(d_attn, h->attn, b_attn, cudaMemcpyHostToDevice, st));
+  if (h->pos) CUDA_TRY(c, cudaMemcpyAsync(d_pos, h->pos, b_pos, cudaMemcpyHostToDevice, st));
+  a.tokens = d_tok; a.attn = (const float*)d_attn; a.pos = h->pos ? (const int*)d_pos : nullptr;
+  a.out_tokens = d_out; a.kept_idx = (int*)d_kidx;
+  a.pos_out = h->pos_out ? (int*)d_po : nullptr;
+  a.scores_out = h->scores_out ? (float*)d_sc : nullptr;
+  rc = ficoco_v_reduce(c, &a, prm, st);
+  if (rc) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(h->out_tokens, d_out, b_out, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaMemcpyAsync(h->kept_idx, d_kidx, b_kidx, cudaMemcpyDeviceToHost, st));
+  if (h->pos_out) CUDA_TRY(c, cudaMemcpyAsync(h->pos_out, d_po, b_posout, cudaMemcpyDeviceToHost, st));
+  if (h->scores_out) CUDA_TRY(c, cudaMemcpyAsync(h->scores_out, d_sc, b_sc, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaStreamSynchronize(st));
+  return FICOCO_OK;
+}
+
+extern "C" int ficoco_l_reduce_host(ficoco_ctx* c, const ficoco_l_args* h, const ficoco_params* prm) {
+  if (!c || !h || !prm) return FICOCO_ERR_INVALID_ARG;
+  if (!h->tokens || !h->attn_t2v || !h->keep || !h->out_tokens || !h->kept_idx || h->batch < 1 ||
+      h->dim < 1 || h->heads < 1 || h->n_vision < 1 || h->n_text < 1 ||
+      (h->n_keep != 1 && h->n_keep != h->batch))
+    return FICOCO_ERR_INVALID_ARG;
+  if (h->dtype != FICOCO_FP32 && h->dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
+  const size_t es = h->dtype == FICOCO_BF16 ? 2 : 4;
+  long long orows = 0;
+  for (int b = 0; b < h->batch; ++b) {
+    const int k = h->keep[h->n_keep == 1 ? 0 : b];
+    if (k < 0 || k > h->n_vision) return FICOCO_ERR_KEEP_RANGE;
+    orows += k + h->n_text;
+  }
+  const long long rows = (long long)h->batch * (h->n_vision + h->n_text);
+  if (rows > c->max_tokens) return FICOCO_ERR_WORKSPACE;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+  const size_t b_tok = (size_t)rows * h->dim * es;
+  const size_t b_attn = (size_t)h->batch * h->heads * h->n_text * h->n_vision * 4;
+  const size_t b_out = (size_t)orows * h->dim * es, b_kidx = (size_t)orows * 4;
+  const size_t b_sc = h->scores_out ? (size_t)h->batch * h->n_vision * 4 : 0;
+  const size_t total = align_up(b_tok, 256) + align_up(b_attn, 256) + align_up(b_out, 256) +
+                       align_up(b_kidx, 256) + align_up(b_sc, 256) + 256;
+  int rc = ensure_staging(c, total);
+  if (rc) return rc;
+  Carver dv(c->hs_dev);
+  char* d_tok = dv.take<char>(b_tok);
+  char* d_attn = dv.take<char>(b_attn);
+  char* d_out = dv.take<char>(b_out);
+  char* d_kidx = dv.take<char>(b_kidx);
+  char* d_sc = dv.take<char>(b_sc);
+  cudaStream_t st = c->hs_stream;
+  CUDA_TRY(c, cudaMemcpyAsync(d_tok, h->tokens, b_tok, cudaMemcpyHostToDevice, st));
+  CUDA_TRY(c, cudaMemcpyAsync(d_attn, h->attn_t2v, b_attn, cudaMemcpyHostToDevice, st));
+  ficoco_l_args a = *h;
+  a.tokens = d_tok; a.attn_t2v = (const float*)d_attn; a.out_tokens = d_out; a.kept_idx = (int*)d_kidx;
+  a.scores_out = h->scores_out ? (float*)d_sc : nullptr;
+  rc = ficoco_l_reduce(c, &a, prm, st);
+  if (rc) return rc;
+  CUDA_TRY(c, cudaMemcpyAsync(h->out_tokens, d_out, b_out, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaMemcpyAsync(h->kept_idx, d_kidx, b_kidx, cudaMemcpyDeviceToHost, st));
+  if (h->scores_out) CUDA_TRY(c, cudaMemcpyAsync(h->scores_out, d_sc, b_sc, cudaMemcpyDeviceToHost, st));
+  CUDA_TRY(c, cudaStreamSynchronize(st));
+  return FICOCO_OK;
+}

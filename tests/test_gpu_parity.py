@@ -1,0 +1,242 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 checker, element by
+element, on seeded inputs whose discrete decisions were made unambiguous beforehand."""
+import copy
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ficoco_oracle as fo, gaps
+from paper_2411_17686_b200 import binding, packing, synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(max_tokens=70000, max_dim=4096, max_batch=32, max_text=64, device=0)
+    yield c
+    c.close()
+
+
+# ---------------------------------------------------------------------------------------
+# scaled-down versions of the five workloads: several tiles, ragged tails, every stage
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("idx", [1, 2, 3, 4])
+def test_small_workloads_v(ctx, idx):
+    batch = synth.workload(idx, small=True)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what=batch.name)
+
+
+def test_small_workload_l(ctx):
+    batch = synth.workload(5, small=True)
+    gaps.repair_l(batch)
+    parity.run_and_compare_l(ctx, batch, fo.Params(), DEV, what=batch.name)
+
+
+@pytest.mark.parametrize("idx", [2, 3])
+def test_small_progressive_schedule(ctx, idx):
+    """Every step of the schedule is checked on the checker's previous output (so both
+    sides always see identical inputs), with attention regenerated and pos chained."""
+    batch = synth.workload(idx, small=True)
+    sched = synth.SCHEDULES_SMALL[idx]
+    p = fo.Params()
+    for step, keep in enumerate(sched):
+        batch.keep = [keep] * batch.batch
+        gaps.repair_v(batch)
+        _, results = parity.run_and_compare_v(ctx, batch, p, DEV, what=f"{batch.name} step {step}")
+        batch.tokens = [r.out for r in results]
+        batch.pos = [r.pos_out for r in results]
+        if step + 1 < len(sched):
+            synth.regenerate_attention(batch, 1000 * idx, step + 1, 1.5 if idx == 2 else 1.0)
+
+
+# ---------------------------------------------------------------------------------------
+# variants and edge cases
+# ---------------------------------------------------------------------------------------
+@pytest.mark.parametrize("p", [
+    fo.Params(local_penalty=False),
+    fo.Params(eps=0.97),                       # longer top lists (several targets per token)
+    fo.Params(eps=1.0),                        # tau = row maximum
+    fo.Params(max_targets=0),                  # pruning only
+    fo.Params(max_targets=2),                  # fixed K
+    fo.Params(window=3, penalty_coef=1.5),
+    fo.Params(window=1),
+    fo.Params(lam=0.8),
+], ids=["nopenalty", "eps097", "eps1", "prune", "fixedK2", "win3", "win1", "lam08"])
+def test_variants(ctx, p):
+    batch = synth.make_v_batch(77, 3, 13, 11, 192, 5, 80, "bf16", True, 1.2)
+    gaps.repair_v(batch, p)
+    parity.run_and_compare_v(ctx, batch, p, DEV, what="variant")
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("keep", [0, 1, 2, 99, 100])
+def test_edge_keep_counts(ctx, dtype, keep):
+    batch = synth.make_v_batch(78, 2, 10, 10, 64, 3, keep, dtype, True, 1.0)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what=f"keep{keep}")
+
+
+def test_no_cls_and_holes_in_pos(ctx):
+    batch = synth.make_v_batch(79, 2, 12, 12, 128, 4, 50, "bf16", False, 1.0)
+    # drop a third of the grid cells so windows are partially or completely empty
+    for b in range(2):
+        alive = np.sort(synth.rng_for(79, b, 8).permutation(144)[:96]).astype(np.int32)
+        batch.tokens[b] = batch.tokens[b][alive]
+        batch.attn[b] = batch.attn[b][:, alive].copy()
+        batch.pos[b] = alive
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="holes")
+
+
+@pytest.mark.parametrize("dim", [8, 72, 1280, 2048, 4096])
+def test_hidden_sizes(ctx, dim):
+    batch = synth.make_v_batch(80, 2, 6, 7, dim, 2, 20, "bf16", True, 1.0)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what=f"dim{dim}")
+
+
+def test_fp32_wide_rows(ctx):
+    batch = synth.make_v_batch(81, 1, 6, 6, 2052, 2, 20, "fp32", True, 1.0)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="fp32-wide")
+
+
+def test_l_variants(ctx):
+    for p in (fo.Params(gamma=1.0), fo.Params(beta=1.0), fo.Params(eps=0.9), fo.Params(max_targets=0)):
+        batch = synth.make_l_batch(82, 2, 100, 9, 256, 3, 30, "bf16", scale=1.0 / 16)
+        gaps.repair_l(batch, p)
+        parity.run_and_compare_l(ctx, batch, p, DEV, what="l-variant")
+    batch = synth.make_l_batch(83, 1, 70, 5, 128, 2, 20, "fp32", scale=1.0)
+    gaps.repair_l(batch)
+    parity.run_and_compare_l(ctx, batch, fo.Params(), DEV, what="l-fp32")
+
+
+def test_run_to_run_determinism_and_host_entry_point(ctx):
+    batch = synth.workload(2, small=True)
+    gaps.repair_v(batch)
+    pk = packing.pack_v(batch, DEV)
+    a = ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **pk.call_kwargs())
+    a_out, a_idx = binding.to_numpy(a.out_tokens), binding.to_numpy(a.kept_idx)
+    b = ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **pk.call_kwargs())
+    assert np.array_equal(a_out, binding.to_numpy(b.out_tokens))
+    assert np.array_equal(a_idx, binding.to_numpy(b.kept_idx))
+    ph = packing.pack_v(batch, None, pin=True)
+    h = ctx.ficoco_v_reduce_host(ph.tokens, ph.attn, ph.keep, ph.grid_h, ph.grid_w, ph.heads, **ph.call_kwargs())
+    assert np.array_equal(a_out, binding.to_numpy(h.out_tokens))
+    assert np.array_equal(a_idx, binding.to_numpy(h.kept_idx))
+    lb = synth.workload(5, small=True)
+    gaps.repair_l(lb)
+    pl = packing.pack_l(lb, DEV)
+    d = ctx.ficoco_l_reduce(pl.tokens, pl.attn_t2v, pl.keep, pl.n_vision, pl.n_text, pl.heads)
+    plh = packing.pack_l(lb, None, pin=True)
+    hh = ctx.ficoco_l_reduce_host(plh.tokens, plh.attn_t2v, plh.keep, plh.n_vision, plh.n_text, plh.heads)
+    assert np.array_equal(binding.to_numpy(d.out_tokens), binding.to_numpy(hh.out_tokens))
+    assert np.array_equal(binding.to_numpy(d.kept_idx), binding.to_numpy(hh.kept_idx))
+
+
+def test_canaries_around_outputs(ctx):
+    """Nothing is written outside the documented output extents."""
+    batch = synth.workload(4, small=True)
+    gaps.repair_v(batch)
+    pk = packing.pack_v(batch, DEV)
+    rows = sum(pk.keep)
+    pad = 64
+    out = torch.full((rows + 2 * pad, batch.dim), 7.0, dtype=torch.bfloat16, device=DEV)
+    kidx = torch.full((rows + 2 * pad,), -7, dtype=torch.int32, device=DEV)
+    pout = torch.full((rows + 2 * pad,), -7, dtype=torch.int32, device=DEV)
+    ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads,
+                        params=binding.make_params(has_cls=False),
+                        out_tokens=out[pad:pad + rows], kept_idx=kidx[pad:pad + rows],
+                        pos_out=pout[pad:pad + rows], **pk.call_kwargs())
+    torch.cuda.synchronize()
+    for t, v in ((out, 7.0), (kidx, -7), (pout, -7)):
+        assert bool((t[:pad] == v).all()) and bool((t[pad + rows:] == v).all())
+    assert bool((kidx[pad:pad + rows] >= 0).all())
+
+
+def test_error_codes_and_status(ctx):
+    batch = synth.make_v_batch(84, 2, 6, 6, 64, 2, 20, "bf16", True, 1.0)
+    pk = packing.pack_v(batch, DEV)
+    kw = pk.call_kwargs()
+
+    def call(**over):
+        args = dict(tokens=pk.tokens, attn=pk.attn, keep=pk.keep, grid_h=pk.grid_h, grid_w=pk.grid_w,
+                    heads=pk.heads)
+        args.update(kw)
+        args.update(over)
+        return ctx.ficoco_v_reduce(**args)
+
+    with pytest.raises(binding.FicocoError) as e:
+        call(keep=[37, 20])
+    assert e.value.code == -3
+    with pytest.raises(binding.FicocoError) as e:
+        call(grid_h=[5, 5])
+    assert e.value.code == -8
+    with pytest.raises(binding.FicocoError) as e:
+        call(params=binding.make_params(eps=0.5))      # top list of 11 of 20 fits; eps=0.1 does not
+        call(params=binding.make_params(eps=0.1))
+    assert e.value.code == -2
+    with pytest.raises(binding.FicocoError) as e:
+        call(params=binding.make_params(eps=1.5))
+    assert e.value.code == -1
+    small = binding.Context(max_tokens=50, max_dim=64, max_batch=2)
+    with pytest.raises(binding.FicocoError) as e:
+        small.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **kw)
+    assert e.value.code == -4
+    small.close()
+    odd = torch.zeros((74, 12), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(binding.FicocoError) as e:
+        ctx.ficoco_v_reduce(odd, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, n_tokens=37)
+    assert e.value.code == -2
+    # a position outside the grid is reported through the status word, not a fault
+    bad = pk.pos.clone()
+    bad[5] = 36 + 1000
+    call(pos=bad)
+    assert ctx.ficoco_status() == 1
+    call()
+    assert ctx.ficoco_status() == 0
+
+
+# ---------------------------------------------------------------------------------------
+# full-size workloads, in the launch configuration the benchmark times
+# ---------------------------------------------------------------------------------------
+def test_full_c1(ctx):
+    batch = synth.workload(1)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="c1")
+
+
+def test_full_c2_schedule(ctx):
+    batch = synth.workload(2)
+    p = fo.Params()
+    for step, keep in enumerate(synth.SCHEDULES[2]):
+        batch.keep = [keep] * batch.batch
+        gaps.repair_v(batch)
+        _, results = parity.run_and_compare_v(ctx, batch, p, DEV, what=f"c2 step {step}")
+        batch.tokens = [r.out for r in results]
+        batch.pos = [r.pos_out for r in results]
+        if step + 1 < 3:
+            synth.regenerate_attention(batch, 2000, step + 1, 1.5)
+
+
+def test_full_c3_first_step(ctx):
+    batch = synth.workload(3)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="c3")
+
+
+def test_full_c4(ctx):
+    batch = synth.workload(4)
+    gaps.repair_v(batch)
+    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="c4")
+
+
+def test_full_c5(ctx):
+    batch = synth.workload(5)
+    gaps.repair_l(batch)
+    parity.run_and_compare_l(ctx, batch, fo.Params(), DEV, what="c5")
