@@ -79,12 +79,15 @@ def margins(res: fo.StepResult, pos: Optional[np.ndarray], grid: Optional[Tuple[
             v = np.sort(C[i])
             if p.max_targets is None:
                 tau = res.tau[i]
-                d = np.abs(v - tau)
-                g = float(d.min())
-                # also the two order statistics the interpolation uses must be distinct
                 q = p.eps * (nt - 1)
                 lo = int(np.floor(q)); hi = min(lo + 1, nt - 1)
-                if hi > lo:
+                if q == lo:
+                    # tau is the order statistic v[lo] itself (it passes by equality on both
+                    # sides); what must be unambiguous is which element holds that rank
+                    g = float(v[lo] - v[lo - 1]) if lo >= 1 else np.inf
+                else:
+                    g = float(np.abs(v - tau).min())
+                    # the two order statistics the interpolation uses must be distinct
                     g = min(g, float(v[hi] - v[lo]))
             else:
                 k = min(p.max_targets, nt)
@@ -102,6 +105,8 @@ def ok(m: Margins) -> bool:
 def _band(res: fo.StepResult, m: Margins, rng: np.random.Generator, coeff: float):
     """Preserved tokens whose score lies within 1.5 * SEL_GAP of the last discarded one,
     with the attention increase that takes each of them below that band."""
+    if coeff < 1e-3:
+        raise ValueError("the attention term has (almost) no weight in the score: it cannot move the boundary")
     s_hi = res.score[m.sel_pair[0]]
     out = []
     for j in res.T.tolist():

@@ -107,7 +107,7 @@ def test_fp32_wide_rows(ctx):
 
 
 def test_l_variants(ctx):
-    for p in (fo.Params(gamma=1.0), fo.Params(beta=1.0), fo.Params(eps=0.9), fo.Params(max_targets=0)):
+    for p in (fo.Params(gamma=1.0), fo.Params(beta=0.9), fo.Params(eps=0.9), fo.Params(max_targets=0)):
         batch = synth.make_l_batch(82, 2, 100, 9, 256, 3, 30, "bf16", scale=1.0 / 16)
         gaps.repair_l(batch, p)
         parity.run_and_compare_l(ctx, batch, p, DEV, what="l-variant")
