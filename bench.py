@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the FiCoCo-V reduce step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole reduce step (filter, correlate, compress, compact) over one
+batch of 32 synthetic images of 577 x 1024 bf16 tokens, reducing 576 -> 288 patch tokens.
+Rank 0 prints one JSON line.  With N > 1 every rank reduces its own batch (images are
+independent, there is no collective on the data path) and the value is the aggregate.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "images/sec of FiCoCo-V reduce step, B=32x577x1024 bf16"
+UNIT = "images/s"
+B, GH, GW, D, H, KEEP = 32, 24, 24, 1024, 16, 288
+WORKLOAD = "c2 step 1: 32 images x (1 CLS + 24x24 patches) x 1024 bf16, 576 -> 288 patch tokens"
+N_INSTANCES = 8       # distinct input/output buffer sets cycled through: 8 x 58 MB > 3 x L2
+
+
+def algorithmic_bytes() -> dict:
+    """Per-step algorithmic HBM traffic: read X once, read attention, write the output, plus
+    the index arrays (pos in, kept_idx and pos_out out)."""
+    n, npatch = 1 + GH * GW, GH * GW
+    x_in = B * n * D * 2
+    attn = B * H * npatch * 4
+    out = B * (1 + KEEP) * D * 2
+    idx = B * 4 * (npatch + 2 * KEEP)
+    return {"tokens_in": x_in, "attn": attn, "tokens_out": out, "index": idx,
+            "total": x_in + attn + out + idx}
+
+
+def peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index),
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx = float(f[1])
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def make_instances(rank: int):
+    """One generated batch, laid out N_INSTANCES times with the image order rotated, so every
+    step reads and writes memory that is not in L2 from the step before."""
+    from paper_2411_17686_b200 import synth
+    batch = synth.make_v_batch(2000 + rank, B, GH, GW, D, H, KEEP, "bf16", True, 1.5, name="c2")
+    return batch
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    from paper_2411_17686_b200 import binding, build, packing
+    build.build()
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    batch = make_instances(rank)
+    n = 1 + GH * GW
+    base = packing.pack_v(batch, None)
+    tok_h = base.tokens.view(B, n, D)
+    attn_h = base.attn.view(B, H, GH * GW)
+    insts = []
+    for k in range(N_INSTANCES):
+        perm = [(b + k) % B for b in range(B)]
+        insts.append(dict(
+            tokens=tok_h[perm].reshape(B * n, D).contiguous().to(dev),
+            attn=attn_h[perm].reshape(-1).contiguous().to(dev),
+            pos=base.pos.to(dev),
+            out=torch.empty((B * (1 + KEEP), D), dtype=torch.bfloat16, device=dev),
+            kidx=torch.empty((B * (1 + KEEP),), dtype=torch.int32, device=dev),
+            pout=torch.empty((B * KEEP,), dtype=torch.int32, device=dev)))
+    ctx = binding.Context(max_tokens=B * n, max_dim=D, max_batch=B, device=local_rank)
+    prm = binding.ficoco_default_params()
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i: int):
+        it = insts[i % N_INSTANCES]
+        ctx.ficoco_v_reduce(it["tokens"], it["attn"], KEEP, GH, GW, H, n_tokens=n, pos=it["pos"], params=prm,
+                            out_tokens=it["out"], kept_idx=it["kidx"], pos_out=it["pout"],
+                            stream=stream.cuda_stream)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for i in range(max(args.warmup, 3)):
+            step(i)
+    torch.cuda.synchronize()
+    launches_per_step = ctx.ficoco_last_launch_count()
+
+    # optional CUDA graph over one cycle of the instances (launch overhead off the GPU timeline)
+    graph = None
+    if args.graph and args.steps % N_INSTANCES == 0:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for i in range(N_INSTANCES):
+                step(i)
+        graph.replay()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        if graph is not None:
+            for _ in range(args.steps // N_INSTANCES):
+                graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
+        e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * B / (ms_per_step * 1e-3)
+
+    if rank != 0:
+        return None
+
+    # per-kernel durations, measured live with events between the launches of the same steps
+    ctx.ficoco_profile(True)
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            step(i)
+    torch.cuda.synchronize()
+    prof = ctx.ficoco_profile_read()
+    ctx.ficoco_profile(False)
+    kern = {nm: {"avg_us": 1e3 * t / max(cnt, 1), "launches_per_step": cnt / args.steps} for nm, t, cnt in prof}
+    tot_us = sum(v["avg_us"] * v["launches_per_step"] for v in kern.values())
+    for v in kern.values():
+        v["share"] = v["avg_us"] * v["launches_per_step"] / tot_us if tot_us else 0.0
+    dom = max(kern, key=lambda k: kern[k]["share"])
+
+    pk = peaks()
+    ab = algorithmic_bytes()
+    roof = kernel_roofline(dom, kern[dom]["avg_us"], pk, ab)
+    t_roof_us = max(ab["total"] / (pk["hbm_gbs"] * 1e3), 2.0 * B * (GH * GW - KEEP) * KEEP * D / (pk["bf16_tflops"] * 1e6))
+
+    # end to end through the host-buffer entry point (pinned host tensors, copies inside)
+    hp = packing.pack_v(batch, None, pin=True)
+    out_h = torch.empty((B * (1 + KEEP), D), dtype=torch.bfloat16).pin_memory()
+    kidx_h = torch.empty((B * (1 + KEEP),), dtype=torch.int32).pin_memory()
+    e2e_steps = max(5, min(args.steps, 50))
+    for _ in range(3):
+        ctx.ficoco_v_reduce_host(hp.tokens, hp.attn, KEEP, GH, GW, H, n_tokens=n, pos=hp.pos, params=prm,
+                                 out_tokens=out_h, kept_idx=kidx_h)
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctx.ficoco_v_reduce_host(hp.tokens, hp.attn, KEEP, GH, GW, H, n_tokens=n, pos=hp.pos, params=prm,
+                                 out_tokens=out_h, kept_idx=kidx_h)
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    h2d = hp.tokens.numel() * 2 + hp.attn.numel() * 4 + hp.pos.numel() * 4
+    d2h = out_h.numel() * 2 + kidx_h.numel() * 4
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch_per_gpu": B, "tokens_per_image": n, "dim": D, "heads": H,
+                   "keep": KEEP, "l2": f"inputs larger than L2: {N_INSTANCES} buffer sets cycled",
+                   "cuda_graph": graph is not None},
+        "tokens_per_s": value * n,
+        "clocks": clocks,
+        "e2e": {"value": world * B / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roof,
+        "step_roofline": {"bound": "hbm" if ab["total"] / (pk["hbm_gbs"] * 1e3) >= t_roof_us - 1e-9 else "tensor",
+                          "t_roof_us": t_roof_us, "t_measured_us": ms_per_step * 1e3,
+                          "frac": t_roof_us / (ms_per_step * 1e3), "algorithmic_bytes": ab["total"],
+                          "peak": f"{pk['source']} {pk['hbm_gbs']} GB/s, {pk['bf16_tflops']} TFLOP/s bf16"},
+        "kernels": kern,
+    }
+    line["cpu_baseline"] = cpu_baseline(batch, budget_s=args.cpu_budget)
+    ctx.close()
+    return line
+
+
+def kernel_roofline(name: str, avg_us: float, pk: dict, ab: dict) -> dict:
+    """Roofline entry of the dominant kernel: its own algorithmic bytes (or flops) per launch
+    over its measured average duration."""
+    npatch, ns = GH * GW, GH * GW - KEEP
+    src = pk["source"]
+    if name == "correlate":
+        flops = 2.0 * B * ns * KEEP * D
+        ach = flops / (avg_us * 1e-6) / 1e12
+        return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": ach / pk["bf16_tflops"], "traffic": None, "of": src,
+                "algorithmic_flops_per_launch": flops}
+    per = {
+        "colsum": ab["tokens_in"],                                   # X read once from HBM
+        "score": ab["tokens_in"] + ab["attn"],                       # X again (L2-resident) + attention
+        "merge_compact": ab["tokens_out"] * 2,                       # rows in, rows out
+        "select": B * npatch * 4 * 3, "finalize": B * ns * 16, "rownorm": ab["tokens_in"],
+    }.get(name, ab["total"])
+    ach = per / (avg_us * 1e-6) / 1e9
+    return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+            "frac": ach / pk["hbm_gbs"], "traffic": None, "of": src, "algorithmic_bytes_per_launch": per}
+
+
+def cpu_baseline(batch, budget_s: float = 12.0) -> dict:
+    """The float64 checker as it stands, on the host cores, over whole batches of the same
+    workload until the time budget is used."""
+    from oracle import ficoco_oracle as fo
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+    done, t0 = 0, time.perf_counter()
+    while True:
+        for b in range(batch.batch):
+            fo.ficoco_v_reduce(batch.tokens[b], batch.attn[b], batch.pos[b], batch.grid[b], batch.keep[b], True)
+            done += 1
+            if time.perf_counter() - t0 > budget_s:
+                break
+        if time.perf_counter() - t0 > budget_s:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": done / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{done} images of the same workload in {dt:.1f} s (numpy float64)"}
+
+
+def run_reference(args, rank: int):
+    """Reference arm: the float64 checker on the host cores, each step a bounded sample
+    (4 images) of the workload."""
+    if rank != 0:
+        return None
+    from oracle import ficoco_oracle as fo
+    batch = make_instances(0)
+    sample = 4
+    cores = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        pass
+
+    def step(i):
+        for b in range(sample):
+            k = (i * sample + b) % batch.batch
+            fo.ficoco_v_reduce(batch.tokens[k], batch.attn[k], batch.pos[k], batch.grid[k], batch.keep[k], True)
+
+    for i in range(max(1, min(args.warmup, 3))):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(i)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample_per_step": f"{sample} of {B} images"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} images per step, {args.steps} steps"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", dest="graph", action="store_false")
+    ap.add_argument("--cpu-budget", type=float, default=12.0)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        args.steps = args.steps if args.steps is not None else 20
+        args.warmup = args.warmup if args.warmup is not None else 2
+        line = run_reference(args, rank)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return
+    args.steps = args.steps if args.steps is not None else 2000
+    args.warmup = args.warmup if args.warmup is not None else 10
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    line = run_ours(args, rank, world, local_rank)
+    if line is not None:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

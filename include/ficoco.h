@@ -208,6 +208,19 @@ int ficoco_inspect(ficoco_ctx* ctx, int what, void* host_dst, size_t bytes, size
 /* Number of kernels the most recent reduce call launched (for launch accounting). */
 int ficoco_last_launch_count(const ficoco_ctx* ctx);
 
+/*
+ * Per-kernel timing.  ficoco_profile(ctx, 1) clears the accumulators and makes every later
+ * reduce call record a CUDA event in front of each kernel it launches (on the call's stream)
+ * and one after the last; ficoco_profile(ctx, 0) stops that.  Do not enable it during stream
+ * capture.  ficoco_profile_read synchronises the device, folds the recorded intervals into
+ * per-kernel totals and returns entry `index` (kernels in first-launch order): its name
+ * (NUL-terminated, at most name_cap bytes), the summed milliseconds and the launch count.
+ * It returns FICOCO_ERR_INVALID_ARG once `index` is past the last entry.
+ */
+int ficoco_profile(ficoco_ctx* ctx, int enable);
+int ficoco_profile_read(ficoco_ctx* ctx, int index, char* name, int name_cap, double* total_ms,
+                        long long* launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,6 +31,7 @@ EXPORTS = [
     "ficoco_create", "ficoco_destroy", "ficoco_strerror", "ficoco_last_cuda_error",
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
+    "ficoco_profile", "ficoco_profile_read",
 ]
 
 
@@ -89,6 +90,9 @@ def load_library() -> C.CDLL:
     lib.ficoco_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
     lib.ficoco_inspect.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.ficoco_last_launch_count.argtypes = [C.c_void_p]
+    lib.ficoco_profile.argtypes = [C.c_void_p, C.c_int]
+    lib.ficoco_profile_read.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_int, C.POINTER(C.c_double),
+                                        C.POINTER(C.c_longlong)]
     _lib = lib
     return lib
 
@@ -312,6 +316,22 @@ class Context:
 
     def ficoco_last_launch_count(self) -> int:
         return int(self.lib.ficoco_last_launch_count(self.h))
+
+    def ficoco_profile(self, enable: bool) -> None:
+        _check(self.h, self.lib.ficoco_profile(self.h, 1 if enable else 0))
+
+    def ficoco_profile_read(self):
+        """[(kernel name, total ms, launches), ...] since profiling was enabled."""
+        out = []
+        i = 0
+        while True:
+            name = C.create_string_buffer(64)
+            ms, n = C.c_double(0), C.c_longlong(0)
+            if self.lib.ficoco_profile_read(self.h, i, name, 64, C.byref(ms), C.byref(n)) != 0:
+                break
+            out.append((name.value.decode(), ms.value, n.value))
+            i += 1
+        return out
 
 
 # ----------------------------------------------------------------------------------------

@@ -95,6 +95,14 @@ struct ficoco_ctx {
   Plan plans[N_PLANS];
   Plan* last_plan = nullptr;
 
+  // optional per-kernel timing (events recorded between launches)
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev;
+  size_t prof_used = 0;
+  std::vector<int> prof_name;            // per recorded event: index into prof_acc, -1 = end of call
+  struct ProfAcc { const char* name; double ms; long long launches; };
+  std::vector<ProfAcc> prof_acc;
+
   // grow-only staging for the host-buffer entry points
   char* hs_dev = nullptr;
   size_t hs_dev_bytes = 0;
@@ -109,6 +117,68 @@ struct ficoco_ctx {
       return FICOCO_ERR_CUDA;                                \
     }                                                        \
   } while (0)
+
+namespace {
+
+// Record an event in front of the kernel about to be launched (name) or at the end of a
+// call (nullptr).  The time between two consecutive events is attributed to the first.
+void prof_tick(ficoco_ctx* c, cudaStream_t st, const char* name) {
+  if (!c->prof_on) return;
+  if (c->prof_used == c->prof_ev.size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    c->prof_ev.push_back(e);
+  }
+  int idx = -1;
+  if (name) {
+    for (size_t i = 0; i < c->prof_acc.size(); ++i)
+      if (c->prof_acc[i].name == name) idx = (int)i;
+    if (idx < 0) { c->prof_acc.push_back({name, 0.0, 0}); idx = (int)c->prof_acc.size() - 1; }
+  }
+  cudaEventRecord(c->prof_ev[c->prof_used], st);
+  if (c->prof_name.size() <= c->prof_used) c->prof_name.resize(c->prof_used + 1);
+  c->prof_name[c->prof_used] = idx;
+  ++c->prof_used;
+}
+
+void prof_flush(ficoco_ctx* c) {
+  if (c->prof_used == 0) return;
+  cudaDeviceSynchronize();
+  for (size_t i = 0; i + 1 < c->prof_used; ++i) {
+    const int idx = c->prof_name[i];
+    if (idx < 0) continue;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[i], c->prof_ev[i + 1]) == cudaSuccess) {
+      c->prof_acc[idx].ms += ms;
+      c->prof_acc[idx].launches += 1;
+    }
+  }
+  c->prof_used = 0;
+}
+
+}  // namespace
+
+extern "C" int ficoco_profile(ficoco_ctx* c, int enable) {
+  if (!c) return FICOCO_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  c->prof_used = 0;
+  c->prof_acc.clear();
+  c->prof_on = enable != 0;
+  return FICOCO_OK;
+}
+
+extern "C" int ficoco_profile_read(ficoco_ctx* c, int index, char* name, int name_cap, double* total_ms,
+                                   long long* launches) {
+  if (!c || index < 0 || !name || name_cap < 2 || !total_ms || !launches) return FICOCO_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  prof_flush(c);
+  if (index >= (int)c->prof_acc.size()) return FICOCO_ERR_INVALID_ARG;
+  strncpy(name, c->prof_acc[index].name, name_cap - 1);
+  name[name_cap - 1] = 0;
+  *total_ms = c->prof_acc[index].ms;
+  *launches = c->prof_acc[index].launches;
+  return FICOCO_OK;
+}
 
 extern "C" const char* ficoco_strerror(int code) {
   switch (code) {
@@ -213,6 +283,7 @@ extern "C" int ficoco_destroy(ficoco_ctx* c) {
   if (c->h_stage) cudaFreeHost(c->h_stage);
   if (c->hs_dev) cudaFree(c->hs_dev);
   if (c->hs_stream) cudaStreamDestroy(c->hs_stream);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return FICOCO_OK;
 }
@@ -398,6 +469,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
+  prof_tick(c, st, vpl <= 8 ? "colsum" : "rownorm");
   if (vpl <= 8) {
     if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
     else if (vpl <= 2) launch_colsum_fused<T, 2>(c, p, tok, D, st);
@@ -407,29 +479,37 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     c->launches += 1;
   } else {
     k_rownorm<T><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn);
+    prof_tick(c, st, "colsum");
     const int slabs = (nvec + 255) / 256;
     k_colsum<T, 8, false><<<dim3(p->n_rows, slabs), 256, 8 * 32 * E * sizeof(float), st>>>(
         tok, D, p->d_desc, p->d_rows, c->rn, c->partial);
     c->launches += 2;
   }
+  prof_tick(c, st, "score");
   k_score<T><<<p->n_rows, 256, (size_t)(D + p->max_rc) * sizeof(float), st>>>(
       tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
   const size_t sel_smem = align_up((size_t)p->max_np * 4, 8) + (size_t)(penalty ? p->max_nwin_cells : 0) * 8 + 16;
+  prof_tick(c, st, "select");
   k_select<<<p->key.batch, 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
                                                   pos_out, c->status);
   c->launches += 2;
   if (p->n_corr > 0) {
+    prof_tick(c, st, "correlate");
     k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
                                                    c->T_idx, tmean, M, gamma, c->part_val, c->part_idx);
     c->launches += 1;
   }
+  prof_tick(c, st, "finalize");
   k_finalize<<<p->key.batch, 256, (size_t)(2 * p->max_tgt + 2) * sizeof(int), st>>>(
       p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->corr_tgt, c->corr_w, c->corr_c, c->tau,
       c->seg_off, c->seg_src, c->seg_w);
+  prof_tick(c, st, "merge_compact");
   k_merge_compact<T><<<p->n_out, 256, 0, st>>>(tok, D, p->d_desc, p->d_out, c->S_idx, c->T_idx,
                                                c->seg_off, c->seg_src, c->seg_w, out_tokens);
   c->launches += 2;
+  prof_tick(c, st, nullptr);
+  if (c->prof_used > 60000) prof_flush(c);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { c->last_cuda = (int)e; return FICOCO_ERR_CUDA; }
   return FICOCO_OK;
@@ -516,6 +596,7 @@ extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const fico
   if (rc) return rc;
   c->last_plan = p;
   c->launches = 0;
+  prof_tick(c, st, "head_mean");
   k_head_mean<<<a->batch * a->n_text, 256, 0, st>>>(a->attn_t2v, a->heads, a->n_text, a->n_vision, c->tmean);
   c->launches += 1;
   if (a->dtype == FICOCO_BF16)
