@@ -62,7 +62,8 @@ enum ficoco_error {
   FICOCO_ERR_CUDA = -5,          /* a CUDA runtime call failed (see ficoco_last_cuda_error) */
   FICOCO_ERR_TIMEOUT = -6,       /* a bounded device-side wait ran out */
   FICOCO_ERR_CAPTURE = -7,       /* a new plan would have to be uploaded during stream capture */
-  FICOCO_ERR_GRID = -8           /* grid_h * grid_w smaller than the number of alive patches */
+  FICOCO_ERR_GRID = -8,          /* grid_h * grid_w smaller than the number of alive patches */
+  FICOCO_ERR_STATIC_LIMIT = -9   /* problem larger than the fixed scratch of the allocation-free entry point */
 };
 
 enum ficoco_flags {
@@ -220,6 +221,39 @@ int ficoco_last_launch_count(const ficoco_ctx* ctx);
 int ficoco_profile(ficoco_ctx* ctx, int enable);
 int ficoco_profile_read(ficoco_ctx* ctx, int index, char* name, int name_cap, double* total_ms,
                         long long* launches);
+
+/*
+ * Allocation-free vision-aware redundancy.  (The paper has no counterpart to this entry
+ * point: it exists for callers of this library that are not allowed to allocate.)
+ *
+ * For a uniform batch it writes, for every patch token, v_i = (1/Np) sum_j cos(x_i, x_j) over
+ * the alive patches of its image (j = i included): the first term of Eq. 1, the same numbers
+ * ficoco_v_reduce produces as scores when lambda = 1 and the local penalty is off.
+ *
+ * It needs no context and calls neither cudaMalloc nor cudaFree nor anything else that
+ * allocates.  It is meant for code that runs where device allocation is off limits, typically
+ * the per-step callback of a serving engine that gave all device memory to its own pool at
+ * start-up: there a cudaMalloc can fail, and it synchronises the whole device.  Its scratch
+ * (inverse norms and column-sum partials, about 4.7 MB) is a fixed array inside the library,
+ * held by every GPU that loads the library until the process exits.  Hence:
+ *   - limits: batch <= FICOCO_NOALLOC_MAX_BATCH, dim <= FICOCO_NOALLOC_MAX_DIM,
+ *     batch * Np <= FICOCO_NOALLOC_MAX_ROWS; anything larger returns FICOCO_ERR_STATIC_LIMIT
+ *     and launches nothing;
+ *   - all calls on one device share the array and it keeps the previous call's contents;
+ *     every word a call reads it has written itself first, so nothing needs clearing, but two
+ *     calls that overlap on the GPU (different streams, no ordering) race on it;
+ *   - the first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ * The device that owns `tokens`, `v_out` and `cuda_stream` must be the calling thread's
+ * current device.  tokens: device, [batch, n_tokens, dim] (n_tokens includes the CLS row when
+ * flags has FICOCO_HAS_CLS), 16-byte aligned rows; v_out: device fp32 [batch, Np].  Work is
+ * enqueued on cuda_stream; the call does not synchronise.
+ */
+#define FICOCO_NOALLOC_MAX_ROWS 32768
+#define FICOCO_NOALLOC_MAX_BATCH 64
+#define FICOCO_NOALLOC_MAX_DIM 2048
+int ficoco_vision_redundancy_noalloc(const void* tokens, int dtype, int batch, int n_tokens, int dim,
+                                     unsigned flags, float* v_out, void* cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -31,7 +31,7 @@ EXPORTS = [
     "ficoco_create", "ficoco_destroy", "ficoco_strerror", "ficoco_last_cuda_error",
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
-    "ficoco_profile", "ficoco_profile_read",
+    "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
 ]
 
 
@@ -93,6 +93,8 @@ def load_library() -> C.CDLL:
     lib.ficoco_profile.argtypes = [C.c_void_p, C.c_int]
     lib.ficoco_profile_read.argtypes = [C.c_void_p, C.c_int, C.c_char_p, C.c_int, C.POINTER(C.c_double),
                                         C.POINTER(C.c_longlong)]
+    lib.ficoco_vision_redundancy_noalloc.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint,
+                                                     C.c_void_p, C.c_void_p]
     _lib = lib
     return lib
 
@@ -332,6 +334,28 @@ class Context:
             out.append((name.value.decode(), ms.value, n.value))
             i += 1
         return out
+
+
+def ficoco_vision_redundancy_noalloc(tokens, n_tokens: int, has_cls: bool = True, v_out=None,
+                                     stream: Optional[int] = None):
+    """First term of Eq. 1 for a uniform batch, for callers that may not allocate device memory
+    (for example a serving engine's step callback whose engine owns all of it): no context, the
+    scratch is a fixed array inside the library.  ``tokens``: cuda tensor [batch * n_tokens, D];
+    ``v_out``: cuda fp32 [batch * Np], which the caller should pass in (it is only created here,
+    with torch, as a convenience for tests).  Limits and sharing rules: see ficoco.h."""
+    import torch
+    lib = load_library()
+    batch = tokens.shape[0] // n_tokens
+    np_ = n_tokens - (1 if has_cls else 0)
+    if v_out is None:
+        v_out = torch.empty((batch * np_,), dtype=torch.float32, device=tokens.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(tokens.device).cuda_stream
+    rc = lib.ficoco_vision_redundancy_noalloc(tokens.data_ptr(), _dtype_code(tokens), batch, n_tokens,
+                                              tokens.shape[-1], FICOCO_HAS_CLS if has_cls else 0,
+                                              v_out.data_ptr(), C.c_void_p(stream))
+    _check(None, rc)
+    return v_out
 
 
 # ----------------------------------------------------------------------------------------

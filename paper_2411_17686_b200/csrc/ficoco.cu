@@ -191,6 +191,9 @@ extern "C" const char* ficoco_strerror(int code) {
     case FICOCO_ERR_TIMEOUT: return "device-side wait timed out";
     case FICOCO_ERR_CAPTURE: return "a new plan cannot be uploaded during stream capture";
     case FICOCO_ERR_GRID: return "grid smaller than the number of alive patches";
+    case FICOCO_ERR_STATIC_LIMIT:
+      return "problem exceeds the fixed scratch of the allocation-free entry point "
+             "(at most 64 images, dim 2048, 32768 patch tokens in total)";
     default: return "unknown error";
   }
 }
