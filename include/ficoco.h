@@ -183,7 +183,9 @@ int ficoco_l_reduce_host(ficoco_ctx* ctx, const ficoco_l_args* host_args,
                          const ficoco_params* params);
 
 /* Synchronise `cuda_stream`, read and clear the device status word into *device_status
- * (0 = clean; bit 0: a pos entry outside grid_h*grid_w was ignored by the local penalty). */
+ * (0 = clean; bit 0 (1): a pos entry outside grid_h*grid_w was ignored by the local penalty;
+ * bit 2 (4): a bounded wait inside the tensor-core correlate kernel ran out, the step's
+ * outputs are then invalid). */
 int ficoco_status(ficoco_ctx* ctx, void* cuda_stream, int* device_status);
 
 /*

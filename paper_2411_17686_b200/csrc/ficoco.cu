@@ -11,6 +11,7 @@
 #include "../../include/ficoco.h"
 #include "common.cuh"
 #include "kernels_correlate.cuh"
+#include "kernels_correlate_umma.cuh"
 #include "kernels_filter.cuh"
 #include "kernels_merge.cuh"
 
@@ -21,7 +22,7 @@ namespace {
 constexpr int N_PLANS = 8;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
 constexpr int OUT_ROWS_PER_CTA = 32;
-constexpr int NSPLIT_MAX = 8;
+constexpr int NSPLIT_MAX = 16;
 constexpr int TARGET_CTAS = 2 * 148;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -50,7 +51,11 @@ struct Plan {
   int n_rows = 0, n_corr = 0, n_out = 0;
   // totals and maxima used to size launches and inspection copies
   int tot_patch = 0, tot_src = 0, tot_tgt = 0, tot_out_rows = 0;
-  int max_np = 0, max_tgt = 0, max_rc = 0, max_nwin_cells = 0;
+  int max_np = 0, max_tgt = 0, max_src = 0, max_rc = 0, max_nwin_cells = 0;
+  // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
+  bool umma = false;
+  int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
+  size_t um_smem = 0;
   std::vector<ImgDesc> h_desc;
 };
 
@@ -76,13 +81,10 @@ struct ficoco_ctx {
   float* part_val = nullptr;
   int* part_idx = nullptr;
   int* corr_cnt = nullptr;
-  int* corr_tgt = nullptr;
-  float* corr_w = nullptr;
-  float* corr_c = nullptr;
+  int* e_tgt = nullptr;     // compact per-image entry arrays, L slots per discarded token
+  float* e_w = nullptr;
+  float* e_c = nullptr;
   float* tau = nullptr;
-  int* seg_off = nullptr;
-  int* seg_src = nullptr;
-  float* seg_w = nullptr;
   float* tmean = nullptr;
   unsigned* status = nullptr;
   char* plan_slots = nullptr;
@@ -247,7 +249,6 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
   const size_t o_cc = carve(T * 4), o_ct = carve(T * KCAP * 4), o_cw = carve(T * KCAP * 4);
   const size_t o_c = carve(T * KCAP * 4), o_tau = carve(T * 4);
-  const size_t o_so = carve((T + B + 1) * 4), o_ss = carve(T * KCAP * 4), o_sw = carve(T * KCAP * 4);
   const size_t o_tm = carve(max_text > 0 ? T * (size_t)max_text * 4 : 256);
   const size_t o_st = carve(256);
   const size_t o_pl = carve(c->slot_bytes * N_PLANS);
@@ -262,15 +263,16 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->s_raw = (float*)(b + o_sraw); c->s_pen = (float*)(b + o_spen);
   c->S_idx = (int*)(b + o_S); c->T_idx = (int*)(b + o_T);
   c->part_val = (float*)(b + o_pv); c->part_idx = (int*)(b + o_pi);
-  c->corr_cnt = (int*)(b + o_cc); c->corr_tgt = (int*)(b + o_ct); c->corr_w = (float*)(b + o_cw);
-  c->corr_c = (float*)(b + o_c); c->tau = (float*)(b + o_tau);
-  c->seg_off = (int*)(b + o_so); c->seg_src = (int*)(b + o_ss); c->seg_w = (float*)(b + o_sw);
+  c->corr_cnt = (int*)(b + o_cc); c->e_tgt = (int*)(b + o_ct); c->e_w = (float*)(b + o_cw);
+  c->e_c = (float*)(b + o_c); c->tau = (float*)(b + o_tau);
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
   c->plan_slots = b + o_pl;
 
   // kernels that may need more than 48 KB of dynamic shared memory
   cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  cudaFuncSetAttribute(k_finalize, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaGetLastError();
@@ -303,7 +305,11 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   p->h_desc.assign(B, ImgDesc());
   std::vector<WorkItem> rows, corr, outw;
   long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
-  p->max_np = p->max_tgt = p->max_rc = p->max_nwin_cells = 0;
+  p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = 0;
+  p->umma = key.mode == 0 && key.dtype == FICOCO_BF16 && key.dim % UKB == 0;
+  const int tile_rows_max = p->umma ? UM : CBM;       // source rows per correlate CTA
+  const int col_granule = p->umma ? 16 : CBN;
+  int um_a_rows = 8, um_cols = 16;
 
   // first pass: sizes
   long long base_strips = 0;
@@ -337,11 +343,11 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     }
     d.list_len = L;
     d.frac = frac;
-    if (L > 0) base_strips += (d.n_src + CBM - 1) / CBM;
+    if (L > 0) base_strips += (d.n_src + tile_rows_max - 1) / tile_rows_max;
   }
   int want_split = 1;
   if (base_strips > 0) {
-    want_split = (int)((TARGET_CTAS + base_strips - 1) / base_strips);
+    want_split = (int)(TARGET_CTAS / base_strips);
     if (want_split < 1) want_split = 1;
     if (want_split > NSPLIT_MAX) want_split = NSPLIT_MAX;
   }
@@ -366,15 +372,22 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     d.nsplit = 1; d.cols_per_split = d.n_tgt > 0 ? d.n_tgt : 1;
     if (d.list_len > 0) {
       int ns = want_split;
-      const int max_by_cols = (d.n_tgt + CBN - 1) / CBN;
+      const int max_by_cols = (d.n_tgt + col_granule - 1) / col_granule;
       if (ns > max_by_cols) ns = max_by_cols;
       int cps = (d.n_tgt + ns - 1) / ns;
-      cps = (cps + CBN - 1) / CBN * CBN;
+      cps = (cps + col_granule - 1) / col_granule * col_granule;
+      if (p->umma && cps > UN_MAX) cps = UN_MAX;
       ns = (d.n_tgt + cps - 1) / cps;
       d.nsplit = ns; d.cols_per_split = cps;
-      for (int s0 = 0; s0 < d.n_src; s0 += CBM)
+      // source tiles of equal size (rounded to 8 rows)
+      const int ntile = (d.n_src + tile_rows_max - 1) / tile_rows_max;
+      int trows = (d.n_src + ntile - 1) / ntile;
+      trows = (trows + 7) / 8 * 8;
+      if (trows > um_a_rows) um_a_rows = trows;
+      if (cps > um_cols) um_cols = cps;
+      for (int s0 = 0; s0 < d.n_src; s0 += trows)
         for (int sp = 0; sp < ns; ++sp) {
-          WorkItem w; w.img = b; w.r0 = s0; w.nrows = (d.n_src - s0 < CBM) ? d.n_src - s0 : CBM; w.aux = sp;
+          WorkItem w; w.img = b; w.r0 = s0; w.nrows = (d.n_src - s0 < trows) ? d.n_src - s0 : trows; w.aux = sp;
           corr.push_back(w);
         }
       part0 += (long long)d.n_src * ns * d.list_len;
@@ -390,6 +403,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     chunk0 += d.n_chunks;
     if (d.np > p->max_np) p->max_np = d.np;
     if (d.n_tgt > p->max_tgt) p->max_tgt = d.n_tgt;
+    if (d.n_src > p->max_src) p->max_src = d.n_src;
     if (key.mode == 0 && d.gh * d.gw > p->max_nwin_cells) p->max_nwin_cells = d.gh * d.gw;
   }
   if (row0 > c->max_tokens || B > c->max_batch || key.dim > c->max_dim || tail > c->max_text)
@@ -399,6 +413,21 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     return FICOCO_ERR_WORKSPACE;
   p->tot_patch = (int)patch0; p->tot_src = (int)src0; p->tot_tgt = (int)tgt0; p->tot_out_rows = (int)out0;
   p->n_rows = (int)rows.size(); p->n_corr = (int)corr.size(); p->n_out = (int)outw.size();
+  if (p->umma) {
+    // shared-memory ring of the tensor-core correlate: prefer a size that lets two CTAs share an SM
+    p->um_a_bytes = um_a_rows * 128;
+    p->um_stage_bytes = p->um_a_bytes + um_cols * 128;
+    p->um_tmem_cols = 32;
+    while (p->um_tmem_cols < um_cols) p->um_tmem_cols *= 2;
+    const size_t slack = 1024 + (p->um_stage_bytes < UM * 128 ? UM * 128 - p->um_stage_bytes : 0);
+    p->um_nstage = 0;
+    for (int ns = 4; ns >= 2 && !p->um_nstage; --ns)
+      if ((size_t)ns * p->um_stage_bytes + slack <= 106 * 1024) p->um_nstage = ns;
+    for (int ns = 4; ns >= 2 && !p->um_nstage; --ns)
+      if ((size_t)ns * p->um_stage_bytes + slack <= 220 * 1024) p->um_nstage = ns;
+    if (!p->um_nstage) return FICOCO_ERR_UNSUPPORTED;
+    p->um_smem = (size_t)p->um_nstage * p->um_stage_bytes + slack;
+  }
 
   char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
   p->d_desc = (ImgDesc*)slot_dev;
@@ -498,19 +527,35 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
                                                   pos_out, c->status);
   c->launches += 2;
   if (p->n_corr > 0) {
-    prof_tick(c, st, "correlate");
-    k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
-                                                   c->T_idx, tmean, M, gamma, c->part_val, c->part_idx);
+    if (p->umma && tmean == nullptr && sizeof(T) == 2) {
+      prof_tick(c, st, "correlate_umma");
+      const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
+      if (p->um_nstage == 4)
+        k_correlate_umma<4><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
+            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
+      else if (p->um_nstage == 3)
+        k_correlate_umma<3><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
+            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
+      else
+        k_correlate_umma<2><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
+            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
+    } else {
+      prof_tick(c, st, "correlate_simt");
+      k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
+                                                     c->T_idx, tmean, M, gamma, c->part_val, c->part_idx);
+    }
     c->launches += 1;
   }
-  prof_tick(c, st, "finalize");
-  k_finalize<<<p->key.batch, 256, (size_t)(2 * p->max_tgt + 2) * sizeof(int), st>>>(
-      p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->corr_tgt, c->corr_w, c->corr_c, c->tau,
-      c->seg_off, c->seg_src, c->seg_w);
+  if (p->max_src > 0) {
+    prof_tick(c, st, "finalize");
+    k_finalize_src<<<dim3(p->key.batch, (p->max_src + 255) / 256), 256, 0, st>>>(
+        p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c);
+    c->launches += 1;
+  }
   prof_tick(c, st, "merge_compact");
-  k_merge_compact<T><<<p->n_out, 256, 0, st>>>(tok, D, p->d_desc, p->d_out, c->S_idx, c->T_idx,
-                                               c->seg_off, c->seg_src, c->seg_w, out_tokens);
-  c->launches += 2;
+  k_merge_scan<T><<<p->n_out, 256, 0, st>>>(tok, D, p->d_desc, p->d_out, c->S_idx, c->T_idx, c->e_tgt,
+                                            c->e_w, out_tokens);
+  c->launches += 1;
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);
   cudaError_t e = cudaGetLastError();
@@ -636,9 +681,9 @@ extern "C" int ficoco_inspect(ficoco_ctx* c, int what, void* host_dst, size_t by
     case FICOCO_INSPECT_SRC_IDX: src = c->S_idx; n = (size_t)p->tot_src * 4; break;
     case FICOCO_INSPECT_TGT_IDX: src = c->T_idx; n = (size_t)p->tot_tgt * 4; break;
     case FICOCO_INSPECT_CORR_CNT: src = c->corr_cnt; n = (size_t)p->tot_src * 4; break;
-    case FICOCO_INSPECT_CORR_TGT: src = c->corr_tgt; n = (size_t)p->tot_src * KCAP * 4; break;
-    case FICOCO_INSPECT_CORR_W: src = c->corr_w; n = (size_t)p->tot_src * KCAP * 4; break;
-    case FICOCO_INSPECT_CORR_C: src = c->corr_c; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_CORR_TGT: src = c->e_tgt; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_CORR_W: src = c->e_w; n = (size_t)p->tot_src * KCAP * 4; break;
+    case FICOCO_INSPECT_CORR_C: src = c->e_c; n = (size_t)p->tot_src * KCAP * 4; break;
     case FICOCO_INSPECT_TAU: src = c->tau; n = (size_t)p->tot_src * 4; break;
     default: return FICOCO_ERR_INVALID_ARG;
   }
@@ -646,6 +691,20 @@ extern "C" int ficoco_inspect(ficoco_ctx* c, int what, void* host_dst, size_t by
   if (!host_dst || bytes == 0) return FICOCO_OK;
   CUDA_TRY(c, cudaSetDevice(c->device));
   CUDA_TRY(c, cudaDeviceSynchronize());
+  if (what == FICOCO_INSPECT_CORR_TGT || what == FICOCO_INSPECT_CORR_W || what == FICOCO_INSPECT_CORR_C) {
+    // the device keeps L slots per discarded token; widen to KCAP per token for the caller
+    long long tot_ent = 0;
+    for (const ImgDesc& d : p->h_desc) tot_ent += (long long)d.n_src * d.list_len;
+    std::vector<int> compact((size_t)tot_ent + 1);
+    if (tot_ent) CUDA_TRY(c, cudaMemcpy(compact.data(), src, (size_t)tot_ent * 4, cudaMemcpyDeviceToHost));
+    std::vector<int> wide((size_t)p->tot_src * KCAP, what == FICOCO_INSPECT_CORR_TGT ? -1 : 0);
+    for (const ImgDesc& d : p->h_desc)
+      for (int s = 0; s < d.n_src; ++s)
+        for (int k = 0; k < d.list_len; ++k)
+          wide[(size_t)(d.src0 + s) * KCAP + k] = compact[(size_t)d.ent0 + (size_t)s * d.list_len + k];
+    memcpy(host_dst, wide.data(), bytes < n ? bytes : n);
+    return FICOCO_OK;
+  }
   CUDA_TRY(c, cudaMemcpy(host_dst, src, bytes < n ? bytes : n, cudaMemcpyDeviceToHost));
   return FICOCO_OK;
 }

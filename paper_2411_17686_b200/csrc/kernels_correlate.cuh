@@ -1,5 +1,4 @@
-// Correlate stage: C_ij for i in S, j in T, per-row top list, tau_i, J_i, alpha_ij, and the
-// inversion of the per-source target lists into per-target source lists.
+// Correlate stage: C_ij for i in S, j in T, per-row top list, tau_i, J_i, alpha_ij.
 #pragma once
 #include <limits.h>
 #include <math_constants.h>
@@ -186,104 +185,72 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
   }
 }
 
+}  // namespace ficoco
+
+namespace ficoco {
+
 // ---------------------------------------------------------------------------------------
-// Per image: merge the column splits' partial top lists, take the quantile threshold
-//   tau_i = v[L-1] + frac * (v[L-2] - v[L-1])   (v descending: the two order statistics
-//   around eps*(n-1)), J_i = { entries >= tau_i }, alpha_ij = C+_ij / sum_{J_i} C+  (Eq. 2),
-// then invert source->targets into per-target segments sorted by source, which fixes the
-// accumulation order of the merge.
-// One CTA (256 threads) per image; dynamic smem: 2 * n_tgt ints.
+// One thread per discarded token: merge the column splits' partial top lists, then
+//   tau_i = v[L-1] + frac * (v[L-2] - v[L-1])  (v descending: the two order statistics around
+//   eps*(n-1)), J_i = { entries >= tau_i }, alpha_ij = C+_ij / sum_{J_i} C+  (Eq. 2).
+// Results go to compact per-image arrays with L slots per token: e_tgt (position in T, or -1),
+// e_w (alpha), e_c (the L largest C, descending).
+// grid = (images, ceil(max N^S / 256)).
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_finalize(
+__global__ void __launch_bounds__(256) k_finalize_src(
     const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
-    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, int* __restrict__ corr_tgt,
-    float* __restrict__ corr_w, float* __restrict__ corr_c, float* __restrict__ tau_out,
-    int* __restrict__ seg_off, int* __restrict__ seg_src, float* __restrict__ seg_w) {
-  extern __shared__ int smi[];
-  __shared__ int warp_tot[33];
+    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
   const ImgDesc d = desc[blockIdx.x];
-  const int img = blockIdx.x;
   const int L = d.list_len;
-  const int tid = threadIdx.x;
-  int* cnt = smi;
-  int* cur = smi + d.n_tgt;
-
-  for (int j = tid; j < d.n_tgt; j += 256) cnt[j] = 0;
-  __syncthreads();
-
-  for (int s = tid; s < d.n_src; s += 256) {
-    const size_t o = (size_t)(d.src0 + s);
-    if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; continue; }
-    float v[KCAP];
-    int ix[KCAP];
+  const int s = blockIdx.y * 256 + threadIdx.x;
+  if (s >= d.n_src) return;
+  const size_t o = (size_t)(d.src0 + s);
+  if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; return; }
+  float v[KCAP];
+  int ix[KCAP];
 #pragma unroll
-    for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-    const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
-    for (int e = 0; e < d.nsplit * L; ++e) {
-      const int id = part_idx[pbase + e];
-      const float val = part_val[pbase + e];
-      if (id >= 0 && toplist_better(val, id, v[L - 1], ix[L - 1])) toplist_insert(v, ix, L, val, id);
-    }
-    const float tau = (L >= 2) ? v[L - 1] + d.frac * (v[L - 2] - v[L - 1]) : v[0];
-    int nj = 0;
-    float den = 0.f;
-    for (int k = 0; k < L; ++k) {
-      if (ix[k] != INT_MAX && v[k] >= tau) { ++nj; den += fmaxf(v[k], 0.f); } else break;
-    }
-    if (!(den > 1e-12f)) nj = 0;
-    corr_cnt[o] = nj;
-    tau_out[o] = tau;
+  for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+  const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
+  const int ne = d.nsplit * L;
+  for (int e = 0; e < ne; ++e) {
+    float cv = part_val[pbase + e];
+    int ci = part_idx[pbase + e];
+    if (ci < 0) continue;
+#pragma unroll
     for (int k = 0; k < KCAP; ++k) {
-      corr_tgt[o * KCAP + k] = k < nj ? ix[k] : -1;
-      corr_w[o * KCAP + k] = k < nj ? fmaxf(v[k], 0.f) / den : 0.f;
-      corr_c[o * KCAP + k] = k < L ? v[k] : 0.f;
-    }
-    for (int k = 0; k < nj; ++k) atomicAdd(&cnt[ix[k]], 1);
-  }
-  __syncthreads();
-
-  int base = 0;
-  for (int j0 = 0; j0 < d.n_tgt; j0 += 256) {
-    const int j = j0 + tid;
-    const int c = j < d.n_tgt ? cnt[j] : 0;
-    int tot;
-    const int ex = base + block_exclusive_scan(c, warp_tot, &tot);
-    if (j < d.n_tgt) {
-      cur[j] = ex;
-      seg_off[d.tgt0 + img + j] = d.ent0 + ex;
-    }
-    base += tot;
-  }
-  if (tid == 0) seg_off[d.tgt0 + img + d.n_tgt] = d.ent0 + base;
-  __syncthreads();
-
-  for (int s = tid; s < d.n_src; s += 256) {
-    const size_t o = (size_t)(d.src0 + s);
-    const int nj = corr_cnt[o];
-    for (int k = 0; k < nj; ++k) {
-      const int j = corr_tgt[o * KCAP + k];
-      const int slot = atomicAdd(&cur[j], 1);
-      seg_src[d.ent0 + slot] = s;
-      seg_w[d.ent0 + slot] = corr_w[o * KCAP + k];
-    }
-  }
-  __syncthreads();
-
-  // ascending source order inside every segment (sources ascend with the token index)
-  for (int j = tid; j < d.n_tgt; j += 256) {
-    const int e1 = d.ent0 + cur[j];
-    const int e0 = e1 - cnt[j];
-    for (int a = e0 + 1; a < e1; ++a) {
-      const int ks = seg_src[a];
-      const float kw = seg_w[a];
-      int b = a - 1;
-      while (b >= e0 && seg_src[b] > ks) {
-        seg_src[b + 1] = seg_src[b];
-        seg_w[b + 1] = seg_w[b];
-        --b;
+      if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
+        const float tv = v[k]; const int ti = ix[k];
+        v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
       }
-      seg_src[b + 1] = ks;
-      seg_w[b + 1] = kw;
+    }
+  }
+  float vl1 = 0.f, vl2 = 0.f;
+#pragma unroll
+  for (int k = 0; k < KCAP; ++k) {
+    if (k == L - 1) vl1 = v[k];
+    if (k == L - 2) vl2 = v[k];
+  }
+  const float tau = (L >= 2) ? vl1 + d.frac * (vl2 - vl1) : vl1;
+  int nj = 0;
+  float den = 0.f;
+  bool open = true;
+#pragma unroll
+  for (int k = 0; k < KCAP; ++k) {
+    if (k < L && open) {
+      if (ix[k] != INT_MAX && v[k] >= tau) { ++nj; den += fmaxf(v[k], 0.f); } else open = false;
+    }
+  }
+  if (!(den > 1e-12f)) nj = 0;
+  corr_cnt[o] = nj;
+  tau_out[o] = tau;
+  const size_t eb = (size_t)d.ent0 + (size_t)s * L;
+#pragma unroll
+  for (int k = 0; k < KCAP; ++k) {
+    if (k < L) {
+      e_tgt[eb + k] = k < nj ? ix[k] : -1;
+      e_w[eb + k] = k < nj ? fmaxf(v[k], 0.f) / den : 0.f;
+      e_c[eb + k] = v[k];
     }
   }
 }

@@ -1,0 +1,273 @@
+// Correlate stage on the 5th-generation tensor cores (bf16 tokens).
+//
+// One CTA owns up to 128 discarded tokens (rows of the accumulator, one TMEM lane each) and
+// one column split (<= 256 preserved tokens) of one image:
+//   warps 0-3  gather the token rows with 16-byte cp.async into a ring of 128B-swizzled,
+//              K-major shared-memory tiles (64 bf16 of the hidden dimension per stage);
+//   warp  4    allocates TMEM and issues tcgen05.mma (M = 128, N = columns rounded to 16,
+//              K = 16 per instruction, fp32 accumulation of exact bf16 products);
+//   warps 0-3  afterwards read their 32 TMEM lanes back with tcgen05.ld, scale by
+//              rn_i * rn_j to cosines and keep each row's L largest entries.
+// Rows / columns past the valid range are never loaded: their shared memory is garbage that
+// only reaches accumulator rows / columns the epilogue ignores.
+// Every wait is bounded; on a timeout the CTA raises STATUS_TIMEOUT, drains its copies,
+// frees its TMEM and returns.
+#pragma once
+#include <limits.h>
+#include <math_constants.h>
+#include "common.cuh"
+
+namespace ficoco {
+
+constexpr int UM = 128;          // accumulator rows per CTA
+constexpr int UN_MAX = 256;      // accumulator columns per CTA
+constexpr int UKB = 64;          // bf16 elements per k-block (one 128-byte swizzle row)
+constexpr unsigned STATUS_TIMEOUT = 4u;
+constexpr int SPIN_LIMIT = 1 << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait on a phase parity; false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  const uint32_t a = smem_u32(bar);
+  for (int it = 0; it < SPIN_LIMIT; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// K-major, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                      // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;            // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                      // descriptor version for sm_100
+  d |= (uint64_t)2 << 61;                      // SWIZZLE_128B
+  return d;
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(UM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+               ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Dynamic shared memory: [1024-aligned] ring of NSTAGE stages, each an A tile (a_bytes: the
+// valid source rows rounded up to 8, x 128 B) followed by a B tile (column rows x 128 B).  The
+// MMA always reads 128 A rows; rows past a_bytes alias the B tile (or the slack the host adds
+// behind the ring) and only feed accumulator rows that are never read.
+template <int NSTAGE>
+__global__ void __launch_bounds__(160) k_correlate_umma(
+    const __nv_bfloat16* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
+    const WorkItem* __restrict__ work, const float* __restrict__ rn,
+    const int* __restrict__ S_idx, const int* __restrict__ T_idx,
+    float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
+    int stage_bytes, int a_bytes, int tmem_cols) {
+  extern __shared__ unsigned char um_raw[];
+  __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int rowS[UM], rowT[UN_MAX];
+  __shared__ float rnT[UN_MAX];
+  __shared__ int failed, acc_committed;
+
+  const WorkItem w = work[blockIdx.x];
+  const ImgDesc d = desc[w.img];
+  const int L = d.list_len;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int col_begin = w.aux * d.cols_per_split;
+  const int ncols = min(d.n_tgt, col_begin + d.cols_per_split) - col_begin;   // 1..256
+  const int n_pad = (ncols + 15) & ~15;
+  const int nkb = D / UKB;
+  const uint32_t ring = (smem_u32(um_raw) + 1023u) & ~1023u;
+
+  if (tid == 0) {
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full_bar[s], 128); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&acc_bar, 1);
+    failed = 0;
+    acc_committed = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < UM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
+  for (int c = tid; c < UN_MAX; c += 160) {
+    const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
+    rowT[c] = p;
+    rnT[c] = p >= 0 ? rn[d.patch0 + p] : 0.f;
+  }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  if (warp < 4) {
+    // ---------------- producer: gather rows, 16 bytes per thread per copy -------------------
+    const int chunk = tid & 7;          // 16-byte chunk inside the 128-byte row
+    const int rsub = tid >> 3;          // 0..15
+    const __nv_bfloat16* tbase = tokens + (size_t)(d.row0 + d.n_cls) * D + chunk * 8;
+    bool ok = true;
+    for (int kb = 0; kb < nkb + (NSTAGE - 1); ++kb) {
+      if (kb < nkb) {
+        const int s = kb % NSTAGE;
+        if (kb >= NSTAGE && ok) ok = mbar_wait(&empty_bar[s], ((kb / NSTAGE) - 1) & 1);
+        if (ok) {
+          const uint32_t a0 = ring + (uint32_t)s * stage_bytes;
+          const uint32_t b0 = a0 + (uint32_t)a_bytes;
+          const __nv_bfloat16* src = tbase + (size_t)kb * UKB;
+          for (int r = rsub; r < w.nrows; r += 16)
+            cp_async16(a0 + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4),
+                       src + (size_t)rowS[r] * D);
+          for (int r = rsub; r < ncols; r += 16)
+            cp_async16(b0 + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4),
+                       src + (size_t)rowT[r] * D);
+        }
+      }
+      cp_async_commit();
+      // the group committed NSTAGE-1 iterations ago has landed: publish that stage
+      const int done = kb - (NSTAGE - 1);
+      if (done >= 0) {
+        cp_async_wait<NSTAGE - 1>();
+        fence_proxy_async();
+        mbar_arrive(&full_bar[done % NSTAGE]);
+      }
+    }
+    cp_async_wait<0>();
+    if (!ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+
+    // ---------------- epilogue: lane = accumulator row ---------------------------------------
+    bool acc_ok = ok && mbar_wait(&acc_bar, 0);
+    if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
+    tc_fence_after();
+    const int row = tid;                               // TMEM lane == accumulator row
+    const bool row_valid = row < w.nrows;
+    const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
+    float v[KCAP];
+    int ix[KCAP];
+#pragma unroll
+    for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    float vmin = -CUDART_INF_F;                        // value of entry L-1
+    int imin = INT_MAX;
+    if (acc_ok) {
+      for (int c0 = 0; c0 < n_pad; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int c = c0 + j;
+          const float val = (rs * rnT[c]) * __uint_as_float(r[j]);
+          const int idx = col_begin + c;
+          if (c < ncols && row_valid && toplist_better(val, idx, vmin, imin)) {
+            // insert into the descending list, dropping entry L-1
+            float cv = val;
+            int ci = idx;
+#pragma unroll
+            for (int k = 0; k < KCAP; ++k) {
+              if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
+                const float tv = v[k]; const int ti = ix[k];
+                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+              }
+            }
+#pragma unroll
+            for (int k = 0; k < KCAP; ++k)
+              if (k == L - 1) { vmin = v[k]; imin = ix[k]; }
+          }
+        }
+      }
+    }
+    if (row_valid) {
+      const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
+#pragma unroll
+      for (int k = 0; k < KCAP; ++k)
+        if (k < L) {
+          part_val[o + k] = v[k];
+          part_idx[o + k] = ix[k] == INT_MAX ? -1 : ix[k];
+        }
+    }
+  } else {
+    // ---------------- MMA issuer (one lane) ---------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(n_pad);
+      bool ok = true;
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % NSTAGE;
+        ok = mbar_wait(&full_bar[s], (kb / NSTAGE) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t a0 = ring + (uint32_t)s * stage_bytes;
+        const uint64_t ad = umma_smem_desc(a0), bd = umma_smem_desc(a0 + (uint32_t)a_bytes);
+#pragma unroll
+        for (int k4 = 0; k4 < UKB / 16; ++k4)
+          umma_bf16(tmem_base, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc,
+                    (kb > 0 || k4 > 0) ? 1u : 0u);
+        umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
+      }
+      if (ok) { umma_commit(&acc_bar); acc_committed = 1; }   // accumulator complete
+      else { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+    }
+    __syncwarp();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    if (failed) {
+      // MMAs may still be in flight: give them a bounded time to drain before freeing TMEM
+      if (lane == 0) {
+        if (!acc_committed) umma_commit(&acc_bar);
+        mbar_wait(&acc_bar, 0);
+      }
+      __syncwarp();
+    }
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
+                 : "memory");
+  }
+}
+
+}  // namespace ficoco
