@@ -270,12 +270,12 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
 
   // kernels that may need more than 48 KB of dynamic shared memory
   cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+  cudaFuncSetAttribute(k_correlate_umma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
-  cudaGetLastError();
+  if (cudaGetLastError() != cudaSuccess) { ficoco_destroy(c); return FICOCO_ERR_CUDA; }
   *out = c;
   return FICOCO_OK;
 }
