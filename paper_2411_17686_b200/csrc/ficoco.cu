@@ -21,7 +21,7 @@ namespace {
 
 constexpr int N_PLANS = 8;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
-constexpr int OUT_ROWS_PER_CTA = 32;
+constexpr int OUT_ROWS_PER_CTA = 8;   // == MROWS of the merge kernel
 constexpr int NSPLIT_MAX = 16;
 constexpr int TARGET_CTAS = 2 * 148;
 
@@ -51,7 +51,7 @@ struct Plan {
   int n_rows = 0, n_corr = 0, n_out = 0;
   // totals and maxima used to size launches and inspection copies
   int tot_patch = 0, tot_src = 0, tot_tgt = 0, tot_out_rows = 0;
-  int max_np = 0, max_tgt = 0, max_src = 0, max_rc = 0, max_nwin_cells = 0;
+  int max_np = 0, max_tgt = 0, max_src = 0, max_rc = 0, max_nwin_cells = 0, max_list = 0;
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
   bool umma = false;
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
@@ -270,9 +270,18 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
 
   // kernels that may need more than 48 KB of dynamic shared memory
   cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
-  cudaFuncSetAttribute(k_correlate_umma<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 221 * 1024);
+  {
+    const int um_smem_max = 221 * 1024;
+    cudaFuncSetAttribute(k_correlate_umma<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<3, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<4, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<2, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<3, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+  }
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   if (cudaGetLastError() != cudaSuccess) { ficoco_destroy(c); return FICOCO_ERR_CUDA; }
@@ -305,7 +314,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   p->h_desc.assign(B, ImgDesc());
   std::vector<WorkItem> rows, corr, outw;
   long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
-  p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = 0;
+  p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = p->max_list = 0;
   p->umma = key.mode == 0 && key.dtype == FICOCO_BF16 && key.dim % UKB == 0;
   const int tile_rows_max = p->umma ? UM : CBM;       // source rows per correlate CTA
   const int col_granule = p->umma ? 16 : CBN;
@@ -343,6 +352,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     }
     d.list_len = L;
     d.frac = frac;
+    if (L > p->max_list) p->max_list = L;
     if (L > 0) base_strips += (d.n_src + tile_rows_max - 1) / tile_rows_max;
   }
   int want_split = 1;
@@ -530,15 +540,21 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     if (p->umma && tmean == nullptr && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
-      if (p->um_nstage == 4)
-        k_correlate_umma<4><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
-            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
-      else if (p->um_nstage == 3)
-        k_correlate_umma<3><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
-            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
-      else
-        k_correlate_umma<2><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
-            c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols);
+#define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
+  k_correlate_umma<NS, LC><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
+      c->S_idx, c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes,        \
+      p->um_tmem_cols)
+#define FICOCO_UMMA_STAGES(LC)                                                                         \
+  do {                                                                                                 \
+    if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                                  \
+    else if (p->um_nstage == 3) FICOCO_UMMA_LAUNCH(3, LC);                                             \
+    else FICOCO_UMMA_LAUNCH(2, LC);                                                                    \
+  } while (0)
+      if (p->max_list <= 2) FICOCO_UMMA_STAGES(2);
+      else if (p->max_list <= 4) FICOCO_UMMA_STAGES(4);
+      else FICOCO_UMMA_STAGES(16);
+#undef FICOCO_UMMA_STAGES
+#undef FICOCO_UMMA_LAUNCH
     } else {
       prof_tick(c, st, "correlate_simt");
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,

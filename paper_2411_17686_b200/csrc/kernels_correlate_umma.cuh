@@ -7,7 +7,7 @@
 //   warp  4    allocates TMEM and issues tcgen05.mma (M = 128, N = columns rounded to 16,
 //              K = 16 per instruction, fp32 accumulation of exact bf16 products);
 //   warps 0-3  afterwards read their 32 TMEM lanes back with tcgen05.ld, scale by
-//              rn_i * rn_j to cosines and keep each row's L largest entries.
+//              rn_i * rn_j to cosines and keep each row's L <= LCAP largest entries in registers.
 // Rows / columns past the valid range are never loaded: their shared memory is garbage that
 // only reaches accumulator rows / columns the epilogue ignores.
 // Every wait is bounded; on a timeout the CTA raises STATUS_TIMEOUT, drains its copies,
@@ -99,7 +99,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 // valid source rows rounded up to 8, x 128 B) followed by a B tile (column rows x 128 B).  The
 // MMA always reads 128 A rows; rows past a_bytes alias the B tile (or the slack the host adds
 // behind the ring) and only feed accumulator rows that are never read.
-template <int NSTAGE>
+template <int NSTAGE, int LCAP>
 __global__ void __launch_bounds__(160) k_correlate_umma(
     const __nv_bfloat16* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const float* __restrict__ rn,
@@ -152,7 +152,10 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int rsub = tid >> 3;          // 0..15
     const __nv_bfloat16* tbase = tokens + (size_t)(d.row0 + d.n_cls) * D + chunk * 8;
     bool ok = true;
-    for (int kb = 0; kb < nkb + (NSTAGE - 1); ++kb) {
+    // a stage is published LAG iterations after its copies were issued; LAG < NSTAGE - 1 leaves
+    // the MMA a full iteration to drain a stage before the producer needs it again
+    constexpr int LAG = NSTAGE >= 3 ? NSTAGE - 2 : 1;
+    for (int kb = 0; kb < nkb + LAG; ++kb) {
       if (kb < nkb) {
         const int s = kb % NSTAGE;
         if (kb >= NSTAGE && ok) ok = mbar_wait(&empty_bar[s], ((kb / NSTAGE) - 1) & 1);
@@ -169,10 +172,10 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
         }
       }
       cp_async_commit();
-      // the group committed NSTAGE-1 iterations ago has landed: publish that stage
-      const int done = kb - (NSTAGE - 1);
+      // the group committed LAG iterations ago has landed: publish that stage
+      const int done = kb - LAG;
       if (done >= 0) {
-        cp_async_wait<NSTAGE - 1>();
+        cp_async_wait<LAG>();
         fence_proxy_async();
         mbar_arrive(&full_bar[done % NSTAGE]);
       }
@@ -188,10 +191,10 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
     const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    float v[KCAP];
-    int ix[KCAP];
+    float v[LCAP];
+    int ix[LCAP];
 #pragma unroll
-    for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
     float vmin = -CUDART_INF_F;                        // value of entry L-1
     int imin = INT_MAX;
     if (acc_ok) {
@@ -208,14 +211,14 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
             float cv = val;
             int ci = idx;
 #pragma unroll
-            for (int k = 0; k < KCAP; ++k) {
+            for (int k = 0; k < LCAP; ++k) {
               if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
                 const float tv = v[k]; const int ti = ix[k];
                 v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
               }
             }
 #pragma unroll
-            for (int k = 0; k < KCAP; ++k)
+            for (int k = 0; k < LCAP; ++k)
               if (k == L - 1) { vmin = v[k]; imin = ix[k]; }
           }
         }
@@ -224,7 +227,7 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     if (row_valid) {
       const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
 #pragma unroll
-      for (int k = 0; k < KCAP; ++k)
+      for (int k = 0; k < LCAP; ++k)
         if (k < L) {
           part_val[o + k] = v[k];
           part_idx[o + k] = ix[k] == INT_MAX ? -1 : ix[k];
