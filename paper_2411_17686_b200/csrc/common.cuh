@@ -86,20 +86,26 @@ __device__ __forceinline__ uint32_t order_key(float s) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Exclusive prefix sum of one value per thread over the block (blockDim.x <= 1024, multiple
-// of 32).  `warp_tot` is a 33-int shared scratch.  Returns the exclusive prefix; *total gets
-// the block total.  Contains __syncthreads, call from all threads.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+// Barrier over the first `n` threads of the CTA (n a multiple of 32) on hardware barrier `id`;
+// cta_sync(0, blockDim.x) is __syncthreads().
+__device__ __forceinline__ void cta_sync(int id, int n) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
+}
+
+// Exclusive prefix sum of one value per thread over `nthr` threads (<= 1024, multiple of 32)
+// that synchronise on barrier `bar`.  `warp_tot` is a 33-int shared scratch.  Returns the
+// exclusive prefix; *total gets the total.  Contains barriers: call from all `nthr` threads.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* total, int bar, int nthr) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = nthr >> 5;
   int inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
     if (lane >= o) inc += n;
   }
-  __syncthreads();
+  cta_sync(bar, nthr);
   if (lane == 31) warp_tot[warp] = inc;
-  __syncthreads();
+  cta_sync(bar, nthr);
   if (warp == 0) {
     int w = (lane < nwarp) ? warp_tot[lane] : 0;
     int winc = w;
@@ -111,7 +117,7 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_tot, int* t
     if (lane < nwarp) warp_tot[lane] = winc - w;
     if (lane == 31) warp_tot[32] = winc;
   }
-  __syncthreads();
+  cta_sync(bar, nthr);
   *total = warp_tot[32];
   return warp_tot[warp] + inc - v;
 }

@@ -13,6 +13,7 @@
 #include "kernels_correlate.cuh"
 #include "kernels_correlate_umma.cuh"
 #include "kernels_filter.cuh"
+#include "kernels_filter_fused.cuh"
 #include "kernels_merge.cuh"
 
 using namespace ficoco;
@@ -52,6 +53,11 @@ struct Plan {
   // totals and maxima used to size launches and inspection copies
   int tot_patch = 0, tot_src = 0, tot_tgt = 0, tot_out_rows = 0;
   int max_np = 0, max_tgt = 0, max_src = 0, max_rc = 0, max_nwin_cells = 0, max_list = 0;
+  // fused persistent filter kernel
+  bool fused = false;
+  int* d_ctafirst = nullptr;
+  int f_grid = 0, f_nstage = 0, f_max_piece = 0, f_vpl = 0;
+  size_t f_smem = 0;
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
   bool umma = false;
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
@@ -87,9 +93,12 @@ struct ficoco_ctx {
   float* tau = nullptr;
   float* tmean = nullptr;
   unsigned* status = nullptr;
+  int* img_cnt = nullptr;   // 2 * max_batch per-image piece counters of the fused filter kernel
+  int num_sms = 0;
+  bool coop_ok = false;
   char* plan_slots = nullptr;
   size_t slot_bytes = 0;
-  size_t off_rows = 0, off_corr = 0, off_out = 0;
+  size_t off_rows = 0, off_corr = 0, off_out = 0, off_ctaf = 0;
   int cap_rows = 0, cap_corr = 0, cap_out = 0;
   long long cap_part = 0;
 
@@ -232,18 +241,29 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   if (e != cudaSuccess) { delete c; return FICOCO_ERR_CUDA; }
 
   const size_t T = (size_t)max_tokens, B = (size_t)max_batch;
+  {
+    int v = 0;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device);
+    c->num_sms = v > 0 ? v : 1;
+    v = 0;
+    cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, device);
+    c->coop_ok = v != 0;
+  }
   c->cap_rows = (int)(MAX_CHUNKS * B);
+  if (c->cap_rows < c->num_sms + (int)B + 8) c->cap_rows = c->num_sms + (int)B + 8;
   c->cap_corr = (int)(2 * (T / CBM + B) + 2048);
   c->cap_out = (int)(T / OUT_ROWS_PER_CTA + B);
   c->cap_part = (long long)T * PART_PER_TOKEN;
   c->off_rows = align_up(B * sizeof(ImgDesc), 256);
   c->off_corr = c->off_rows + align_up((size_t)c->cap_rows * sizeof(WorkItem), 256);
   c->off_out = c->off_corr + align_up((size_t)c->cap_corr * sizeof(WorkItem), 256);
-  c->slot_bytes = c->off_out + align_up((size_t)c->cap_out * sizeof(WorkItem), 256);
+  c->off_ctaf = c->off_out + align_up((size_t)c->cap_out * sizeof(WorkItem), 256);
+  c->slot_bytes = c->off_ctaf + align_up((size_t)(c->num_sms + 2) * sizeof(int), 256);
 
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
-  const size_t o_rn = carve(T * 4), o_partial = carve((size_t)MAX_CHUNKS * B * max_dim * 4);
+  const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
+  const size_t o_icnt = carve(2 * B * 4);
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
@@ -266,6 +286,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->corr_cnt = (int*)(b + o_cc); c->e_tgt = (int*)(b + o_ct); c->e_w = (float*)(b + o_cw);
   c->e_c = (float*)(b + o_c); c->tau = (float*)(b + o_tau);
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
+  c->img_cnt = (int*)(b + o_icnt);
   c->plan_slots = b + o_pl;
 
   // kernels that may need more than 48 KB of dynamic shared memory
@@ -281,6 +302,15 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
     cudaFuncSetAttribute(k_correlate_umma<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+  }
+  {
+    const int fmax = 221 * 1024;
+#define FICOCO_FUSED_ATTR(TT, V) cudaFuncSetAttribute(k_filter_fused<TT, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, fmax)
+    FICOCO_FUSED_ATTR(float, 1); FICOCO_FUSED_ATTR(float, 2); FICOCO_FUSED_ATTR(float, 4);
+    FICOCO_FUSED_ATTR(float, 5); FICOCO_FUSED_ATTR(float, 8);
+    FICOCO_FUSED_ATTR(__nv_bfloat16, 1); FICOCO_FUSED_ATTR(__nv_bfloat16, 2); FICOCO_FUSED_ATTR(__nv_bfloat16, 4);
+    FICOCO_FUSED_ATTR(__nv_bfloat16, 5); FICOCO_FUSED_ATTR(__nv_bfloat16, 8);
+#undef FICOCO_FUSED_ATTR
   }
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -355,6 +385,29 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     if (L > p->max_list) p->max_list = L;
     if (L > 0) base_strips += (d.n_src + tile_rows_max - 1) / tile_rows_max;
   }
+  // ---- fused filter kernel: piece size and feasibility -------------------------------------
+  const int esz = key.dtype == FICOCO_BF16 ? 2 : 4;
+  const int f_nvec = key.dim / (16 / esz);
+  p->f_vpl = (f_nvec + 31) / 32;
+  p->fused = c->coop_ok && p->f_vpl <= 8;
+  int f_rc = 0;
+  if (p->fused) {
+    long long total = 0;
+    for (int b = 0; b < B; ++b) total += p->h_desc[b].np;
+    auto count = [&](int rc) {
+      long long n = 0;
+      for (int b = 0; b < B; ++b) n += (p->h_desc[b].np + rc - 1) / rc;
+      return n;
+    };
+    int rc0 = (int)((total + c->num_sms - 1) / c->num_sms);
+    if (rc0 < 32) rc0 = 32;
+    rc0 = (rc0 + 7) / 8 * 8;
+    int rc1 = rc0;
+    while (count(rc1) > c->num_sms && rc1 < 2 * rc0) rc1 += 8;
+    // one piece per CTA if that costs at most 60 % more rows per CTA, else several pieces per CTA
+    f_rc = (count(rc1) <= c->num_sms && rc1 * 10 <= rc0 * 16) ? rc1 : rc0;
+  }
+
   int want_split = 1;
   if (base_strips > 0) {
     want_split = (int)(TARGET_CTAS / base_strips);
@@ -367,10 +420,14 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     d.row0 = (int)row0; d.patch0 = (int)patch0; d.out_row0 = (int)out0;
     d.src0 = (int)src0; d.tgt0 = (int)tgt0; d.ent0 = (int)ent0; d.part0 = (int)part0;
     d.attn0 = 0;  // set by the caller-specific code below
-    // row chunks
+    // row chunks (fused filter: equal pieces of at most f_rc rows)
     int rc = (d.np + MAX_CHUNKS - 1) / MAX_CHUNKS;
     rc = (rc + 7) / 8 * 8;
     if (rc < 64) rc = 64;
+    if (p->fused) {
+      const int npc = (d.np + f_rc - 1) / f_rc;
+      rc = ((d.np + npc - 1) / npc + 7) / 8 * 8;
+    }
     d.n_chunks = (d.np + rc - 1) / rc;
     d.chunk0 = (int)chunk0;
     for (int k = 0; k < d.n_chunks; ++k) {
@@ -418,6 +475,45 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   }
   if (row0 > c->max_tokens || B > c->max_batch || key.dim > c->max_dim || tail > c->max_text)
     return FICOCO_ERR_WORKSPACE;
+  // ---- fused filter kernel: pieces -> CTAs, shared memory -----------------------------------
+  std::vector<int> cta_first;
+  if (p->fused) {
+    long long total = 0;
+    for (const WorkItem& w : rows) total += w.nrows;
+    const long long target = (total + c->num_sms - 1) / c->num_sms;
+    cta_first.push_back(0);
+    long long acc_rows = 0;
+    int items = 0;
+    for (size_t i = 0; i < rows.size(); ++i) {
+      if (items > 0 && (acc_rows + rows[i].nrows > target + 8 || items >= F_MAXWON) &&
+          (int)cta_first.size() < c->num_sms) {
+        cta_first.push_back((int)i);
+        acc_rows = 0;
+        items = 0;
+      }
+      acc_rows += rows[i].nrows;
+      ++items;
+      if (items > F_MAXWON) p->fused = false;
+    }
+    cta_first.push_back((int)rows.size());
+    p->f_grid = (int)cta_first.size() - 1;
+    p->f_max_piece = p->max_rc;
+    const size_t stage = (size_t)FROWS * key.dim * esz;
+    const size_t fixed = (size_t)FROWS * key.dim * 4 + (size_t)p->f_max_piece * 4 + 256;
+    const size_t budget = 216 * 1024;
+    int ns = budget > fixed ? (int)((budget - fixed) / stage) : 0;
+    if (ns > F_MAXSTAGE) ns = F_MAXSTAGE;
+    size_t sel_need = 0;
+    for (int b = 0; b < B; ++b) {
+      const ImgDesc& d = p->h_desc[b];
+      const size_t need = align_up((size_t)d.np * 4, 8) + (key.mode == 0 ? (size_t)d.gh * d.gw * 8 : 0);
+      if (need > sel_need) sel_need = need;
+    }
+    if (ns < 2 || sel_need > (size_t)ns * stage) p->fused = false;
+    p->f_nstage = ns;
+    p->f_smem = (size_t)ns * stage + fixed;
+  }
+  if (!p->fused && rows.size() > (size_t)MAX_CHUNKS * B) return FICOCO_ERR_UNSUPPORTED;
   if ((int)rows.size() > c->cap_rows || (int)corr.size() > c->cap_corr || (int)outw.size() > c->cap_out ||
       part0 > c->cap_part)
     return FICOCO_ERR_WORKSPACE;
@@ -444,7 +540,9 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   p->d_rows = (WorkItem*)(slot_dev + c->off_rows);
   p->d_corr = (WorkItem*)(slot_dev + c->off_corr);
   p->d_out = (WorkItem*)(slot_dev + c->off_out);
+  p->d_ctafirst = (int*)(slot_dev + c->off_ctaf);
   p->key = key;
+  if (p->fused) memcpy(c->h_stage + c->off_ctaf, cta_first.data(), cta_first.size() * sizeof(int));
   memcpy(c->h_stage + c->off_rows, rows.data(), rows.size() * sizeof(WorkItem));
   memcpy(c->h_stage + c->off_corr, corr.data(), corr.size() * sizeof(WorkItem));
   memcpy(c->h_stage + c->off_out, outw.data(), outw.size() * sizeof(WorkItem));
@@ -495,6 +593,27 @@ int get_plan(ficoco_ctx* c, const PlanKey& key, long long attn_rows, cudaStream_
 }
 
 template <class T, int VPL>
+cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn,
+                                int attn_rows, float cA, const int* pos, int window, float coef, int penalty,
+                                int* kept_idx, int* pos_out, float* scores_out, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p->f_grid);
+  cfg.blockDim = dim3(F_THREADS);
+  cfg.dynamicSmemBytes = p->f_smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeCooperative;
+  at[0].val.cooperative = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_filter_fused<T, VPL>, tok, D, (const ImgDesc*)p->d_desc,
+                            (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
+                            attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
+                            c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
+                            p->f_nstage, p->f_max_piece);
+}
+
+template <class T, int VPL>
 void launch_colsum_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, cudaStream_t st) {
   constexpr int E = VecTraits<T>::E;
   k_colsum<T, VPL, true><<<dim3(p->n_rows, 1), 256, VPL * 32 * E * sizeof(float), st>>>(
@@ -511,6 +630,20 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
+  if (p->fused) {
+    prof_tick(c, st, "filter_fused");
+    cudaError_t fe;
+#define FICOCO_FUSED_GO(V) fe = launch_filter_fused<T, V>(c, p, tok, D, attn, attn_rows, cA, pos, window, coef, \
+                                                          penalty, kept_idx, pos_out, scores_out, st)
+    if (vpl <= 1) FICOCO_FUSED_GO(1);
+    else if (vpl <= 2) FICOCO_FUSED_GO(2);
+    else if (vpl <= 4) FICOCO_FUSED_GO(4);
+    else if (vpl <= 5) FICOCO_FUSED_GO(5);
+    else FICOCO_FUSED_GO(8);
+#undef FICOCO_FUSED_GO
+    if (fe != cudaSuccess) { c->last_cuda = (int)fe; return FICOCO_ERR_CUDA; }
+    c->launches += 1;
+  } else {
   prof_tick(c, st, vpl <= 8 ? "colsum" : "rownorm");
   if (vpl <= 8) {
     if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
@@ -536,6 +669,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
                                                   pos_out, c->status);
   c->launches += 2;
+  }
   if (p->n_corr > 0) {
     if (p->umma && tmean == nullptr && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
@@ -681,6 +815,11 @@ extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_statu
   CUDA_TRY(c, cudaMemcpyAsync(&v, c->status, 4, cudaMemcpyDeviceToHost, st));
   CUDA_TRY(c, cudaMemsetAsync(c->status, 0, 4, st));
   CUDA_TRY(c, cudaStreamSynchronize(st));
+  if (v & STATUS_TIMEOUT) {
+    // a kernel gave up half-way: its per-image counters may be left non-zero
+    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 2 * (size_t)c->max_batch * sizeof(int), st));
+    CUDA_TRY(c, cudaStreamSynchronize(st));
+  }
   *device_status = (int)v;
   return FICOCO_OK;
 }

@@ -206,55 +206,51 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
 }
 
 // ---------------------------------------------------------------------------------------
-// Local penalty + top-N^S selection.  One CTA (1024 threads) per image.
+// Local penalty + top-N^S selection of one image by `nthr` threads (tid 0..nthr-1) that
+// synchronise on hardware barrier `bar`.
 //   1. every alive token bids (score key, lower index wins ties) for its window with a
 //      64-bit shared-memory max; the winner's score is multiplied by `coef`;
 //   2. an 8-bit-per-pass radix select over order-preserving keys finds the N^S-th largest
 //      score; ties at the threshold go to the lower index;
 //   3. a block scan turns the membership flags into ascending index lists S and T, the kept
 //      row indices and the surviving grid positions.
+// `keys` (np words) and `win` (one 64-bit word per window) are shared-memory work areas.
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ desc,
-                                                 const float* __restrict__ s_raw,
-                                                 const int* __restrict__ pos, int window, float coef,
-                                                 int penalty, float* __restrict__ s_pen,
-                                                 float* __restrict__ scores_out,
-                                                 int* __restrict__ S_idx, int* __restrict__ T_idx,
-                                                 int* __restrict__ kept_idx, int* __restrict__ pos_out,
-                                                 unsigned* __restrict__ status) {
-  extern __shared__ unsigned char sm_raw[];
-  const ImgDesc d = desc[blockIdx.x];
-  const int np = d.np;
-  uint32_t* keys = reinterpret_cast<uint32_t*>(sm_raw);                       // [np]
-  unsigned long long* win =
-      reinterpret_cast<unsigned long long*>(sm_raw + (((size_t)np * 4 + 7) & ~(size_t)7));
-  __shared__ int hist[256];
-  __shared__ int warp_tot[33];
-  __shared__ uint32_t sh_prefix;
-  __shared__ int sh_remaining;
+struct SelectShared {
+  int hist[256];
+  int warp_tot[33];
+  uint32_t prefix;
+  int remaining;
+};
 
-  const int tid = threadIdx.x;
+__device__ __forceinline__ void select_image(
+    const ImgDesc& d, const float* s_raw, const int* __restrict__ pos, int window, float coef,
+    int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
+    int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
+    unsigned* __restrict__ status, uint32_t* keys, unsigned long long* win, SelectShared& sh,
+    int tid, int nthr, int bar) {
+  const int np = d.np;
   const int nwc = (d.gw + window - 1) / window;
   const int nwr = (d.gh + window - 1) / window;
   const int nwin = penalty ? nwc * nwr : 0;
 
-  for (int i = tid; i < nwin; i += 1024) win[i] = 0ull;
-  __syncthreads();
+  for (int i = tid; i < nwin; i += nthr) win[i] = 0ull;
+  cta_sync(bar, nthr);
 
   // ---- local penalty ------------------------------------------------------------------
   if (penalty) {
-    for (int i = tid; i < np; i += 1024) {
+    for (int i = tid; i < np; i += nthr) {
       const int p = pos ? pos[d.patch0 + i] : i;
       if (p < 0 || p >= d.gh * d.gw) { atomicOr(status, STATUS_POS_RANGE); continue; }
       const int wid = (p / d.gw / window) * nwc + (p % d.gw) / window;
       const unsigned long long bid =
-          ((unsigned long long)order_key(s_raw[d.patch0 + i]) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)i);
+          ((unsigned long long)order_key(__ldcg(s_raw + d.patch0 + i)) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)i);
       atomicMax(&win[wid], bid);
     }
-    __syncthreads();
+    cta_sync(bar, nthr);
   }
-  for (int i = tid; i < np; i += 1024) {
-    float s = s_raw[d.patch0 + i];
+  for (int i = tid; i < np; i += nthr) {
+    float s = __ldcg(s_raw + d.patch0 + i);
     if (penalty) {
       const int p = pos ? pos[d.patch0 + i] : i;
       if (p >= 0 && p < d.gh * d.gw) {
@@ -266,32 +262,32 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
     if (scores_out) scores_out[d.patch0 + i] = s;
     keys[i] = order_key(s);
   }
-  __syncthreads();
+  cta_sync(bar, nthr);
 
   // ---- radix select: key of the n_src-th largest ------------------------------------------
   const int k = d.n_src;
   uint32_t thr = 0;       // threshold key
   int need_eq = 0;        // how many keys equal to thr are selected (lowest indices)
   if (k > 0 && k < np) {
-    if (tid == 0) { sh_prefix = 0; sh_remaining = k; }
+    if (tid == 0) { sh.prefix = 0; sh.remaining = k; }
     uint32_t mask = 0;
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      if (tid < 256) hist[tid] = 0;
-      __syncthreads();
-      const uint32_t prefix = sh_prefix;
-      for (int i = tid; i < np; i += 1024) {
+      if (tid < 256) sh.hist[tid] = 0;
+      cta_sync(bar, nthr);
+      const uint32_t prefix = sh.prefix;
+      for (int i = tid; i < np; i += nthr) {
         const uint32_t key = keys[i];
-        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255], 1);
       }
-      __syncthreads();
+      cta_sync(bar, nthr);
       if (tid < 32) {
         // lane l owns bins 255-8l .. 248-8l (descending); find where the running count
         // from the top reaches `remaining`
-        const int remaining = sh_remaining;
+        const int remaining = sh.remaining;
         int c[8], tot = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = hist[255 - 8 * tid - j]; tot += c[j]; }
+        for (int j = 0; j < 8; ++j) { c[j] = sh.hist[255 - 8 * tid - j]; tot += c[j]; }
         int inc = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -304,23 +300,23 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             if (cum < remaining && cum + c[j] >= remaining) {
-              sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
-              sh_remaining = remaining - cum;
+              sh.prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh.remaining = remaining - cum;
             }
             cum += c[j];
           }
         }
       }
       mask |= 0xFFu << shift;
-      __syncthreads();
+      cta_sync(bar, nthr);
     }
-    thr = sh_prefix;
-    need_eq = sh_remaining;
+    thr = sh.prefix;
+    need_eq = sh.remaining;
   }
 
   // ---- ordered compaction into S and T ------------------------------------------------------
   int eq_base = 0, sel_base = 0;
-  for (int base = 0; base < np; base += 1024) {
+  for (int base = 0; base < np; base += nthr) {
     const int i = base + tid;
     const bool valid = i < np;
     const uint32_t key = valid ? keys[i] : 0u;
@@ -329,10 +325,10 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
     else if (k >= np) { gt = valid; eq = false; }
     else { gt = valid && key > thr; eq = valid && key == thr; }
     int tot;
-    const int eq_rank = eq_base + block_exclusive_scan(eq ? 1 : 0, warp_tot, &tot);
+    const int eq_rank = eq_base + block_exclusive_scan(eq ? 1 : 0, sh.warp_tot, &tot, bar, nthr);
     eq_base += tot;
     const bool sel = gt || (eq && eq_rank < need_eq);
-    const int sel_rank = sel_base + block_exclusive_scan(sel ? 1 : 0, warp_tot, &tot);
+    const int sel_rank = sel_base + block_exclusive_scan(sel ? 1 : 0, sh.warp_tot, &tot, bar, nthr);
     sel_base += tot;
     if (valid) {
       if (sel) {
@@ -345,9 +341,28 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
       }
     }
   }
-  for (int i = tid; i < d.n_cls; i += 1024) kept_idx[d.out_row0 + i] = i;
-  for (int i = tid; i < d.n_tail; i += 1024)
+  for (int i = tid; i < d.n_cls; i += nthr) kept_idx[d.out_row0 + i] = i;
+  for (int i = tid; i < d.n_tail; i += nthr)
     kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
+}
+
+// One CTA (1024 threads) per image.
+__global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ desc,
+                                                 const float* __restrict__ s_raw,
+                                                 const int* __restrict__ pos, int window, float coef,
+                                                 int penalty, float* __restrict__ s_pen,
+                                                 float* __restrict__ scores_out,
+                                                 int* __restrict__ S_idx, int* __restrict__ T_idx,
+                                                 int* __restrict__ kept_idx, int* __restrict__ pos_out,
+                                                 unsigned* __restrict__ status) {
+  extern __shared__ unsigned char sm_raw[];
+  __shared__ SelectShared sh;
+  const ImgDesc d = desc[blockIdx.x];
+  uint32_t* keys = reinterpret_cast<uint32_t*>(sm_raw);
+  unsigned long long* win =
+      reinterpret_cast<unsigned long long*>(sm_raw + (((size_t)d.np * 4 + 7) & ~(size_t)7));
+  select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
+               status, keys, win, sh, threadIdx.x, 1024, 0);
 }
 
 }  // namespace ficoco
