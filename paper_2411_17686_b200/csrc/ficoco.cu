@@ -499,14 +499,14 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     p->f_grid = (int)cta_first.size() - 1;
     p->f_max_piece = p->max_rc;
     const size_t stage = (size_t)FROWS * key.dim * esz;
-    const size_t fixed = (size_t)FROWS * key.dim * 4 + (size_t)p->f_max_piece * 4 + 256;
+    const size_t fixed = (size_t)FFOLD * key.dim * 4 + (size_t)p->f_max_piece * 4 + 256;
     const size_t budget = 216 * 1024;
     int ns = budget > fixed ? (int)((budget - fixed) / stage) : 0;
     if (ns > F_MAXSTAGE) ns = F_MAXSTAGE;
     size_t sel_need = 0;
     for (int b = 0; b < B; ++b) {
       const ImgDesc& d = p->h_desc[b];
-      const size_t need = align_up((size_t)d.np * 4, 8) + (key.mode == 0 ? (size_t)d.gh * d.gw * 8 : 0);
+      const size_t need = select_work_bytes(d.np, key.mode == 0 ? d.gh * d.gw : 0);
       if (need > sel_need) sel_need = need;
     }
     if (ns < 2 || sel_need > (size_t)ns * stage) p->fused = false;
@@ -663,7 +663,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   prof_tick(c, st, "score");
   k_score<T><<<p->n_rows, 256, (size_t)(D + p->max_rc) * sizeof(float), st>>>(
       tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
-  const size_t sel_smem = align_up((size_t)p->max_np * 4, 8) + (size_t)(penalty ? p->max_nwin_cells : 0) * 8 + 16;
+  const size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
   prof_tick(c, st, "select");
   k_select<<<p->key.batch, 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,

@@ -214,8 +214,13 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
 //      score; ties at the threshold go to the lower index;
 //   3. a block scan turns the membership flags into ascending index lists S and T, the kept
 //      row indices and the surviving grid positions.
-// `keys` (np words) and `win` (one 64-bit word per window) are shared-memory work areas.
+// `work` is a shared-memory area of select_work_bytes(np, windows) bytes: the scores and grid
+// positions are read from global memory once and kept there with the keys and window bids.
 // ---------------------------------------------------------------------------------------
+__host__ __device__ inline size_t select_work_bytes(int np, int nwin) {
+  return (size_t)np * 12 + 8 + (size_t)nwin * 8;
+}
+
 struct SelectShared {
   int hist[256];
   int warp_tot[33];
@@ -227,32 +232,39 @@ __device__ __forceinline__ void select_image(
     const ImgDesc& d, const float* s_raw, const int* __restrict__ pos, int window, float coef,
     int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
     int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
-    unsigned* __restrict__ status, uint32_t* keys, unsigned long long* win, SelectShared& sh,
-    int tid, int nthr, int bar) {
+    unsigned* __restrict__ status, unsigned char* work, SelectShared& sh, int tid, int nthr, int bar) {
   const int np = d.np;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(work);
+  float* sc = reinterpret_cast<float*>(work + (size_t)np * 4);
+  int* pp = reinterpret_cast<int*>(work + (size_t)np * 8);
+  unsigned long long* win = reinterpret_cast<unsigned long long*>(work + (((size_t)np * 12 + 7) & ~(size_t)7));
   const int nwc = (d.gw + window - 1) / window;
   const int nwr = (d.gh + window - 1) / window;
   const int nwin = penalty ? nwc * nwr : 0;
 
   for (int i = tid; i < nwin; i += nthr) win[i] = 0ull;
+  for (int i = tid; i < np; i += nthr) {
+    sc[i] = __ldcg(s_raw + d.patch0 + i);
+    pp[i] = pos ? pos[d.patch0 + i] : i;
+  }
   cta_sync(bar, nthr);
 
   // ---- local penalty ------------------------------------------------------------------
   if (penalty) {
     for (int i = tid; i < np; i += nthr) {
-      const int p = pos ? pos[d.patch0 + i] : i;
+      const int p = pp[i];
       if (p < 0 || p >= d.gh * d.gw) { atomicOr(status, STATUS_POS_RANGE); continue; }
       const int wid = (p / d.gw / window) * nwc + (p % d.gw) / window;
       const unsigned long long bid =
-          ((unsigned long long)order_key(__ldcg(s_raw + d.patch0 + i)) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)i);
+          ((unsigned long long)order_key(sc[i]) << 32) | (unsigned)(0xFFFFFFFFu - (unsigned)i);
       atomicMax(&win[wid], bid);
     }
     cta_sync(bar, nthr);
   }
   for (int i = tid; i < np; i += nthr) {
-    float s = __ldcg(s_raw + d.patch0 + i);
+    float s = sc[i];
     if (penalty) {
-      const int p = pos ? pos[d.patch0 + i] : i;
+      const int p = pp[i];
       if (p >= 0 && p < d.gh * d.gw) {
         const int wid = (p / d.gw / window) * nwc + (p % d.gw) / window;
         if ((unsigned)(win[wid] & 0xFFFFFFFFull) == 0xFFFFFFFFu - (unsigned)i) s *= coef;
@@ -337,7 +349,7 @@ __device__ __forceinline__ void select_image(
         const int tp = i - sel_rank;
         T_idx[d.tgt0 + tp] = i;
         kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
-        if (pos_out) pos_out[d.tgt0 + tp] = pos ? pos[d.patch0 + i] : i;
+        if (pos_out) pos_out[d.tgt0 + tp] = pp[i];
       }
     }
   }
@@ -358,11 +370,8 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
   extern __shared__ unsigned char sm_raw[];
   __shared__ SelectShared sh;
   const ImgDesc d = desc[blockIdx.x];
-  uint32_t* keys = reinterpret_cast<uint32_t*>(sm_raw);
-  unsigned long long* win =
-      reinterpret_cast<unsigned long long*>(sm_raw + (((size_t)d.np * 4 + 7) & ~(size_t)7));
   select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-               status, keys, win, sh, threadIdx.x, 1024, 0);
+               status, sm_raw, sh, threadIdx.x, 1024, 0);
 }
 
 }  // namespace ficoco

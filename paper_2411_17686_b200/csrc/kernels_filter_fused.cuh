@@ -1,12 +1,13 @@
 // Filter stage as one persistent kernel (Eq. 1, local penalty, top-N^S selection).
 //
 // Launched cooperatively with one CTA per SM at most, so all CTAs are co-resident.  Every CTA
-// owns a fixed list of "pieces" (consecutive patch rows of one image).  Warp 8 streams the
-// rows of its pieces, 8 rows per stage, into a shared-memory ring with bulk copies (TMA);
-// the 8 consumer warps take one row each per stage.
+// owns a fixed list of "pieces" (consecutive patch rows of one image).  Warp 16 streams the
+// rows of its pieces, 16 rows (one bulk copy) per stage, into a shared-memory ring (TMA);
+// the 16 consumer warps take one row each per stage.
 //   pass 1  rn_i = 1/||x_i||, column sums of the normalised rows -> one partial per piece;
 //           the piece's image counter is bumped;
-//   pass 2  (rows streamed again, now from L2) once all pieces of the image are in:
+//   pass 2  (rows read again, now L2-resident, with plain 16-byte loads, three rows in flight
+//           per warp) once all pieces of the image are in:
 //           v_i = rn_i (x_i . sum of partials) / Np,  s_i = cA v_i - (1 - cA) a_i;
 //           the CTA that finishes the last piece of an image runs the local penalty and the
 //           radix select for that image and resets the image's counters.
@@ -18,12 +19,15 @@
 
 namespace ficoco {
 
-constexpr int FROWS = 8;          // rows per ring stage == consumer warps
-constexpr int F_NCONS = 256;      // consumer threads
-constexpr int F_THREADS = 288;    // + one producer warp
+constexpr int FWARPS = 16;        // consumer warps
+constexpr int FROWS = 16;         // rows per ring stage (one 16-row bulk copy), one per consumer warp
+constexpr int FFOLD = 8;          // rows of the fold buffer (warps w and w + 8 share a row)
+constexpr int F_NCONS = 512;      // consumer threads
+constexpr int F_THREADS = 544;    // + one producer warp
 constexpr int F_MAXSTAGE = 16;
 constexpr int F_MAXWON = 32;      // pieces per CTA (and therefore selections it can win)
 constexpr int F_POLL_LIMIT = 1 << 20;
+constexpr int F_P2ROWS = 3;       // rows a warp keeps in flight in pass 2
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
@@ -53,39 +57,38 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   const int stage_bytes = FROWS * row_bytes;
   const int nvec = D / E;
   unsigned char* ring = fs_raw;
-  float* fold = reinterpret_cast<float*>(fs_raw + (size_t)nstage * stage_bytes);   // [8][D], msum aliases fold[0]
-  float* a_s = fold + (size_t)FROWS * D;                                           // [max_piece]
+  float* fold = reinterpret_cast<float*>(fs_raw + (size_t)nstage * stage_bytes);   // [FFOLD][D], msum aliases fold[0]
+  float* a_s = fold + (size_t)FFOLD * D;                                            // [max_piece]
   const int p_begin = cta_first[blockIdx.x], p_end = cta_first[blockIdx.x + 1];
 
   if (tid == 0) {
-    for (int s = 0; s < nstage; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FROWS); }
+    for (int s = 0; s < nstage; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FWARPS); }
     nwon = 0;
     failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  if (warp == FROWS) {
-    // ------------------------------- producer ---------------------------------------------
+  if (warp == FWARPS) {
+    // ------------------------------- producer (pass 1 only) -------------------------------
     if (lane == 0) {
       int seq = 0;
       bool ok = true;
-      for (int pass = 0; pass < 2 && ok; ++pass)
-        for (int pi = p_begin; pi < p_end && ok; ++pi) {
-          const WorkItem w = pieces[pi];
-          const ImgDesc d = desc[w.img];
-          const unsigned char* base =
-              reinterpret_cast<const unsigned char*>(tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D);
-          for (int g = 0; g * FROWS < w.nrows && ok; ++g, ++seq) {
-            const int s = seq % nstage;
-            if (seq >= nstage) ok = mbar_wait(&empty_bar[s], ((seq / nstage) - 1) & 1);
-            if (!ok) break;
-            const int rows = min(FROWS, w.nrows - g * FROWS);
-            mbar_expect_tx(&full_bar[s], (uint32_t)(rows * row_bytes));
-            bulk_load(ring + (size_t)s * stage_bytes, base + (size_t)g * stage_bytes,
-                      (uint32_t)(rows * row_bytes), &full_bar[s]);
-          }
+      for (int pi = p_begin; pi < p_end && ok; ++pi) {
+        const WorkItem w = pieces[pi];
+        const ImgDesc d = desc[w.img];
+        const unsigned char* base =
+            reinterpret_cast<const unsigned char*>(tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D);
+        for (int g = 0; g * FROWS < w.nrows && ok; ++g, ++seq) {
+          const int s = seq % nstage;
+          if (seq >= nstage) ok = mbar_wait(&empty_bar[s], ((seq / nstage) - 1) & 1);
+          if (!ok) break;
+          const int rows = min(FROWS, w.nrows - g * FROWS);
+          mbar_expect_tx(&full_bar[s], (uint32_t)(rows * row_bytes));
+          bulk_load(ring + (size_t)s * stage_bytes, base + (size_t)g * stage_bytes,
+                    (uint32_t)(rows * row_bytes), &full_bar[s]);
         }
+      }
       if (!ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     }
     return;
@@ -110,16 +113,24 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       if (r < w.nrows) {
         const unsigned char* rp = ring + (size_t)s * stage_bytes + (size_t)warp * row_bytes;
         uint4 u[VPL];
-        float ss = 0.f;
+        float ssk[VPL];
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
           const int v = lane + 32 * k;
           u[k] = v < nvec ? *reinterpret_cast<const uint4*>(rp + (size_t)v * 16) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
           float f[E];
           unpack(u[k], f, (const T*)nullptr);
+          float t = 0.f;
 #pragma unroll
-          for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
+          for (int e = 0; e < E; ++e) t = fmaf(f[e], f[e], t);
+          ssk[k] = t;
         }
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) ss += ssk[k];
         ss = warp_sum(ss);
         const float s1 = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
         if (lane == 0) rn[d.patch0 + w.r0 + r] = s1;
@@ -134,13 +145,35 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty_bar[s]);
     }
-    // fold the 8 warps in a fixed order -> partial of this piece
+    // fold the 16 warps in a fixed order -> partial of this piece: warps 0-7 store, warps 8-15
+    // add into the row of warp - 8, then the 8 rows are summed per column
+    if (warp < FFOLD) {
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int v = lane + 32 * k;
-      if (v < nvec) {
+      for (int k = 0; k < VPL; ++k) {
+        const int v = lane + 32 * k;
+        if (v < nvec) {
+          float4* dst = reinterpret_cast<float4*>(fold + (size_t)warp * D + (size_t)v * E);
+          dst[0] = make_float4(acc[k][0], acc[k][1], acc[k][2], acc[k][3]);
+          if (E == 8) dst[1] = make_float4(acc[k][E - 4], acc[k][E - 3], acc[k][E - 2], acc[k][E - 1]);
+        }
+      }
+    }
+    cta_sync(1, F_NCONS);
+    if (warp >= FFOLD) {
 #pragma unroll
-        for (int e = 0; e < E; ++e) fold[(size_t)warp * D + (size_t)v * E + e] = acc[k][e];
+      for (int k = 0; k < VPL; ++k) {
+        const int v = lane + 32 * k;
+        if (v < nvec) {
+          float4* dst = reinterpret_cast<float4*>(fold + (size_t)(warp - FFOLD) * D + (size_t)v * E);
+          float4 x = dst[0];
+          x.x += acc[k][0]; x.y += acc[k][1]; x.z += acc[k][2]; x.w += acc[k][3];
+          dst[0] = x;
+          if (E == 8) {
+            float4 y = dst[1];
+            y.x += acc[k][E - 4]; y.y += acc[k][E - 3]; y.z += acc[k][E - 2]; y.w += acc[k][E - 1];
+            dst[1] = y;
+          }
+        }
       }
     }
     cta_sync(1, F_NCONS);
@@ -148,15 +181,16 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     for (int c = tid; c < D; c += F_NCONS) {
       float t = 0.f;
 #pragma unroll
-      for (int ww = 0; ww < FROWS; ++ww) t += fold[(size_t)ww * D + c];
+      for (int ww = 0; ww < FFOLD; ++ww) t += fold[(size_t)ww * D + c];
       pout[c] = t;
     }
     __threadfence();
     cta_sync(1, F_NCONS);
     if (tid == 0) atomicAdd(&cnt[w.img], 1);
   }
+  if (!ok && lane == 0) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
 
-  // pass 2: scores
+  // pass 2: scores; the rows are L2-resident now and are read with plain loads
   for (int pi = p_begin; pi < p_end; ++pi) {
     const WorkItem w = pieces[pi];
     const ImgDesc d = desc[w.img];
@@ -168,48 +202,65 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       }
       if (!in) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     }
-    cta_sync(1, F_NCONS);
-    float* msum = fold;
-    for (int c = tid; c < D; c += F_NCONS) {
-      float t = 0.f;
-      for (int k = 0; k < d.n_chunks; ++k) t += __ldcg(partial + (size_t)(d.chunk0 + k) * D + c);
-      msum[c] = t;
-    }
     const float inv_h = 1.0f / (float)H;
-    for (int r = tid; r < w.nrows; r += F_NCONS) {
+    for (int r = tid; r < w.nrows; r += F_NCONS) {     // attention term, does not depend on the wait
       const float* a = attn + d.attn0 + w.r0 + r;
       float t = 0.f;
       for (int h = 0; h < H; ++h) t += __ldg(a + (size_t)h * d.np);
       a_s[r] = t * inv_h;
     }
     cta_sync(1, F_NCONS);
+    float* msum = fold;
+    for (int c = tid; c < D; c += F_NCONS) {
+      float t = 0.f;
+      for (int k0 = 0; k0 < d.n_chunks; k0 += 8) {
+        float q[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          q[k] = k0 + k < d.n_chunks ? __ldcg(partial + (size_t)(d.chunk0 + k0 + k) * D + c) : 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t += q[k];
+      }
+      msum[c] = t;
+    }
+    cta_sync(1, F_NCONS);
     const float inv_np = 1.0f / (float)d.np;
-    for (int g = 0; g * FROWS < w.nrows; ++g, ++seq) {
-      const int s = seq % nstage;
-      if (ok) ok = mbar_wait(&full_bar[s], (seq / nstage) & 1);
-      const int r = g * FROWS + warp;
-      if (r < w.nrows) {
-        const unsigned char* rp = ring + (size_t)s * stage_bytes + (size_t)warp * row_bytes;
-        float dot = 0.f;
+    const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D;
+    for (int r0 = warp; r0 < w.nrows; r0 += FWARPS * F_P2ROWS) {
+      uint4 u[F_P2ROWS][VPL];
+#pragma unroll
+      for (int j = 0; j < F_P2ROWS; ++j) {
+        const int r = r0 + j * FWARPS;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
           const int v = lane + 32 * k;
-          if (v < nvec) {
-            float f[E];
-            unpack(*reinterpret_cast<const uint4*>(rp + (size_t)v * 16), f, (const T*)nullptr);
-            const float* m = msum + (size_t)v * E;
-#pragma unroll
-            for (int e = 0; e < E; ++e) dot = fmaf(f[e], m[e], dot);
-          }
+          u[j][k] = (r < w.nrows && v < nvec) ? ldg16(base + (size_t)r * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
         }
+      }
+#pragma unroll
+      for (int j = 0; j < F_P2ROWS; ++j) {
+        const int r = r0 + j * FWARPS;
+        float dk[VPL];
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+          const int v = lane + 32 * k;
+          float f[E];
+          unpack(u[j][k], f, (const T*)nullptr);
+          const float* m = msum + (size_t)(v < nvec ? v : 0) * E;
+          float t = 0.f;
+#pragma unroll
+          for (int e = 0; e < E; ++e) t = fmaf(f[e], m[e], t);
+          dk[k] = t;
+        }
+        float dot = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) dot += dk[k];
         dot = warp_sum(dot);
-        if (lane == 0) {
+        if (lane == 0 && r < w.nrows) {
           const float v_i = dot * __ldcg(rn + d.patch0 + w.r0 + r) * inv_np;
           s_raw[d.patch0 + w.r0 + r] = cA * v_i - (1.0f - cA) * a_s[r];
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&empty_bar[s]);
     }
     __threadfence();
     cta_sync(1, F_NCONS);
@@ -219,7 +270,6 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       __threadfence();
     }
   }
-  if (!ok && lane == 0) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
   cta_sync(1, F_NCONS);
 
   // selections this CTA won (the ring is idle now and serves as work area)
@@ -228,10 +278,8 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   for (int k = 0; k < nw; ++k) {
     const int img = won[k];
     const ImgDesc d = desc[img];
-    uint32_t* keys = reinterpret_cast<uint32_t*>(ring);
-    unsigned long long* win = reinterpret_cast<unsigned long long*>(ring + (((size_t)d.np * 4 + 7) & ~(size_t)7));
     select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-                 status, keys, win, sel_sh, tid, F_NCONS, 1);
+                 status, ring, sel_sh, tid, F_NCONS, 1);
     cta_sync(1, F_NCONS);
     if (tid == 0) { cnt[img] = 0; cnt[B + img] = 0; }
   }
