@@ -29,6 +29,9 @@ UNIT = "images/s"
 B, GH, GW, D, H, KEEP = 32, 24, 24, 1024, 16, 288
 WORKLOAD = "c2 step 1: 32 images x (1 CLS + 24x24 patches) x 1024 bf16, 576 -> 288 patch tokens"
 N_INSTANCES = 8       # distinct input/output buffer sets cycled through: 8 x 58 MB > 3 x L2
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
+# profiles/ (bytes); an entry is removed when its kernel changes after the capture.
+NCU_TRAFFIC = {}
 
 
 def algorithmic_bytes() -> dict:
@@ -249,24 +252,30 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
 def kernel_roofline(name: str, avg_us: float, pk: dict, ab: dict) -> dict:
     """Roofline entry of the dominant kernel: its own algorithmic bytes (or flops) per launch
-    over its measured average duration."""
+    over its measured average duration.  Algorithmic figures per launch (one batch of B images):
+      filter_fused / colsum : X read once from HBM (+ attention)          -> hbm
+      correlate_*           : 2 * N^S * N^T * D flops per image            -> tensor
+      merge_compact         : preserved rows in (L2-resident) + rows out   -> hbm
+    """
     npatch, ns = GH * GW, GH * GW - KEEP
     src = pk["source"]
-    if name == "correlate":
+    if name.startswith("correlate"):
         flops = 2.0 * B * ns * KEEP * D
         ach = flops / (avg_us * 1e-6) / 1e12
         return {"kernel": name, "bound": "tensor", "achieved": ach, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": ach / pk["bf16_tflops"], "traffic": None, "of": src,
+                "frac": ach / pk["bf16_tflops"], "traffic": NCU_TRAFFIC.get(name), "of": src,
                 "algorithmic_flops_per_launch": flops}
     per = {
-        "colsum": ab["tokens_in"],                                   # X read once from HBM
-        "score": ab["tokens_in"] + ab["attn"],                       # X again (L2-resident) + attention
-        "merge_compact": ab["tokens_out"] * 2,                       # rows in, rows out
+        "filter_fused": ab["tokens_in"] + ab["attn"] + B * npatch * 4,   # X once, attention, pos
+        "colsum": ab["tokens_in"],
+        "score": ab["tokens_in"] + ab["attn"],
+        "merge_compact": ab["tokens_out"] * 2,
         "select": B * npatch * 4 * 3, "finalize": B * ns * 16, "rownorm": ab["tokens_in"],
     }.get(name, ab["total"])
     ach = per / (avg_us * 1e-6) / 1e9
     return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
-            "frac": ach / pk["hbm_gbs"], "traffic": None, "of": src, "algorithmic_bytes_per_launch": per}
+            "frac": ach / pk["hbm_gbs"], "traffic": NCU_TRAFFIC.get(name), "of": src,
+            "algorithmic_bytes_per_launch": per}
 
 
 def cpu_baseline(batch, budget_s: float = 12.0) -> dict:
