@@ -31,6 +31,7 @@ struct ImgDesc {
   float frac;      // interpolation weight of the quantile
   int nsplit;      // column splits of the correlate step
   int cols_per_split;
+  int corr_items;  // correlate work items (CTAs) of this image
   int chunk0;      // first row chunk (column-sum partials)
   int n_chunks;
   long long attn0; // offset (floats) of this image's attention block

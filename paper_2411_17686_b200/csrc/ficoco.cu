@@ -59,6 +59,7 @@ struct Plan {
   int f_grid = 0, f_nstage = 0, f_max_piece = 0, f_vpl = 0;
   size_t f_smem = 0;
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
+  bool need_finalize = false;   // some image merges nothing: its per-token counts are zeroed by a kernel
   bool umma = false;
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
   size_t um_smem = 0;
@@ -263,7 +264,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
-  const size_t o_icnt = carve(2 * B * 4);
+  const size_t o_icnt = carve(3 * B * 4);
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
@@ -345,6 +346,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   std::vector<WorkItem> rows, corr, outw;
   long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
   p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = p->max_list = 0;
+  p->need_finalize = false;
   p->umma = key.mode == 0 && key.dtype == FICOCO_BF16 && key.dim % UKB == 0;
   const int tile_rows_max = p->umma ? UM : CBM;       // source rows per correlate CTA
   const int col_granule = p->umma ? 16 : CBN;
@@ -436,7 +438,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     }
     if (rc > p->max_rc) p->max_rc = rc;
     // correlate
-    d.nsplit = 1; d.cols_per_split = d.n_tgt > 0 ? d.n_tgt : 1;
+    d.nsplit = 1; d.cols_per_split = d.n_tgt > 0 ? d.n_tgt : 1; d.corr_items = 0;
+    if (d.list_len == 0 && d.n_src > 0) p->need_finalize = true;
     if (d.list_len > 0) {
       int ns = want_split;
       const int max_by_cols = (d.n_tgt + col_granule - 1) / col_granule;
@@ -446,6 +449,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       if (p->umma && cps > UN_MAX) cps = UN_MAX;
       ns = (d.n_tgt + cps - 1) / cps;
       d.nsplit = ns; d.cols_per_split = cps;
+      const size_t corr_before = corr.size();
       // source tiles of equal size (rounded to 8 rows)
       const int ntile = (d.n_src + tile_rows_max - 1) / tile_rows_max;
       int trows = (d.n_src + ntile - 1) / ntile;
@@ -457,6 +461,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
           WorkItem w; w.img = b; w.r0 = s0; w.nrows = (d.n_src - s0 < trows) ? d.n_src - s0 : trows; w.aux = sp;
           corr.push_back(w);
         }
+      d.corr_items = (int)(corr.size() - corr_before);
       part0 += (long long)d.n_src * ns * d.list_len;
       ent0 += (long long)d.n_src * d.list_len;
     }
@@ -677,7 +682,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
   k_correlate_umma<NS, LC><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
       c->S_idx, c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes,        \
-      p->um_tmem_cols)
+      p->um_tmem_cols, c->img_cnt + 2 * c->max_batch, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                                  \
@@ -692,11 +697,13 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     } else {
       prof_tick(c, st, "correlate_simt");
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
-                                                     c->T_idx, tmean, M, gamma, c->part_val, c->part_idx);
+                                                     c->T_idx, tmean, M, gamma, c->part_val, c->part_idx,
+                                                     c->img_cnt + 2 * c->max_batch, c->corr_cnt, c->tau,
+                                                     c->e_tgt, c->e_w, c->e_c);
     }
     c->launches += 1;
   }
-  if (p->max_src > 0) {
+  if (p->max_src > 0 && p->need_finalize) {
     prof_tick(c, st, "finalize");
     k_finalize_src<<<dim3(p->key.batch, (p->max_src + 255) / 256), 256, 0, st>>>(
         p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c);
@@ -817,7 +824,7 @@ extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_statu
   CUDA_TRY(c, cudaStreamSynchronize(st));
   if (v & STATUS_TIMEOUT) {
     // a kernel gave up half-way: its per-image counters may be left non-zero
-    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 2 * (size_t)c->max_batch * sizeof(int), st));
+    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 3 * (size_t)c->max_batch * sizeof(int), st));
     CUDA_TRY(c, cudaStreamSynchronize(st));
   }
   *device_status = (int)v;

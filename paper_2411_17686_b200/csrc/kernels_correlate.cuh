@@ -10,6 +10,11 @@ constexpr int CBM = 64;   // source rows per CTA
 constexpr int CBN = 64;   // target columns per tile
 constexpr int CKC = 16;   // reduction chunk
 
+__device__ __forceinline__ void correlate_tail(
+    const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
+    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem);
+
 // ---------------------------------------------------------------------------------------
 // fp32 SIMT correlate (the path for fp32 tokens, where 1e-5 relative accuracy rules out
 // bf16 tensor-core products).  One CTA owns up to 64 discarded tokens of one image and one
@@ -24,7 +29,10 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     const WorkItem* __restrict__ work, const float* __restrict__ rn,
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     const float* __restrict__ tmean, int M, float gamma,
-    float* __restrict__ part_val, int* __restrict__ part_idx) {
+    float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ img_done,
+    int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
+    float* __restrict__ e_w, float* __restrict__ e_c) {
+  __shared__ int is_last;
   __shared__ __align__(16) float As[CKC][CBM + 4];
   __shared__ __align__(16) float Bs[CKC][CBN + 4];
   __shared__ float Cs[CBM][CBN + 1];
@@ -183,6 +191,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     part_val[o] = lv[r][k];
     part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
   }
+  correlate_tail(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
@@ -197,14 +206,11 @@ namespace ficoco {
 // e_w (alpha), e_c (the L largest C, descending).
 // grid = (images, ceil(max N^S / 256)).
 // ---------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_finalize_src(
-    const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
-    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
-    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
-  const ImgDesc d = desc[blockIdx.x];
+__device__ __forceinline__ void finalize_source(
+    const ImgDesc& d, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
+    int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
+    float* __restrict__ e_w, float* __restrict__ e_c) {
   const int L = d.list_len;
-  const int s = blockIdx.y * 256 + threadIdx.x;
-  if (s >= d.n_src) return;
   const size_t o = (size_t)(d.src0 + s);
   if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; return; }
   float v[KCAP];
@@ -214,8 +220,8 @@ __global__ void __launch_bounds__(256) k_finalize_src(
   const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
   const int ne = d.nsplit * L;
   for (int e = 0; e < ne; ++e) {
-    float cv = part_val[pbase + e];
-    int ci = part_idx[pbase + e];
+    float cv = __ldcg(part_val + pbase + e);
+    int ci = __ldcg(part_idx + pbase + e);
     if (ci < 0) continue;
 #pragma unroll
     for (int k = 0; k < KCAP; ++k) {
@@ -253,6 +259,38 @@ __global__ void __launch_bounds__(256) k_finalize_src(
       e_c[eb + k] = v[k];
     }
   }
+}
+
+__global__ void __launch_bounds__(256) k_finalize_src(
+    const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
+    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
+  const ImgDesc d = desc[blockIdx.x];
+  const int s = blockIdx.y * 256 + threadIdx.x;
+  if (s >= d.n_src) return;
+  finalize_source(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
+}
+
+// Tail of a correlate CTA: once its partial lists are written it bumps the image's counter;
+// the CTA that completes the image (the last of d.corr_items) turns the partial lists of all of
+// the image's discarded tokens into tau_i, J_i and alpha_ij, and resets the counter.  Nobody
+// waits: there is no spinning.  Call from all threads of the CTA.
+__device__ __forceinline__ void correlate_tail(
+    const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
+    const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int old = atomicAdd(&img_done[img], 1);
+    const int last = old == d.corr_items - 1;
+    if (last) { __threadfence(); img_done[img] = 0; }
+    *is_last_smem = last;
+  }
+  __syncthreads();
+  if (*is_last_smem)
+    for (int s = threadIdx.x; s < d.n_src; s += blockDim.x)
+      finalize_source(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
 }  // namespace ficoco

@@ -17,6 +17,7 @@
 #include <math_constants.h>
 #include "async_ops.cuh"
 #include "common.cuh"
+#include "kernels_correlate.cuh"
 
 namespace ficoco {
 
@@ -72,13 +73,14 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const WorkItem* __restrict__ work, const float* __restrict__ rn,
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
-    int stage_bytes, int a_bytes, int tmem_cols) {
+    int stage_bytes, int a_bytes, int tmem_cols, int* __restrict__ img_done, int* __restrict__ corr_cnt,
+    float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
   __shared__ int rowS[UM], rowT[UN_MAX];
   __shared__ float rnT[UN_MAX];
-  __shared__ int failed, acc_committed;
+  __shared__ int failed, acc_committed, is_last;
 
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
@@ -238,6 +240,7 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                  : "memory");
   }
+  correlate_tail(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco

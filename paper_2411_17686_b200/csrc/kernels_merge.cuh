@@ -5,7 +5,7 @@
 namespace ficoco {
 
 constexpr int MROWS = 8;       // output rows per CTA
-constexpr int MLIST = 768;     // (source, alpha) entries a CTA can hold in shared memory
+constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
 constexpr int MHEAVY = 8;      // rows with more sources than this are shared by all warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
@@ -63,7 +63,7 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
 //   (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
 //   * rows with few sources: one warp per row;
 //   * rows with many sources (hub targets): all 8 warps take consecutive slices of the list,
-//     the partial sums are combined in warp order through shared memory;
+//     the partial sums are combined in a fixed order through shared memory;
 //   * if the CTA's rows receive more than MLIST sources in total, a slow in-order rescan.
 template <class T>
 __global__ void __launch_bounds__(256) k_merge_scan(
@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   __shared__ float lw[MLIST];
   __shared__ int tsrc[MLIST];
   __shared__ float tw[MLIST];
-  __shared__ __align__(16) float part[8][32 * MVB][E];
+  __shared__ __align__(16) float part[4][32 * MVB][E];   // warps w and w + 4 share a row
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -216,17 +216,26 @@ __global__ void __launch_bounds__(256) k_merge_scan(
 #pragma unroll
         for (int q = 0; q < E; ++q) acc[b][q] = 0.f;
       merge_accumulate<T>(acc, pbase, D, lsrc, lw, k0, k1, vs + lane, nvec);
+      if (warp < 4) {
 #pragma unroll
-      for (int b = 0; b < MVB; ++b)
+        for (int b = 0; b < MVB; ++b)
 #pragma unroll
-        for (int q = 0; q < E; ++q) part[warp][lane + 32 * b][q] = acc[b][q];
+          for (int q = 0; q < E; ++q) part[warp][lane + 32 * b][q] = acc[b][q];
+      }
+      __syncthreads();
+      if (warp >= 4) {
+#pragma unroll
+        for (int b = 0; b < MVB; ++b)
+#pragma unroll
+          for (int q = 0; q < E; ++q) part[warp - 4][lane + 32 * b][q] += acc[b][q];
+      }
       __syncthreads();
       if (tid < 32 * MVB) {
         const int v = vs + tid;
         if (v < nvec) {
           float f[E];
           unpack(ldg16(src + (size_t)v * E), f, (const T*)nullptr);
-          for (int ww = 0; ww < 8; ++ww)
+          for (int ww = 0; ww < 4; ++ww)
 #pragma unroll
             for (int q = 0; q < E; ++q) f[q] += part[ww][tid][q];
 #pragma unroll
