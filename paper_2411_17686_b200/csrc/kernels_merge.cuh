@@ -4,74 +4,72 @@
 
 namespace ficoco {
 
-constexpr int MROWS = 8;       // output rows per CTA
+constexpr int MROWS = 32;      // output rows per CTA (four per warp)
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
 constexpr int MHEAVY = 8;      // rows with more sources than this are shared by all warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
+__device__ __forceinline__ void prefetch_l1(const void* p) {
+  asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+}
+// Lanes of a warp touch every 128-byte line of one token row.
+__device__ __forceinline__ void prefetch_row(const void* row, int row_bytes, int lane) {
+  for (int o = lane * 128; o < row_bytes; o += 32 * 128)
+    prefetch_l1(reinterpret_cast<const unsigned char*>(row) + o);
+}
+
 // acc[b][.] += sum over list entries [k0, k1) of alpha * x, for the MVB vectors v0 + 32 b of
-// each row; source rows are fetched two at a time so that 2 * MVB loads are in flight per lane.
+// each row; source rows are fetched four at a time so that 4 * MVB loads are in flight per lane.
 template <class T>
 __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>::E], const T* pbase, int D,
                                                  const int* lsrc, const float* lw, int k0, int k1,
                                                  int v0, int nvec) {
   constexpr int E = VecTraits<T>::E;
-  int k = k0;
-  for (; k + 1 < k1; k += 2) {
-    const T* x0 = pbase + (size_t)lsrc[k] * D;
-    const T* x1 = pbase + (size_t)lsrc[k + 1] * D;
-    const float a0 = lw[k], a1 = lw[k + 1];
-    uint4 u0[MVB], u1[MVB];
+  for (int k = k0; k < k1; k += 4) {
+    uint4 u[4][MVB];
+    float a[4];
 #pragma unroll
-    for (int b = 0; b < MVB; ++b) {
-      const int v = v0 + 32 * b;
-      u0[b] = v < nvec ? ldg16(x0 + (size_t)v * E) : make_uint4(0, 0, 0, 0);
-      u1[b] = v < nvec ? ldg16(x1 + (size_t)v * E) : make_uint4(0, 0, 0, 0);
-    }
+    for (int j = 0; j < 4; ++j) {
+      const bool on = k + j < k1;
+      const T* x = pbase + (size_t)lsrc[on ? k + j : k] * D;
+      a[j] = on ? lw[k + j] : 0.f;
 #pragma unroll
-    for (int b = 0; b < MVB; ++b) {
-      float f[E];
-      unpack(u0[b], f, (const T*)nullptr);
-#pragma unroll
-      for (int q = 0; q < E; ++q) acc[b][q] = fmaf(a0, f[q], acc[b][q]);
-      unpack(u1[b], f, (const T*)nullptr);
-#pragma unroll
-      for (int q = 0; q < E; ++q) acc[b][q] = fmaf(a1, f[q], acc[b][q]);
-    }
-  }
-  if (k < k1) {
-    const T* x0 = pbase + (size_t)lsrc[k] * D;
-    const float a0 = lw[k];
-#pragma unroll
-    for (int b = 0; b < MVB; ++b) {
-      const int v = v0 + 32 * b;
-      if (v < nvec) {
-        float f[E];
-        unpack(ldg16(x0 + (size_t)v * E), f, (const T*)nullptr);
-#pragma unroll
-        for (int q = 0; q < E; ++q) acc[b][q] = fmaf(a0, f[q], acc[b][q]);
+      for (int b = 0; b < MVB; ++b) {
+        const int v = v0 + 32 * b;
+        u[j][b] = (on && v < nvec) ? ldg16(x + (size_t)v * E) : make_uint4(0, 0, 0, 0);
       }
     }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int b = 0; b < MVB; ++b) {
+        float f[E];
+        unpack(u[j][b], f, (const T*)nullptr);
+#pragma unroll
+        for (int q = 0; q < E; ++q) acc[b][q] = fmaf(a[j], f[q], acc[b][q]);
+      }
   }
 }
 
-// Compress + compact.  No per-target lists are built in global memory.  A CTA owns up to 8
-// consecutive output rows of one image.  It scans the image's (source -> target) entries
-// twice (count, then fill) to file those that hit its rows into per-row lists in shared
-// memory (token index, alpha), orders every list by token index so that the fp32 sums have one
-// fixed order and no atomics touch floats, and then forms
-//   (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
-//   * rows with few sources: one warp per row;
-//   * rows with many sources (hub targets): all 8 warps take consecutive slices of the list,
-//     the partial sums are combined in a fixed order through shared memory;
-//   * if the CTA's rows receive more than MLIST sources in total, a slow in-order rescan.
+// Compress + compact.  No per-target lists are built in global memory.  A CTA owns up to 32
+// consecutive output rows of one image (warp w: rows w, w + 8, w + 16, w + 24).
+//   1. every warp resolves the input row of its output rows and prefetches those rows into L1;
+//   2. meanwhile the CTA scans the image's (source -> target) entries twice (count, then fill)
+//      to file those that hit its rows into per-row lists in shared memory (token index,
+//      alpha), prefetching the source rows, and orders every list by token index so that the
+//      fp32 sums have one fixed order and no atomics touch floats;
+//   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
+//      rows with few sources by their own warp, hub rows by all 8 warps (consecutive slices of
+//      the list, partial sums combined in a fixed order through shared memory).
+// If the CTA's rows receive more than MLIST sources in total, a slow in-order rescan is used.
 template <class T>
 __global__ void __launch_bounds__(256) k_merge_scan(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out) {
   constexpr int E = VecTraits<T>::E;
-  __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS];
+  __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
+  __shared__ float wsum_s[MROWS];
   __shared__ int lsrc[MLIST];
   __shared__ float lw[MLIST];
   __shared__ int tsrc[MLIST];
@@ -81,13 +79,24 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = D / E;
+  const int row_bytes = D * (int)sizeof(T);
   const int L = d.list_len;
   const int tp_lo = max(w.r0 - d.n_cls, 0);
   const int tp_hi = min(w.r0 + w.nrows - d.n_cls, d.n_tgt);
   const int n_ent = d.n_src * L;
   const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
 
-  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
+  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; wsum_s[tid] = 0.f; }
+  // input row of every output row (CLS / preserved token / trailing text row), prefetched
+  for (int r = warp; r < w.nrows; r += 8) {
+    const int orow = w.r0 + r;
+    int srow;
+    if (orow < d.n_cls) srow = orow;
+    else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
+    else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
+    if (lane == 0) srow_s[r] = srow;
+    prefetch_row(tokens + (size_t)(d.row0 + srow) * D, row_bytes, lane);
+  }
   __syncthreads();
   if (tp_hi > tp_lo)
     for (int e = tid; e < n_ent; e += 256) {
@@ -95,10 +104,17 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       if (t >= tp_lo && t < tp_hi) atomicAdd(&cnt[t - tp_lo], 1);
     }
   __syncthreads();
-  if (tid == 0) {
-    int s = 0;
-    for (int r = 0; r < MROWS; ++r) { beg[r] = s; s += cnt[r]; }
-    beg[MROWS] = s;
+  if (warp == 0) {
+    // exclusive scan of the 32 counts
+    const int c = cnt[lane];
+    int inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    beg[lane] = inc - c;
+    if (lane == 31) beg[MROWS] = inc;
   }
   __syncthreads();
   const int total = beg[MROWS];
@@ -108,12 +124,15 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       const int t = e_tgt[d.ent0 + e];
       if (t >= tp_lo && t < tp_hi) {
         const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
-        tsrc[slot] = S_idx[d.src0 + e / L];
+        const int si = S_idx[d.src0 + e / L];
+        tsrc[slot] = si;
         tw[slot] = e_w[d.ent0 + e];
+        const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)si * D);
+        for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
       }
     }
     __syncthreads();
-    // order every list by token index (rank of each entry inside its row)
+    // order every list by token index (rank of each entry inside its row); total weight per row
     for (int i = tid; i < total; i += 256) {
       int r = 0;
       while (i >= beg[r + 1]) ++r;
@@ -123,91 +142,82 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       lsrc[beg[r] + rank] = my;
       lw[beg[r] + rank] = tw[i];
     }
+    __syncthreads();
+    if (tid < MROWS) {
+      float t = 0.f;
+      for (int k = beg[tid]; k < beg[tid + 1]; ++k) t += lw[k];
+      wsum_s[tid] = t;
+    }
   }
   __syncthreads();
 
-  // ---- light rows: one warp per row -----------------------------------------------------------
-  {
-    const int r = warp;
-    if (r < w.nrows) {
-      const int orow = w.r0 + r;
-      T* dst = out + (size_t)(d.out_row0 + orow) * D;
-      int srow, n = 0, li = 0;
-      if (orow < d.n_cls) {
-        srow = orow;
-      } else if (orow < d.n_cls + d.n_tgt) {
-        const int tp = orow - d.n_cls;
-        srow = d.n_cls + T_idx[d.tgt0 + tp];
-        li = tp - tp_lo;
-        n = cnt[li];
-      } else {
-        srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
+  // ---- light rows: four per warp ----------------------------------------------------------------
+  for (int r = warp; r < w.nrows; r += 8) {
+    const int orow = w.r0 + r;
+    T* dst = out + (size_t)(d.out_row0 + orow) * D;
+    const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+    const int li = is_tgt ? orow - d.n_cls - tp_lo : 0;
+    const int n = is_tgt ? cnt[li] : 0;
+    const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
+    if (n == 0) {
+      for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(dst)[v] = ldg16(src + (size_t)v * E);
+    } else if (fits && n <= MHEAVY) {
+      const int b0 = beg[li];
+      const float den = 1.0f + wsum_s[li];
+      for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
+        float acc[MVB][E];
+#pragma unroll
+        for (int b = 0; b < MVB; ++b) {
+          const int v = v0 + 32 * b;
+          unpack(v < nvec ? ldg16(src + (size_t)v * E) : make_uint4(0, 0, 0, 0), acc[b], (const T*)nullptr);
+        }
+        merge_accumulate<T>(acc, pbase, D, lsrc, lw, b0, b0 + n, v0, nvec);
+#pragma unroll
+        for (int b = 0; b < MVB; ++b) {
+          const int v = v0 + 32 * b;
+          if (v < nvec) {
+#pragma unroll
+            for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] / den;
+            reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
+          }
+        }
       }
-      const T* src = tokens + (size_t)(d.row0 + srow) * D;
-      if (n == 0) {
-        for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(dst)[v] = ldg16(src + (size_t)v * E);
-      } else if (fits && n <= MHEAVY) {
-        const int b0 = beg[li];
-        float wsum = 0.f;
-        for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
-        const float den = 1.0f + wsum;
-        for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
-          float acc[MVB][E];
+    } else if (!fits) {
+      // too many sources for shared memory: walk the entries in order (ascending source)
+      const int tp = orow - d.n_cls;
+      float wsum = 0.f;
+      for (int e = 0; e < n_ent; ++e)
+        if (e_tgt[d.ent0 + e] == tp) wsum += e_w[d.ent0 + e];
+      const float den = 1.0f + wsum;
+      for (int v = lane; v < nvec; v += 32) {
+        float acc[E];
+        unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
+        for (int e = 0; e < n_ent; ++e) {
+          if (e_tgt[d.ent0 + e] != tp) continue;
+          const T* x0 = pbase + (size_t)S_idx[d.src0 + e / L] * D;
+          float f[E];
+          unpack(ldg16(x0 + (size_t)v * E), f, (const T*)nullptr);
+          const float a0 = e_w[d.ent0 + e];
 #pragma unroll
-          for (int b = 0; b < MVB; ++b) {
-            const int v = v0 + 32 * b;
-            if (v < nvec) unpack(ldg16(src + (size_t)v * E), acc[b], (const T*)nullptr);
-          }
-          merge_accumulate<T>(acc, pbase, D, lsrc, lw, b0, b0 + n, v0, nvec);
-#pragma unroll
-          for (int b = 0; b < MVB; ++b) {
-            const int v = v0 + 32 * b;
-            if (v < nvec) {
-#pragma unroll
-              for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] / den;
-              reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
-            }
-          }
+          for (int q = 0; q < E; ++q) acc[q] = fmaf(a0, f[q], acc[q]);
         }
-      } else if (!fits) {
-        // too many sources for shared memory: walk the entries in order (ascending source)
-        const int tp = orow - d.n_cls;
-        float wsum = 0.f;
-        for (int e = 0; e < n_ent; ++e)
-          if (e_tgt[d.ent0 + e] == tp) wsum += e_w[d.ent0 + e];
-        const float den = 1.0f + wsum;
-        for (int v = lane; v < nvec; v += 32) {
-          float acc[E];
-          unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
-          for (int e = 0; e < n_ent; ++e) {
-            if (e_tgt[d.ent0 + e] != tp) continue;
-            const T* x0 = pbase + (size_t)S_idx[d.src0 + e / L] * D;
-            float f[E];
-            unpack(ldg16(x0 + (size_t)v * E), f, (const T*)nullptr);
-            const float a0 = e_w[d.ent0 + e];
 #pragma unroll
-            for (int q = 0; q < E; ++q) acc[q] = fmaf(a0, f[q], acc[q]);
-          }
-#pragma unroll
-          for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
-          reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
-        }
+        for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
+        reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
       }
     }
   }
   if (!fits) return;
 
-  // ---- heavy rows: every warp sums a slice of the list, combined in warp order -----------------
+  // ---- hub rows: every warp sums a slice of the list, combined in a fixed order ---------------
   for (int li = 0; li < tp_hi - tp_lo; ++li) {
     const int n = cnt[li];
     if (n <= MHEAVY) continue;                       // uniform over the CTA
     const int tp = tp_lo + li;
     const int b0 = beg[li];
-    const T* src = tokens + (size_t)(d.row0 + d.n_cls + T_idx[d.tgt0 + tp]) * D;
+    const T* src = tokens + (size_t)(d.row0 + srow_s[tp + d.n_cls - w.r0]) * D;
     T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
-    float wsum = 0.f;
-    for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
-    const float den = 1.0f + wsum;
+    const float den = 1.0f + wsum_s[li];
     const int k0 = b0 + (int)((long long)n * warp / 8), k1 = b0 + (int)((long long)n * (warp + 1) / 8);
     for (int vs = 0; vs < nvec; vs += 32 * MVB) {
       float acc[MVB][E];
