@@ -6,7 +6,7 @@ namespace ficoco {
 
 constexpr int MROWS = 32;      // output rows per CTA (four per warp)
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
-constexpr int MHEAVY = 8;      // rows with more sources than this are shared by all warps
+constexpr int MHEAVY = 4;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
 __device__ __forceinline__ void prefetch_l1(const void* p) {
@@ -59,8 +59,8 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
 //      alpha), prefetching the source rows, and orders every list by token index so that the
 //      fp32 sums have one fixed order and no atomics touch floats;
 //   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
-//      rows with few sources by their own warp, hub rows by all 8 warps (consecutive slices of
-//      the list, partial sums combined in a fixed order through shared memory).
+//      rows with few sources by their own warp; hub rows are cut into blocks of 32 vectors that
+//      are dealt to the warps, every lane summing the sources of its vector in list order.
 // If the CTA's rows receive more than MLIST sources in total, a slow in-order rescan is used.
 template <class T>
 __global__ void __launch_bounds__(256) k_merge_scan(
@@ -74,7 +74,8 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   __shared__ float lw[MLIST];
   __shared__ int tsrc[MLIST];
   __shared__ float tw[MLIST];
-  __shared__ __align__(16) float part[4][32 * MVB][E];   // warps w and w + 4 share a row
+  __shared__ int heavy_rows[MROWS];
+  __shared__ int n_heavy;
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -87,6 +88,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
 
   if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; wsum_s[tid] = 0.f; }
+  if (tid == 0) n_heavy = 0;
   // input row of every output row (CLS / preserved token / trailing text row), prefetched
   for (int r = warp; r < w.nrows; r += 8) {
     const int orow = w.r0 + r;
@@ -147,6 +149,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       float t = 0.f;
       for (int k = beg[tid]; k < beg[tid + 1]; ++k) t += lw[k];
       wsum_s[tid] = t;
+      if (cnt[tid] > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = tid;
     }
   }
   __syncthreads();
@@ -209,52 +212,41 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   }
   if (!fits) return;
 
-  // ---- hub rows: every warp sums a slice of the list, combined in a fixed order ---------------
-  for (int li = 0; li < tp_hi - tp_lo; ++li) {
-    const int n = cnt[li];
-    if (n <= MHEAVY) continue;                       // uniform over the CTA
+  // ---- hub rows: (row, block of 32 vectors) items dealt to the warps; each lane sums all the
+  // sources of its one vector in list order, eight source rows in flight ---------------------
+  const int nh = n_heavy;
+  const int nblk = (nvec + 31) / 32;
+  for (int it = warp; it < nh * nblk; it += 8) {
+    const int li = heavy_rows[it / nblk];
+    const int v = (it % nblk) * 32 + lane;
+    if (v >= nvec) continue;
     const int tp = tp_lo + li;
-    const int b0 = beg[li];
+    const int b0 = beg[li], n = cnt[li];
     const T* src = tokens + (size_t)(d.row0 + srow_s[tp + d.n_cls - w.r0]) * D;
     T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
     const float den = 1.0f + wsum_s[li];
-    const int k0 = b0 + (int)((long long)n * warp / 8), k1 = b0 + (int)((long long)n * (warp + 1) / 8);
-    for (int vs = 0; vs < nvec; vs += 32 * MVB) {
-      float acc[MVB][E];
+    float acc[E];
+    unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
+    for (int k = 0; k < n; k += 8) {
+      uint4 u[8];
+      float a[8];
 #pragma unroll
-      for (int b = 0; b < MVB; ++b)
-#pragma unroll
-        for (int q = 0; q < E; ++q) acc[b][q] = 0.f;
-      merge_accumulate<T>(acc, pbase, D, lsrc, lw, k0, k1, vs + lane, nvec);
-      if (warp < 4) {
-#pragma unroll
-        for (int b = 0; b < MVB; ++b)
-#pragma unroll
-          for (int q = 0; q < E; ++q) part[warp][lane + 32 * b][q] = acc[b][q];
+      for (int j = 0; j < 8; ++j) {
+        const bool on = k + j < n;
+        a[j] = on ? lw[b0 + k + j] : 0.f;
+        u[j] = on ? ldg16(pbase + (size_t)lsrc[b0 + k + j] * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
       }
-      __syncthreads();
-      if (warp >= 4) {
 #pragma unroll
-        for (int b = 0; b < MVB; ++b)
+      for (int j = 0; j < 8; ++j) {
+        float f[E];
+        unpack(u[j], f, (const T*)nullptr);
 #pragma unroll
-          for (int q = 0; q < E; ++q) part[warp - 4][lane + 32 * b][q] += acc[b][q];
+        for (int q = 0; q < E; ++q) acc[q] = fmaf(a[j], f[q], acc[q]);
       }
-      __syncthreads();
-      if (tid < 32 * MVB) {
-        const int v = vs + tid;
-        if (v < nvec) {
-          float f[E];
-          unpack(ldg16(src + (size_t)v * E), f, (const T*)nullptr);
-          for (int ww = 0; ww < 4; ++ww)
-#pragma unroll
-            for (int q = 0; q < E; ++q) f[q] += part[ww][tid][q];
-#pragma unroll
-          for (int q = 0; q < E; ++q) f[q] = f[q] / den;
-          reinterpret_cast<uint4*>(dst)[v] = pack(f, (const T*)nullptr);
-        }
-      }
-      __syncthreads();
     }
+#pragma unroll
+    for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
+    reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
   }
 }
 
