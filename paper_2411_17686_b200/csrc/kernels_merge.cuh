@@ -69,7 +69,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out) {
   constexpr int E = VecTraits<T>::E;
   __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
-  __shared__ float wsum_s[MROWS];
   __shared__ int lsrc[MLIST];
   __shared__ float lw[MLIST];
   __shared__ int tsrc[MLIST];
@@ -87,7 +86,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   const int n_ent = d.n_src * L;
   const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
 
-  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; wsum_s[tid] = 0.f; }
+  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
   if (tid == 0) n_heavy = 0;
   // input row of every output row (CLS / preserved token / trailing text row), prefetched
   for (int r = warp; r < w.nrows; r += 8) {
@@ -100,11 +99,34 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     prefetch_row(tokens + (size_t)(d.row0 + srow) * D, row_bytes, lane);
   }
   __syncthreads();
-  if (tp_hi > tp_lo)
-    for (int e = tid; e < n_ent; e += 256) {
-      const int t = e_tgt[d.ent0 + e];
-      if (t >= tp_lo && t < tp_hi) atomicAdd(&cnt[t - tp_lo], 1);
+  // file the entries that hit this CTA's rows.  Up to 1024 entries per image every thread looks
+  // at no more than four, keeps its matches in registers and needs one pass; larger images
+  // take a counting pass and a filling pass.
+  const bool one_pass = n_ent <= 4 * 256;
+  int st_row[4], st_slot[4], st_src[4];
+  float st_w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) st_row[i] = -1;
+  if (tp_hi > tp_lo) {
+    if (one_pass) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int e = tid + 256 * i;
+        const int t = e < n_ent ? e_tgt[d.ent0 + e] : -1;
+        if (t >= tp_lo && t < tp_hi) {
+          st_row[i] = t - tp_lo;
+          st_slot[i] = atomicAdd(&cnt[t - tp_lo], 1);
+          st_src[i] = S_idx[d.src0 + e / L];
+          st_w[i] = e_w[d.ent0 + e];
+        }
+      }
+    } else {
+      for (int e = tid; e < n_ent; e += 256) {
+        const int t = e_tgt[d.ent0 + e];
+        if (t >= tp_lo && t < tp_hi) atomicAdd(&cnt[t - tp_lo], 1);
+      }
     }
+  }
   __syncthreads();
   if (warp == 0) {
     // exclusive scan of the 32 counts
@@ -117,24 +139,37 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     }
     beg[lane] = inc - c;
     if (lane == 31) beg[MROWS] = inc;
+    if (c > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = lane;
   }
   __syncthreads();
   const int total = beg[MROWS];
   const bool fits = total <= MLIST;
   if (fits && total > 0) {
-    for (int e = tid; e < n_ent; e += 256) {
-      const int t = e_tgt[d.ent0 + e];
-      if (t >= tp_lo && t < tp_hi) {
-        const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
-        const int si = S_idx[d.src0 + e / L];
-        tsrc[slot] = si;
-        tw[slot] = e_w[d.ent0 + e];
-        const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)si * D);
-        for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
+    if (one_pass) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (st_row[i] >= 0) {
+          const int slot = beg[st_row[i]] + st_slot[i];
+          tsrc[slot] = st_src[i];
+          tw[slot] = st_w[i];
+          const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)st_src[i] * D);
+          for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
+        }
+    } else {
+      for (int e = tid; e < n_ent; e += 256) {
+        const int t = e_tgt[d.ent0 + e];
+        if (t >= tp_lo && t < tp_hi) {
+          const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
+          const int si = S_idx[d.src0 + e / L];
+          tsrc[slot] = si;
+          tw[slot] = e_w[d.ent0 + e];
+          const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)si * D);
+          for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
+        }
       }
     }
     __syncthreads();
-    // order every list by token index (rank of each entry inside its row); total weight per row
+    // order every list by token index (rank of each entry inside its row)
     for (int i = tid; i < total; i += 256) {
       int r = 0;
       while (i >= beg[r + 1]) ++r;
@@ -144,17 +179,41 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       lsrc[beg[r] + rank] = my;
       lw[beg[r] + rank] = tw[i];
     }
-    __syncthreads();
-    if (tid < MROWS) {
-      float t = 0.f;
-      for (int k = beg[tid]; k < beg[tid + 1]; ++k) t += lw[k];
-      wsum_s[tid] = t;
-      if (cnt[tid] > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = tid;
-    }
   }
   __syncthreads();
 
-  // ---- light rows: four per warp ----------------------------------------------------------------
+  // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
+  for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
+    uint4 u[4][MVB];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = warp + 8 * j;
+      const int orow = w.r0 + r;
+      const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
+      const T* src = tokens + (size_t)(d.row0 + (r < w.nrows ? srow_s[r] : 0)) * D;
+#pragma unroll
+      for (int b = 0; b < MVB; ++b) {
+        const int v = v0 + 32 * b;
+        u[j][b] = (copy && v < nvec) ? ldg16(src + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = warp + 8 * j;
+      const int orow = w.r0 + r;
+      const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
+      T* dst = out + (size_t)(d.out_row0 + orow) * D;
+#pragma unroll
+      for (int b = 0; b < MVB; ++b) {
+        const int v = v0 + 32 * b;
+        if (copy && v < nvec) reinterpret_cast<uint4*>(dst)[v] = u[j][b];
+      }
+    }
+  }
+
+  // ---- rows with a few sources: one warp per row --------------------------------------------------
   for (int r = warp; r < w.nrows; r += 8) {
     const int orow = w.r0 + r;
     T* dst = out + (size_t)(d.out_row0 + orow) * D;
@@ -163,10 +222,12 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const int n = is_tgt ? cnt[li] : 0;
     const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
     if (n == 0) {
-      for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(dst)[v] = ldg16(src + (size_t)v * E);
+      continue;
     } else if (fits && n <= MHEAVY) {
       const int b0 = beg[li];
-      const float den = 1.0f + wsum_s[li];
+      float wsum = 0.f;
+      for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
+      const float den = 1.0f + wsum;
       for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
         float acc[MVB][E];
 #pragma unroll
@@ -224,7 +285,9 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const int b0 = beg[li], n = cnt[li];
     const T* src = tokens + (size_t)(d.row0 + srow_s[tp + d.n_cls - w.r0]) * D;
     T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
-    const float den = 1.0f + wsum_s[li];
+    float wsum = 0.f;
+    for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
+    const float den = 1.0f + wsum;
     float acc[E];
     unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
     for (int k = 0; k < n; k += 8) {
