@@ -10,6 +10,7 @@ constexpr int CBM = 64;   // source rows per CTA
 constexpr int CBN = 64;   // target columns per tile
 constexpr int CKC = 16;   // reduction chunk
 
+template <int LC>
 __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     part_val[o] = lv[r][k];
     part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
   }
-  correlate_tail(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
+  correlate_tail<KCAP>(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
@@ -206,6 +207,8 @@ namespace ficoco {
 // e_w (alpha), e_c (the L largest C, descending).
 // grid = (images, ceil(max N^S / 256)).
 // ---------------------------------------------------------------------------------------
+// LC: compile-time bound on the list length L of the image (lists live in registers).
+template <int LC>
 __device__ __forceinline__ void finalize_source(
     const ImgDesc& d, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
@@ -213,10 +216,10 @@ __device__ __forceinline__ void finalize_source(
   const int L = d.list_len;
   const size_t o = (size_t)(d.src0 + s);
   if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; return; }
-  float v[KCAP];
-  int ix[KCAP];
+  float v[LC];
+  int ix[LC];
 #pragma unroll
-  for (int k = 0; k < KCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+  for (int k = 0; k < LC; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
   const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
   const int ne = d.nsplit * L;
   for (int e = 0; e < ne; ++e) {
@@ -224,7 +227,7 @@ __device__ __forceinline__ void finalize_source(
     int ci = __ldcg(part_idx + pbase + e);
     if (ci < 0) continue;
 #pragma unroll
-    for (int k = 0; k < KCAP; ++k) {
+    for (int k = 0; k < LC; ++k) {
       if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
         const float tv = v[k]; const int ti = ix[k];
         v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
@@ -233,7 +236,7 @@ __device__ __forceinline__ void finalize_source(
   }
   float vl1 = 0.f, vl2 = 0.f;
 #pragma unroll
-  for (int k = 0; k < KCAP; ++k) {
+  for (int k = 0; k < LC; ++k) {
     if (k == L - 1) vl1 = v[k];
     if (k == L - 2) vl2 = v[k];
   }
@@ -242,7 +245,7 @@ __device__ __forceinline__ void finalize_source(
   float den = 0.f;
   bool open = true;
 #pragma unroll
-  for (int k = 0; k < KCAP; ++k) {
+  for (int k = 0; k < LC; ++k) {
     if (k < L && open) {
       if (ix[k] != INT_MAX && v[k] >= tau) { ++nj; den += fmaxf(v[k], 0.f); } else open = false;
     }
@@ -252,7 +255,7 @@ __device__ __forceinline__ void finalize_source(
   tau_out[o] = tau;
   const size_t eb = (size_t)d.ent0 + (size_t)s * L;
 #pragma unroll
-  for (int k = 0; k < KCAP; ++k) {
+  for (int k = 0; k < LC; ++k) {
     if (k < L) {
       e_tgt[eb + k] = k < nj ? ix[k] : -1;
       e_w[eb + k] = k < nj ? fmaxf(v[k], 0.f) / den : 0.f;
@@ -268,13 +271,14 @@ __global__ void __launch_bounds__(256) k_finalize_src(
   const ImgDesc d = desc[blockIdx.x];
   const int s = blockIdx.y * 256 + threadIdx.x;
   if (s >= d.n_src) return;
-  finalize_source(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
+  finalize_source<KCAP>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
 // Tail of a correlate CTA: once its partial lists are written it bumps the image's counter;
 // the CTA that completes the image (the last of d.corr_items) turns the partial lists of all of
 // the image's discarded tokens into tau_i, J_i and alpha_ij, and resets the counter.  Nobody
 // waits: there is no spinning.  Call from all threads of the CTA.
+template <int LC>
 __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
@@ -290,7 +294,7 @@ __device__ __forceinline__ void correlate_tail(
   __syncthreads();
   if (*is_last_smem)
     for (int s = threadIdx.x; s < d.n_src; s += blockDim.x)
-      finalize_source(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
+      finalize_source<LC>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
 }  // namespace ficoco

@@ -53,6 +53,19 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                ::"r"(smem_u32(bar)) : "memory");
 }
+// 32 consecutive accumulator columns of this thread's TMEM lane; completes at tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -167,28 +180,36 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     float vmin = -CUDART_INF_F;                        // value of entry L-1
     int imin = INT_MAX;
     if (acc_ok) {
-      for (int c0 = 0; c0 < n_pad; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, r);
+      // 96 columns at a time: three 32-column TMEM loads are issued back to back and waited
+      // for once (columns past n_pad, rounded up to 32, lie inside the allocation)
+      for (int c0 = 0; c0 < n_pad; c0 += 96) {
+        uint32_t r[96];
+        const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
+        tmem_ld32_issue(t0, r);
+        if (c0 + 32 < n_pad) tmem_ld32_issue(t0 + 32, r + 32);
+        if (c0 + 64 < n_pad) tmem_ld32_issue(t0 + 64, r + 64);
+        tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
+        for (int j = 0; j < 96; ++j) {
           const int c = c0 + j;
-          const float val = (rs * rnT[c]) * __uint_as_float(r[j]);
-          const int idx = col_begin + c;
-          if (c < ncols && row_valid && toplist_better(val, idx, vmin, imin)) {
-            // insert into the descending list, dropping entry L-1
-            float cv = val;
-            int ci = idx;
+          if (c < ncols && row_valid) {
+            const float val = (rs * rnT[c]) * __uint_as_float(r[j]);
+            const int idx = col_begin + c;
+            if (toplist_better(val, idx, vmin, imin)) {
+              // insert into the descending list, dropping entry L-1
+              float cv = val;
+              int ci = idx;
 #pragma unroll
-            for (int k = 0; k < LCAP; ++k) {
-              if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
-                const float tv = v[k]; const int ti = ix[k];
-                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+              for (int k = 0; k < LCAP; ++k) {
+                if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
+                  const float tv = v[k]; const int ti = ix[k];
+                  v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+                }
               }
-            }
 #pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k == L - 1) { vmin = v[k]; imin = ix[k]; }
+              for (int k = 0; k < LCAP; ++k)
+                if (k == L - 1) { vmin = v[k]; imin = ix[k]; }
+            }
           }
         }
       }
@@ -240,7 +261,7 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                  : "memory");
   }
-  correlate_tail(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
+  correlate_tail<LCAP>(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
