@@ -222,15 +222,27 @@ __device__ __forceinline__ void finalize_source(
   for (int k = 0; k < LC; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
   const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
   const int ne = d.nsplit * L;
-  for (int e = 0; e < ne; ++e) {
-    float cv = __ldcg(part_val + pbase + e);
-    int ci = __ldcg(part_idx + pbase + e);
-    if (ci < 0) continue;
+  for (int e0 = 0; e0 < ne; e0 += 8) {
+    // eight entries of the partial lists in flight at a time
+    float pv[8];
+    int pi[8];
 #pragma unroll
-    for (int k = 0; k < LC; ++k) {
-      if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
-        const float tv = v[k]; const int ti = ix[k];
-        v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+    for (int j = 0; j < 8; ++j) {
+      const bool on = e0 + j < ne;
+      pv[j] = on ? __ldcg(part_val + pbase + e0 + j) : 0.f;
+      pi[j] = on ? __ldcg(part_idx + pbase + e0 + j) : -1;
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      float cv = pv[j];
+      int ci = pi[j];
+      if (ci < 0) continue;
+#pragma unroll
+      for (int k = 0; k < LC; ++k) {
+        if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
+          const float tv = v[k]; const int ti = ix[k];
+          v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+        }
       }
     }
   }

@@ -173,12 +173,14 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
     const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    float v[LCAP];
-    int ix[LCAP];
+    // Two independent descending lists (even / odd columns) give the single warp per scheduler
+    // two dependency chains to interleave.  Columns arrive in ascending order, so a value equal
+    // to one already listed never displaces it: plain '>' keeps the lower index first.
+    float v[LCAP], v2[LCAP];
+    int ix[LCAP], ix2[LCAP];
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-    float vmin = -CUDART_INF_F;                        // value of entry L-1
-    int imin = INT_MAX;
+    for (int k = 0; k < LCAP; ++k) { v[k] = v2[k] = -CUDART_INF_F; ix[k] = ix2[k] = INT_MAX; }
+    float vmin = -CUDART_INF_F, vmin2 = -CUDART_INF_F;   // value of entry L-1 of each list
     if (acc_ok) {
       // 96 columns at a time: three 32-column TMEM loads are issued back to back and waited
       // for once (columns past n_pad, rounded up to 32, lie inside the allocation)
@@ -190,27 +192,56 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
         if (c0 + 64 < n_pad) tmem_ld32_issue(t0 + 64, r + 64);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 96; ++j) {
+        for (int j = 0; j < 96; j += 2) {
           const int c = c0 + j;
-          if (c < ncols && row_valid) {
-            const float val = (rs * rnT[c]) * __uint_as_float(r[j]);
-            const int idx = col_begin + c;
-            if (toplist_better(val, idx, vmin, imin)) {
-              // insert into the descending list, dropping entry L-1
-              float cv = val;
-              int ci = idx;
+          const float va = (c < ncols && row_valid) ? (rs * rnT[c]) * __uint_as_float(r[j]) : -CUDART_INF_F;
+          const float vb = (c + 1 < ncols && row_valid) ? (rs * rnT[c + 1]) * __uint_as_float(r[j + 1]) : -CUDART_INF_F;
+          if (va > vmin) {
+            float cv = va;
+            int ci = col_begin + c;
+            bool shift = false;                  // once placed, the rest of the list moves down
 #pragma unroll
-              for (int k = 0; k < LCAP; ++k) {
-                if (k < L && toplist_better(cv, ci, v[k], ix[k])) {
-                  const float tv = v[k]; const int ti = ix[k];
-                  v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
-                }
+            for (int k = 0; k < LCAP; ++k)
+              if (k < L && (shift || cv > v[k])) {
+                const float tv = v[k]; const int ti = ix[k];
+                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+                shift = true;
               }
 #pragma unroll
-              for (int k = 0; k < LCAP; ++k)
-                if (k == L - 1) { vmin = v[k]; imin = ix[k]; }
-            }
+            for (int k = 0; k < LCAP; ++k)
+              if (k == L - 1) vmin = v[k];
           }
+          if (vb > vmin2) {
+            float cv = vb;
+            int ci = col_begin + c + 1;
+            bool shift = false;
+#pragma unroll
+            for (int k = 0; k < LCAP; ++k)
+              if (k < L && (shift || cv > v2[k])) {
+                const float tv = v2[k]; const int ti = ix2[k];
+                v2[k] = cv; ix2[k] = ci; cv = tv; ci = ti;
+                shift = true;
+              }
+#pragma unroll
+            for (int k = 0; k < LCAP; ++k)
+              if (k == L - 1) vmin2 = v2[k];
+          }
+        }
+      }
+      // fold the odd-column list into the even-column one (full tie-break on the index)
+#pragma unroll
+      for (int e = 0; e < LCAP; ++e) {
+        if (e < L && ix2[e] != INT_MAX) {
+          float cv = v2[e];
+          int ci = ix2[e];
+          bool shift = false;
+#pragma unroll
+          for (int k = 0; k < LCAP; ++k)
+            if (k < L && (shift || toplist_better(cv, ci, v[k], ix[k]))) {
+              const float tv = v[k]; const int ti = ix[k];
+              v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+              shift = true;
+            }
         }
       }
     }
