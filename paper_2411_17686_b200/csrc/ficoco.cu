@@ -94,6 +94,7 @@ struct ficoco_ctx {
   float* tau = nullptr;
   float* tmean = nullptr;
   unsigned* status = nullptr;
+  int* tile_cnt = nullptr;  // per source tile: column splits of the correlate kernel that are done
   int* img_cnt = nullptr;   // 2 * max_batch per-image piece counters of the fused filter kernel
   int num_sms = 0;
   bool coop_ok = false;
@@ -264,7 +265,8 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
-  const size_t o_icnt = carve(3 * B * 4);
+  const size_t o_icnt = carve(2 * B * 4);
+  const size_t o_tcnt = carve((size_t)c->cap_corr * 4);
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
@@ -288,6 +290,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->e_c = (float*)(b + o_c); c->tau = (float*)(b + o_tau);
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
   c->img_cnt = (int*)(b + o_icnt);
+  c->tile_cnt = (int*)(b + o_tcnt);
   c->plan_slots = b + o_pl;
 
   // kernels that may need more than 48 KB of dynamic shared memory
@@ -682,7 +685,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
   k_correlate_umma<NS, LC><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
       c->S_idx, c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes,        \
-      p->um_tmem_cols, c->img_cnt + 2 * c->max_batch, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c)
+      p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                                  \
@@ -698,7 +701,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       prof_tick(c, st, "correlate_simt");
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
                                                      c->T_idx, tmean, M, gamma, c->part_val, c->part_idx,
-                                                     c->img_cnt + 2 * c->max_batch, c->corr_cnt, c->tau,
+                                                     c->tile_cnt, c->corr_cnt, c->tau,
                                                      c->e_tgt, c->e_w, c->e_c);
     }
     c->launches += 1;
@@ -824,7 +827,8 @@ extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_statu
   CUDA_TRY(c, cudaStreamSynchronize(st));
   if (v & STATUS_TIMEOUT) {
     // a kernel gave up half-way: its per-image counters may be left non-zero
-    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 3 * (size_t)c->max_batch * sizeof(int), st));
+    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 2 * (size_t)c->max_batch * sizeof(int), st));
+    CUDA_TRY(c, cudaMemsetAsync(c->tile_cnt, 0, (size_t)c->cap_corr * sizeof(int), st));
     CUDA_TRY(c, cudaStreamSynchronize(st));
   }
   *device_status = (int)v;

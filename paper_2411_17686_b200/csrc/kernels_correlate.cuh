@@ -12,7 +12,8 @@ constexpr int CKC = 16;   // reduction chunk
 
 template <int LC>
 __device__ __forceinline__ void correlate_tail(
-    const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
+    const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
+    const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
     int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem);
 
@@ -192,7 +193,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     part_val[o] = lv[r][k];
     part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
   }
-  correlate_tail<KCAP>(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
+  correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
@@ -286,26 +287,28 @@ __global__ void __launch_bounds__(256) k_finalize_src(
   finalize_source<KCAP>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
-// Tail of a correlate CTA: once its partial lists are written it bumps the image's counter;
-// the CTA that completes the image (the last of d.corr_items) turns the partial lists of all of
-// the image's discarded tokens into tau_i, J_i and alpha_ij, and resets the counter.  Nobody
-// waits: there is no spinning.  Call from all threads of the CTA.
+// Tail of a correlate CTA: once its partial lists are written it bumps the counter of its
+// source tile (`tile` = index of the tile's first work item); the CTA that completes the tile
+// (the last of its d.nsplit column splits) turns the partial lists of the tile's discarded
+// tokens into tau_i, J_i and alpha_ij, and resets the counter.  Nobody waits: there is no
+// spinning.  Call from all threads of the CTA.
 template <int LC>
 __device__ __forceinline__ void correlate_tail(
-    const ImgDesc& d, int img, int* __restrict__ img_done, const float* __restrict__ part_val,
+    const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
+    const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
     int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem) {
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int old = atomicAdd(&img_done[img], 1);
-    const int last = old == d.corr_items - 1;
-    if (last) { __threadfence(); img_done[img] = 0; }
+    const int old = atomicAdd(&tile_done[tile], 1);
+    const int last = old == d.nsplit - 1;
+    if (last) { __threadfence(); tile_done[tile] = 0; }
     *is_last_smem = last;
   }
   __syncthreads();
   if (*is_last_smem)
-    for (int s = threadIdx.x; s < d.n_src; s += blockDim.x)
+    for (int s = w.r0 + (int)threadIdx.x; s < w.r0 + w.nrows; s += blockDim.x)
       finalize_source<LC>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 

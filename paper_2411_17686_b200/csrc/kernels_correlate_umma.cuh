@@ -173,14 +173,14 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
     const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    // Two independent descending lists (even / odd columns) give the single warp per scheduler
-    // two dependency chains to interleave.  Columns arrive in ascending order, so a value equal
-    // to one already listed never displaces it: plain '>' keeps the lower index first.
-    float v[LCAP], v2[LCAP];
-    int ix[LCAP], ix2[LCAP];
+    // Branch-free top-L: every entry is a 64-bit key (order-preserving value bits, then the
+    // complemented column index), so "larger key" means larger value and, on equal values, the
+    // lower index.  Inserting is a chain of max/min down the list.  Two lists (even / odd
+    // columns) give the single warp per scheduler two independent chains; they are folded at
+    // the end.  Key 0 marks an empty slot.
+    unsigned long long m[LCAP], m2[LCAP];
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { v[k] = v2[k] = -CUDART_INF_F; ix[k] = ix2[k] = INT_MAX; }
-    float vmin = -CUDART_INF_F, vmin2 = -CUDART_INF_F;   // value of entry L-1 of each list
+    for (int k = 0; k < LCAP; ++k) { m[k] = 0ull; m2[k] = 0ull; }
     if (acc_ok) {
       // 96 columns at a time: three 32-column TMEM loads are issued back to back and waited
       // for once (columns past n_pad, rounded up to 32, lie inside the allocation)
@@ -194,56 +194,46 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
 #pragma unroll
         for (int j = 0; j < 96; j += 2) {
           const int c = c0 + j;
-          const float va = (c < ncols && row_valid) ? (rs * rnT[c]) * __uint_as_float(r[j]) : -CUDART_INF_F;
-          const float vb = (c + 1 < ncols && row_valid) ? (rs * rnT[c + 1]) * __uint_as_float(r[j + 1]) : -CUDART_INF_F;
-          if (va > vmin) {
-            float cv = va;
-            int ci = col_begin + c;
-            bool shift = false;                  // once placed, the rest of the list moves down
+          const float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
+          const float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
+          unsigned long long ka = ((unsigned long long)order_key(va) << 32) | (0xFFFFFFFFu - (uint32_t)(col_begin + c));
+          unsigned long long kb = ((unsigned long long)order_key(vb) << 32) | (0xFFFFFFFFu - (uint32_t)(col_begin + c + 1));
+          if (!(c < ncols && row_valid) || va != va) ka = 0ull;
+          if (!(c + 1 < ncols && row_valid) || vb != vb) kb = 0ull;
 #pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k < L && (shift || cv > v[k])) {
-                const float tv = v[k]; const int ti = ix[k];
-                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
-                shift = true;
-              }
-#pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k == L - 1) vmin = v[k];
-          }
-          if (vb > vmin2) {
-            float cv = vb;
-            int ci = col_begin + c + 1;
-            bool shift = false;
-#pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k < L && (shift || cv > v2[k])) {
-                const float tv = v2[k]; const int ti = ix2[k];
-                v2[k] = cv; ix2[k] = ci; cv = tv; ci = ti;
-                shift = true;
-              }
-#pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k == L - 1) vmin2 = v2[k];
+          for (int k = 0; k < LCAP; ++k) {
+            if (k < L) {
+              const unsigned long long hi = m[k] > ka ? m[k] : ka;
+              ka = m[k] > ka ? ka : m[k];
+              m[k] = hi;
+              const unsigned long long hi2 = m2[k] > kb ? m2[k] : kb;
+              kb = m2[k] > kb ? kb : m2[k];
+              m2[k] = hi2;
+            }
           }
         }
       }
-      // fold the odd-column list into the even-column one (full tie-break on the index)
 #pragma unroll
       for (int e = 0; e < LCAP; ++e) {
-        if (e < L && ix2[e] != INT_MAX) {
-          float cv = v2[e];
-          int ci = ix2[e];
-          bool shift = false;
+        unsigned long long ke = e < L ? m2[e] : 0ull;
 #pragma unroll
-          for (int k = 0; k < LCAP; ++k)
-            if (k < L && (shift || toplist_better(cv, ci, v[k], ix[k]))) {
-              const float tv = v[k]; const int ti = ix[k];
-              v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
-              shift = true;
-            }
+        for (int k = 0; k < LCAP; ++k) {
+          if (k < L) {
+            const unsigned long long hi = m[k] > ke ? m[k] : ke;
+            ke = m[k] > ke ? ke : m[k];
+            m[k] = hi;
+          }
         }
       }
+    }
+    float v[LCAP];
+    int ix[LCAP];
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k) {
+      const uint32_t kv = (uint32_t)(m[k] >> 32);
+      const uint32_t u = (kv & 0x80000000u) ? (kv & 0x7FFFFFFFu) : ~kv;
+      v[k] = m[k] ? __uint_as_float(u) : -CUDART_INF_F;
+      ix[k] = m[k] ? (int)(0xFFFFFFFFu - (uint32_t)m[k]) : INT_MAX;
     }
     if (row_valid) {
       const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
@@ -292,7 +282,8 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                  : "memory");
   }
-  correlate_tail<LCAP>(d, w.img, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
+  correlate_tail<LCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c,
+                       &is_last);
 }
 
 }  // namespace ficoco
