@@ -173,17 +173,18 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
     const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    // Branch-free top-L: every entry is a 64-bit key (order-preserving value bits, then the
-    // complemented column index), so "larger key" means larger value and, on equal values, the
-    // lower index.  Inserting is a chain of max/min down the list.  Two lists (even / odd
-    // columns) give the single warp per scheduler two independent chains; they are folded at
-    // the end.  Key 0 marks an empty slot.
-    unsigned long long m[LCAP], m2[LCAP];
+    // Branch-free top-L in two sweeps over the row's columns, which stay in registers:
+    //   1. the L largest values: a max/min chain down two lists (even / odd columns), so that
+    //      the single warp per scheduler has two independent chains to interleave;
+    //   2. their columns: walking the columns in ascending order, each listed value takes the
+    //      first column not yet taken that holds it (equal values: lower index first).
+    float v[LCAP], v2[LCAP];
+    int ix[LCAP];
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { m[k] = 0ull; m2[k] = 0ull; }
+    for (int k = 0; k < LCAP; ++k) { v[k] = v2[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
     if (acc_ok) {
-      // 96 columns at a time: three 32-column TMEM loads are issued back to back and waited
-      // for once (columns past n_pad, rounded up to 32, lie inside the allocation)
+      // up to 96 columns at a time: three 32-column TMEM loads are issued back to back and
+      // waited for once (columns past n_pad, rounded up to 32, lie inside the allocation)
       for (int c0 = 0; c0 < n_pad; c0 += 96) {
         uint32_t r[96];
         const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
@@ -191,49 +192,68 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
         if (c0 + 32 < n_pad) tmem_ld32_issue(t0 + 32, r + 32);
         if (c0 + 64 < n_pad) tmem_ld32_issue(t0 + 64, r + 64);
         tmem_ld_wait();
+        float nv[LCAP];                      // the L largest values of this chunk merged with v
+#pragma unroll
+        for (int k = 0; k < LCAP; ++k) { nv[k] = v[k]; v2[k] = -CUDART_INF_F; }
 #pragma unroll
         for (int j = 0; j < 96; j += 2) {
           const int c = c0 + j;
-          const float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
-          const float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
-          unsigned long long ka = ((unsigned long long)order_key(va) << 32) | (0xFFFFFFFFu - (uint32_t)(col_begin + c));
-          unsigned long long kb = ((unsigned long long)order_key(vb) << 32) | (0xFFFFFFFFu - (uint32_t)(col_begin + c + 1));
-          if (!(c < ncols && row_valid) || va != va) ka = 0ull;
-          if (!(c + 1 < ncols && row_valid) || vb != vb) kb = 0ull;
+          float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
+          float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
+          if (!(c < ncols && row_valid) || va != va) va = -CUDART_INF_F;
+          if (!(c + 1 < ncols && row_valid) || vb != vb) vb = -CUDART_INF_F;
+          r[j] = __float_as_uint(va);
+          r[j + 1] = __float_as_uint(vb);
 #pragma unroll
-          for (int k = 0; k < LCAP; ++k) {
+          for (int k = 0; k < LCAP; ++k)
             if (k < L) {
-              const unsigned long long hi = m[k] > ka ? m[k] : ka;
-              ka = m[k] > ka ? ka : m[k];
-              m[k] = hi;
-              const unsigned long long hi2 = m2[k] > kb ? m2[k] : kb;
-              kb = m2[k] > kb ? kb : m2[k];
-              m2[k] = hi2;
+              const float hi = fmaxf(nv[k], va);
+              va = fminf(nv[k], va);
+              nv[k] = hi;
+              const float hi2 = fmaxf(v2[k], vb);
+              vb = fminf(v2[k], vb);
+              v2[k] = hi2;
             }
-          }
         }
-      }
 #pragma unroll
-      for (int e = 0; e < LCAP; ++e) {
-        unsigned long long ke = e < L ? m2[e] : 0ull;
+        for (int e = 0; e < LCAP; ++e) {     // fold the odd-column list in
+          float t = e < L ? v2[e] : -CUDART_INF_F;
 #pragma unroll
-        for (int k = 0; k < LCAP; ++k) {
-          if (k < L) {
-            const unsigned long long hi = m[k] > ke ? m[k] : ke;
-            ke = m[k] > ke ? ke : m[k];
-            m[k] = hi;
-          }
+          for (int k = 0; k < LCAP; ++k)
+            if (k < L) {
+              const float hi = fmaxf(nv[k], t);
+              t = fminf(nv[k], t);
+              nv[k] = hi;
+            }
         }
-      }
-    }
-    float v[LCAP];
-    int ix[LCAP];
+        // entries that survive from earlier chunks keep their columns (they are lower);
+        // positions taken by this chunk's values are recovered below
+        int nix[LCAP];
+        bool old_used[LCAP];
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) {
-      const uint32_t kv = (uint32_t)(m[k] >> 32);
-      const uint32_t u = (kv & 0x80000000u) ? (kv & 0x7FFFFFFFu) : ~kv;
-      v[k] = m[k] ? __uint_as_float(u) : -CUDART_INF_F;
-      ix[k] = m[k] ? (int)(0xFFFFFFFFu - (uint32_t)m[k]) : INT_MAX;
+        for (int k = 0; k < LCAP; ++k) { nix[k] = INT_MAX; old_used[k] = false; }
+#pragma unroll
+        for (int k = 0; k < LCAP; ++k)       // previous list first: lower columns win ties
+#pragma unroll
+          for (int q = 0; q < LCAP; ++q)
+            if (k < L && q < L && nix[k] == INT_MAX && !old_used[q] && ix[q] != INT_MAX && v[q] == nv[k]) {
+              nix[k] = ix[q];
+              old_used[q] = true;
+            }
+#pragma unroll
+        for (int j = 0; j < 96; ++j) {
+          const float val = __uint_as_float(r[j]);
+          bool used = val == -CUDART_INF_F;
+#pragma unroll
+          for (int k = 0; k < LCAP; ++k)
+            if (k < L && !used && nix[k] == INT_MAX && val == nv[k]) {
+              nix[k] = col_begin + c0 + j;
+              used = true;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < LCAP; ++k) { v[k] = nv[k]; ix[k] = nv[k] == -CUDART_INF_F ? INT_MAX : nix[k]; }
+      }
     }
     if (row_valid) {
       const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
