@@ -541,6 +541,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       if ((size_t)ns * p->um_stage_bytes + slack <= 220 * 1024) p->um_nstage = ns;
     if (!p->um_nstage) return FICOCO_ERR_UNSUPPORTED;
     p->um_smem = (size_t)p->um_nstage * p->um_stage_bytes + slack;
+    // the epilogue helpers hand their lists back through the ring
+    if (p->um_smem < 1024 + (size_t)UM * KCAP * 8) p->um_smem = 1024 + (size_t)UM * KCAP * 8;
   }
 
   char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
@@ -683,7 +685,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
-  k_correlate_umma<NS, LC><<<p->n_corr, 160, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
+  k_correlate_umma<NS, LC><<<p->n_corr, UTHREADS, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
       c->S_idx, c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes,        \
       p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \

@@ -24,6 +24,7 @@ namespace ficoco {
 constexpr int UM = 128;          // accumulator rows per CTA
 constexpr int UN_MAX = 256;      // accumulator columns per CTA
 constexpr int UKB = 64;          // bf16 elements per k-block (one 128-byte swizzle row)
+constexpr int UTHREADS = 288;    // warps 0-3 gather + epilogue, warp 4 MMA, warps 5-8 epilogue helpers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -76,12 +77,108 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 consecutive accumulator columns of this thread's TMEM lane; completes at tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+
+// Top-L of one accumulator row over the columns [c_lo, c_hi) (multiples of 16), branch-free, in
+// two sweeps over batches of up to 64 columns that stay in registers:
+//   1. the L largest values: a max/min chain down two lists (even / odd columns), so that a
+//      warp has two independent chains to interleave;
+//   2. their columns: walking the columns in ascending order, each listed value takes the
+//      first column not yet taken that holds it (equal values: lower index first).
+// v / ix: descending list, -inf / INT_MAX in empty slots.  Warp-collective (tcgen05.ld).
+template <int LCAP>
+__device__ __forceinline__ void epilogue_scan(uint32_t tmem_lane, int c_lo, int c_hi, int ncols, int col_begin,
+                                              float rs, const float* rnT, bool row_valid, int L,
+                                              float (&v)[LCAP], int (&ix)[LCAP]) {
+  float v2[LCAP];
+#pragma unroll
+  for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+  for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
+    uint32_t r[64];
+    tmem_ld16_issue(tmem_lane + (uint32_t)c0, r);
+    if (c0 + 16 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 16), r + 16);
+    if (c0 + 32 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 32), r + 32);
+    if (c0 + 48 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 48), r + 48);
+    tmem_ld_wait();
+    const int cmax = min(ncols, c_hi);
+    float nv[LCAP];                      // the L largest values of this batch merged with v
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k) { nv[k] = v[k]; v2[k] = -CUDART_INF_F; }
+#pragma unroll
+    for (int j = 0; j < 64; j += 2) {
+      const int c = c0 + j;
+      float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
+      float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
+      if (!(c < cmax && row_valid) || va != va) va = -CUDART_INF_F;
+      if (!(c + 1 < cmax && row_valid) || vb != vb) vb = -CUDART_INF_F;
+      r[j] = __float_as_uint(va);
+      r[j + 1] = __float_as_uint(vb);
+#pragma unroll
+      for (int k = 0; k < LCAP; ++k)
+        if (k < L) {
+          const float hi = fmaxf(nv[k], va);
+          va = fminf(nv[k], va);
+          nv[k] = hi;
+          const float hi2 = fmaxf(v2[k], vb);
+          vb = fminf(v2[k], vb);
+          v2[k] = hi2;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < LCAP; ++e) {     // fold the odd-column list in
+      float t = e < L ? v2[e] : -CUDART_INF_F;
+#pragma unroll
+      for (int k = 0; k < LCAP; ++k)
+        if (k < L) {
+          const float hi = fmaxf(nv[k], t);
+          t = fminf(nv[k], t);
+          nv[k] = hi;
+        }
+    }
+    // entries that survive from earlier batches keep their columns (they are lower);
+    // positions taken by this batch's values are recovered below
+    int nix[LCAP];
+    bool old_used[LCAP];
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k) { nix[k] = INT_MAX; old_used[k] = false; }
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k)       // previous list first: lower columns win ties
+#pragma unroll
+      for (int q = 0; q < LCAP; ++q)
+        if (k < L && q < L && nix[k] == INT_MAX && !old_used[q] && ix[q] != INT_MAX && v[q] == nv[k]) {
+          nix[k] = ix[q];
+          old_used[q] = true;
+        }
+#pragma unroll
+    for (int j = 0; j < 64; ++j) {
+      const float val = __uint_as_float(r[j]);
+      bool used = val == -CUDART_INF_F;
+#pragma unroll
+      for (int k = 0; k < LCAP; ++k)
+        if (k < L && !used && nix[k] == INT_MAX && val == nv[k]) {
+          nix[k] = col_begin + c0 + j;
+          used = true;
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k) { v[k] = nv[k]; ix[k] = nv[k] == -CUDART_INF_F ? INT_MAX : nix[k]; }
+  }
+}
+
 // Dynamic shared memory: [1024-aligned] ring of NSTAGE stages, each an A tile (a_bytes: the
 // valid source rows rounded up to 8, x 128 B) followed by a B tile (column rows x 128 B).  The
 // MMA always reads 128 A rows; rows past a_bytes alias the B tile (or the slack the host adds
 // behind the ring) and only feed accumulator rows that are never read.
 template <int NSTAGE, int LCAP>
-__global__ void __launch_bounds__(160) k_correlate_umma(
+__global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     const __nv_bfloat16* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const float* __restrict__ rn,
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
@@ -113,7 +210,7 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < UM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
-  for (int c = tid; c < UN_MAX; c += 160) {
+  for (int c = tid; c < UN_MAX; c += UTHREADS) {
     const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
     rowT[c] = p;
     rnT[c] = p >= 0 ? rn[d.patch0 + p] : 0.f;
@@ -173,86 +270,38 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
     const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    // Branch-free top-L in two sweeps over the row's columns, which stay in registers:
-    //   1. the L largest values: a max/min chain down two lists (even / odd columns), so that
-    //      the single warp per scheduler has two independent chains to interleave;
-    //   2. their columns: walking the columns in ascending order, each listed value takes the
-    //      first column not yet taken that holds it (equal values: lower index first).
-    float v[LCAP], v2[LCAP];
+    // this warp scans the lower half of the columns, its helper warp (same TMEM lanes) the
+    // upper half; the helper's list comes back through the (now idle) operand ring
+    float v[LCAP];
     int ix[LCAP];
+    const int c_mid = ((n_pad / 16 + 1) / 2) * 16;
+    if (acc_ok) epilogue_scan<LCAP>(tmem_base + ((uint32_t)(warp * 32) << 16), 0, c_mid, ncols, col_begin, rs, rnT,
+                                    row_valid, L, v, ix);
+    else {
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { v[k] = v2[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-    if (acc_ok) {
-      // up to 96 columns at a time: three 32-column TMEM loads are issued back to back and
-      // waited for once (columns past n_pad, rounded up to 32, lie inside the allocation)
-      for (int c0 = 0; c0 < n_pad; c0 += 96) {
-        uint32_t r[96];
-        const uint32_t t0 = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
-        tmem_ld32_issue(t0, r);
-        if (c0 + 32 < n_pad) tmem_ld32_issue(t0 + 32, r + 32);
-        if (c0 + 64 < n_pad) tmem_ld32_issue(t0 + 64, r + 64);
-        tmem_ld_wait();
-        float nv[LCAP];                      // the L largest values of this chunk merged with v
+      for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    }
+    cta_sync(1, 256);                                  // helper lists are in shared memory
+    {
+      const float* hv = reinterpret_cast<const float*>(um_raw + (ring - smem_u32(um_raw)));
+      const int* hi = reinterpret_cast<const int*>(hv + UM * LCAP);
 #pragma unroll
-        for (int k = 0; k < LCAP; ++k) { nv[k] = v[k]; v2[k] = -CUDART_INF_F; }
+      for (int e = 0; e < LCAP; ++e) {
+        if (e < L) {
+          float cv = hv[row * LCAP + e];
+          int ci = hi[row * LCAP + e];
+          bool shift = ci == INT_MAX;                  // empty helper slot: nothing to insert
+          if (!shift) {
+            shift = false;
 #pragma unroll
-        for (int j = 0; j < 96; j += 2) {
-          const int c = c0 + j;
-          float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
-          float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
-          if (!(c < ncols && row_valid) || va != va) va = -CUDART_INF_F;
-          if (!(c + 1 < ncols && row_valid) || vb != vb) vb = -CUDART_INF_F;
-          r[j] = __float_as_uint(va);
-          r[j + 1] = __float_as_uint(vb);
-#pragma unroll
-          for (int k = 0; k < LCAP; ++k)
-            if (k < L) {
-              const float hi = fmaxf(nv[k], va);
-              va = fminf(nv[k], va);
-              nv[k] = hi;
-              const float hi2 = fmaxf(v2[k], vb);
-              vb = fminf(v2[k], vb);
-              v2[k] = hi2;
-            }
+            for (int k = 0; k < LCAP; ++k)
+              if (k < L && (shift || toplist_better(cv, ci, v[k], ix[k]))) {
+                const float tv = v[k]; const int ti = ix[k];
+                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+                shift = true;
+              }
+          }
         }
-#pragma unroll
-        for (int e = 0; e < LCAP; ++e) {     // fold the odd-column list in
-          float t = e < L ? v2[e] : -CUDART_INF_F;
-#pragma unroll
-          for (int k = 0; k < LCAP; ++k)
-            if (k < L) {
-              const float hi = fmaxf(nv[k], t);
-              t = fminf(nv[k], t);
-              nv[k] = hi;
-            }
-        }
-        // entries that survive from earlier chunks keep their columns (they are lower);
-        // positions taken by this chunk's values are recovered below
-        int nix[LCAP];
-        bool old_used[LCAP];
-#pragma unroll
-        for (int k = 0; k < LCAP; ++k) { nix[k] = INT_MAX; old_used[k] = false; }
-#pragma unroll
-        for (int k = 0; k < LCAP; ++k)       // previous list first: lower columns win ties
-#pragma unroll
-          for (int q = 0; q < LCAP; ++q)
-            if (k < L && q < L && nix[k] == INT_MAX && !old_used[q] && ix[q] != INT_MAX && v[q] == nv[k]) {
-              nix[k] = ix[q];
-              old_used[q] = true;
-            }
-#pragma unroll
-        for (int j = 0; j < 96; ++j) {
-          const float val = __uint_as_float(r[j]);
-          bool used = val == -CUDART_INF_F;
-#pragma unroll
-          for (int k = 0; k < LCAP; ++k)
-            if (k < L && !used && nix[k] == INT_MAX && val == nv[k]) {
-              nix[k] = col_begin + c0 + j;
-              used = true;
-            }
-        }
-#pragma unroll
-        for (int k = 0; k < LCAP; ++k) { v[k] = nv[k]; ix[k] = nv[k] == -CUDART_INF_F ? INT_MAX : nix[k]; }
       }
     }
     if (row_valid) {
@@ -264,6 +313,30 @@ __global__ void __launch_bounds__(160) k_correlate_umma(
           part_idx[o + k] = ix[k] == INT_MAX ? -1 : ix[k];
         }
     }
+  } else if (warp > 4) {
+    // ---------------- epilogue helpers: upper half of the columns --------------------------------
+    bool acc_ok = mbar_wait(&acc_bar, 0);
+    if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
+    tc_fence_after();
+    const int grp = warp & 3;                          // TMEM lanes this warp may read
+    const int row = grp * 32 + lane;
+    const bool row_valid = row < w.nrows;
+    const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
+    float v[LCAP];
+    int ix[LCAP];
+    const int c_mid = ((n_pad / 16 + 1) / 2) * 16;
+    if (acc_ok) epilogue_scan<LCAP>(tmem_base + ((uint32_t)(grp * 32) << 16), c_mid, n_pad, ncols, col_begin, rs,
+                                    rnT, row_valid, L, v, ix);
+    else {
+#pragma unroll
+      for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    }
+    float* hv = reinterpret_cast<float*>(um_raw + (ring - smem_u32(um_raw)));
+    int* hi = reinterpret_cast<int*>(hv + UM * LCAP);
+#pragma unroll
+    for (int k = 0; k < LCAP; ++k) { hv[row * LCAP + k] = v[k]; hi[row * LCAP + k] = ix[k]; }
+    cta_sync(1, 256);
   } else {
     // ---------------- MMA issuer (one lane) ---------------------------------------------------
     if (lane == 0) {
