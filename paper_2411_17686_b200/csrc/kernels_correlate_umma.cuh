@@ -266,6 +266,8 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     bool acc_ok = ok && mbar_wait(&acc_bar, 0);
     if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
+    __threadfence_block();
+    asm volatile("bar.arrive 2, 256;" ::: "memory");     // releases the helper warps
     tc_fence_after();
     const int row = tid;                               // TMEM lane == accumulator row
     const bool row_valid = row < w.nrows;
@@ -315,8 +317,10 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     }
   } else if (warp > 4) {
     // ---------------- epilogue helpers: upper half of the columns --------------------------------
-    bool acc_ok = mbar_wait(&acc_bar, 0);
-    if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+    // sleep on hardware barrier 2 until the gather warps have seen the accumulator complete
+    // (polling the mbarrier from here would take issue slots from the gather warps)
+    cta_sync(2, 256);
+    bool acc_ok = !failed;
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
     tc_fence_after();
     const int grp = warp & 3;                          // TMEM lanes this warp may read

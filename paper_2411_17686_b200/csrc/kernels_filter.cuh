@@ -210,11 +210,10 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
 // synchronise on hardware barrier `bar`.
 //   1. every alive token bids (score key, lower index wins ties) for its window with a
 //      64-bit shared-memory max; the winner's score is multiplied by `coef`;
-//   2. the N^S highest scores are found on order-preserving keys, ties going to the lower
-//      index: up to 1024 tokens by counting every key's rank, larger images by an
-//      8-bit-per-pass radix select;
-//   3. ballot prefixes (small images) or block scans turn the membership flags into ascending
-//      index lists S and T, the kept row indices and the surviving grid positions.
+//   2. an 8-bit-per-pass radix select over order-preserving keys finds the N^S-th largest
+//      score; ties at the threshold go to the lower index;
+//   3. a block scan turns the membership flags into ascending index lists S and T, the kept
+//      row indices and the surviving grid positions.
 // `work` is a shared-memory area of select_work_bytes(np, windows) bytes: the scores and grid
 // positions are read from global memory once and kept there with the keys and window bids.
 // ---------------------------------------------------------------------------------------
@@ -276,51 +275,6 @@ __device__ __forceinline__ void select_image(
     keys[i] = order_key(s);
   }
   cta_sync(bar, nthr);
-
-  // ---- small images: rank every key by counting, then place by ballot prefixes ------------------
-  if (np <= 1024) {
-    const int k = d.n_src;
-    int* selflag = reinterpret_cast<int*>(sc);          // the scores are not needed any more
-    for (int i = tid; i < np; i += nthr) {
-      const uint32_t key = keys[i];
-      int rank = 0;                                      // keys that precede key i in the order
-      for (int j = 0; j < np; ++j) {
-        const uint32_t kj = keys[j];
-        rank += (kj > key || (kj == key && j < i)) ? 1 : 0;
-      }
-      selflag[i] = rank < k ? 1 : 0;
-    }
-    cta_sync(bar, nthr);
-    const int lane = tid & 31;
-    for (int base = 0; base < np; base += nthr) {        // selected tokens per 32-token chunk
-      const int i = base + tid;
-      const unsigned mask = __ballot_sync(0xFFFFFFFFu, i < np && selflag[i]);
-      if (lane == 0 && i < np) sh.hist[i >> 5] = __popc(mask);
-    }
-    cta_sync(bar, nthr);
-    for (int base = 0; base < np; base += nthr) {
-      const int i = base + tid;
-      const bool valid = i < np;
-      const bool sel = valid && selflag[i];
-      const unsigned mask = __ballot_sync(0xFFFFFFFFu, sel);
-      if (valid) {
-        int sel_rank = __popc(mask & ((1u << lane) - 1u));
-        for (int c = 0; c < (i >> 5); ++c) sel_rank += sh.hist[c];
-        if (sel) {
-          S_idx[d.src0 + sel_rank] = i;
-        } else {
-          const int tp = i - sel_rank;
-          T_idx[d.tgt0 + tp] = i;
-          kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
-          if (pos_out) pos_out[d.tgt0 + tp] = pp[i];
-        }
-      }
-    }
-    for (int i = tid; i < d.n_cls; i += nthr) kept_idx[d.out_row0 + i] = i;
-    for (int i = tid; i < d.n_tail; i += nthr)
-      kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
-    return;
-  }
 
   // ---- radix select: key of the n_src-th largest ------------------------------------------
   const int k = d.n_src;
