@@ -87,89 +87,45 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
       : "r"(taddr) : "memory");
 }
 
-// Top-L of one accumulator row over the columns [c_lo, c_hi) (multiples of 16), branch-free, in
-// two sweeps over batches of up to 64 columns that stay in registers:
-//   1. the L largest values: a max/min chain down two lists (even / odd columns), so that a
-//      warp has two independent chains to interleave;
-//   2. their columns: walking the columns in ascending order, each listed value takes the
-//      first column not yet taken that holds it (equal values: lower index first).
+// Top-L of one accumulator row over the columns [c_lo, c_hi) (multiples of 16).  The code is
+// kept small on purpose (a rolled loop over 16-column TMEM loads): it runs once per CTA, so a
+// long unrolled body would be paid for in instruction-cache misses.  Insertion is branch-free:
+// once a value is placed the rest of the list shifts down; '>' keeps the lower column first
+// among equal values because columns arrive in ascending order.
 // v / ix: descending list, -inf / INT_MAX in empty slots.  Warp-collective (tcgen05.ld).
 template <int LCAP>
 __device__ __forceinline__ void epilogue_scan(uint32_t tmem_lane, int c_lo, int c_hi, int ncols, int col_begin,
                                               float rs, const float* rnT, bool row_valid, int L,
                                               float (&v)[LCAP], int (&ix)[LCAP]) {
-  float v2[LCAP];
 #pragma unroll
   for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-  for (int c0 = c_lo; c0 < c_hi; c0 += 64) {
-    uint32_t r[64];
+  const int cmax = row_valid ? min(ncols, c_hi) : 0;
+#pragma unroll 1
+  for (int c0 = c_lo; c0 < c_hi; c0 += 16) {
+    uint32_t r[16];
     tmem_ld16_issue(tmem_lane + (uint32_t)c0, r);
-    if (c0 + 16 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 16), r + 16);
-    if (c0 + 32 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 32), r + 32);
-    if (c0 + 48 < c_hi) tmem_ld16_issue(tmem_lane + (uint32_t)(c0 + 48), r + 48);
     tmem_ld_wait();
-    const int cmax = min(ncols, c_hi);
-    float nv[LCAP];                      // the L largest values of this batch merged with v
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { nv[k] = v[k]; v2[k] = -CUDART_INF_F; }
-#pragma unroll
-    for (int j = 0; j < 64; j += 2) {
+    for (int j = 0; j < 16; ++j) {
       const int c = c0 + j;
-      float va = (rs * rnT[min(c, UN_MAX - 1)]) * __uint_as_float(r[j]);
-      float vb = (rs * rnT[min(c + 1, UN_MAX - 1)]) * __uint_as_float(r[j + 1]);
-      if (!(c < cmax && row_valid) || va != va) va = -CUDART_INF_F;
-      if (!(c + 1 < cmax && row_valid) || vb != vb) vb = -CUDART_INF_F;
-      r[j] = __float_as_uint(va);
-      r[j + 1] = __float_as_uint(vb);
+      float cv = (rs * rnT[c]) * __uint_as_float(r[j]);
+      if (!(c < cmax)) cv = -CUDART_INF_F;           // also drops NaN-free padding columns
+      int ci = col_begin + c;
+      bool ins = false;
 #pragma unroll
-      for (int k = 0; k < LCAP; ++k)
+      for (int k = 0; k < LCAP; ++k) {
         if (k < L) {
-          const float hi = fmaxf(nv[k], va);
-          va = fminf(nv[k], va);
-          nv[k] = hi;
-          const float hi2 = fmaxf(v2[k], vb);
-          vb = fminf(v2[k], vb);
-          v2[k] = hi2;
+          const bool p = ins || cv > v[k];
+          const float tv = v[k];
+          const int ti = ix[k];
+          v[k] = p ? cv : tv;
+          ix[k] = p ? ci : ti;
+          cv = p ? tv : cv;
+          ci = p ? ti : ci;
+          ins = p;
         }
+      }
     }
-#pragma unroll
-    for (int e = 0; e < LCAP; ++e) {     // fold the odd-column list in
-      float t = e < L ? v2[e] : -CUDART_INF_F;
-#pragma unroll
-      for (int k = 0; k < LCAP; ++k)
-        if (k < L) {
-          const float hi = fmaxf(nv[k], t);
-          t = fminf(nv[k], t);
-          nv[k] = hi;
-        }
-    }
-    // entries that survive from earlier batches keep their columns (they are lower);
-    // positions taken by this batch's values are recovered below
-    int nix[LCAP];
-    bool old_used[LCAP];
-#pragma unroll
-    for (int k = 0; k < LCAP; ++k) { nix[k] = INT_MAX; old_used[k] = false; }
-#pragma unroll
-    for (int k = 0; k < LCAP; ++k)       // previous list first: lower columns win ties
-#pragma unroll
-      for (int q = 0; q < LCAP; ++q)
-        if (k < L && q < L && nix[k] == INT_MAX && !old_used[q] && ix[q] != INT_MAX && v[q] == nv[k]) {
-          nix[k] = ix[q];
-          old_used[q] = true;
-        }
-#pragma unroll
-    for (int j = 0; j < 64; ++j) {
-      const float val = __uint_as_float(r[j]);
-      bool used = val == -CUDART_INF_F;
-#pragma unroll
-      for (int k = 0; k < LCAP; ++k)
-        if (k < L && !used && nix[k] == INT_MAX && val == nv[k]) {
-          nix[k] = col_begin + c0 + j;
-          used = true;
-        }
-    }
-#pragma unroll
-    for (int k = 0; k < LCAP; ++k) { v[k] = nv[k]; ix[k] = nv[k] == -CUDART_INF_F ? INT_MAX : nix[k]; }
   }
 }
 
