@@ -223,6 +223,7 @@ __device__ __forceinline__ void finalize_source(
   for (int k = 0; k < LC; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
   const size_t pbase = (size_t)d.part0 + (size_t)s * d.nsplit * L;
   const int ne = d.nsplit * L;
+#pragma unroll 1
   for (int e0 = 0; e0 < ne; e0 += 8) {
     // eight entries of the partial lists in flight at a time
     float pv[8];

@@ -214,6 +214,8 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
 //      score; ties at the threshold go to the lower index;
 //   3. a block scan turns the membership flags into ascending index lists S and T, the kept
 //      row indices and the surviving grid positions.
+// The code runs once per image, so it is kept compact (rolled loops, not inlined): a long
+// unrolled body would be paid for in instruction-cache misses.
 // `work` is a shared-memory area of select_work_bytes(np, windows) bytes: the scores and grid
 // positions are read from global memory once and kept there with the keys and window bids.
 // ---------------------------------------------------------------------------------------
@@ -228,7 +230,7 @@ struct SelectShared {
   int remaining;
 };
 
-__device__ __forceinline__ void select_image(
+__device__ __noinline__ void select_image(
     const ImgDesc& d, const float* s_raw, const int* __restrict__ pos, int window, float coef,
     int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
     int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
@@ -242,7 +244,10 @@ __device__ __forceinline__ void select_image(
   const int nwr = (d.gh + window - 1) / window;
   const int nwin = penalty ? nwc * nwr : 0;
 
+  #pragma unroll 1
+
   for (int i = tid; i < nwin; i += nthr) win[i] = 0ull;
+  #pragma unroll 1
   for (int i = tid; i < np; i += nthr) {
     sc[i] = __ldcg(s_raw + d.patch0 + i);
     pp[i] = pos ? pos[d.patch0 + i] : i;
@@ -251,6 +256,7 @@ __device__ __forceinline__ void select_image(
 
   // ---- local penalty ------------------------------------------------------------------
   if (penalty) {
+    #pragma unroll 1
     for (int i = tid; i < np; i += nthr) {
       const int p = pp[i];
       if (p < 0 || p >= d.gh * d.gw) { atomicOr(status, STATUS_POS_RANGE); continue; }
@@ -261,6 +267,7 @@ __device__ __forceinline__ void select_image(
     }
     cta_sync(bar, nthr);
   }
+  #pragma unroll 1
   for (int i = tid; i < np; i += nthr) {
     float s = sc[i];
     if (penalty) {
@@ -283,11 +290,13 @@ __device__ __forceinline__ void select_image(
   if (k > 0 && k < np) {
     if (tid == 0) { sh.prefix = 0; sh.remaining = k; }
     uint32_t mask = 0;
+    #pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       if (tid < 256) sh.hist[tid] = 0;
       cta_sync(bar, nthr);
       const uint32_t prefix = sh.prefix;
+      #pragma unroll 1
       for (int i = tid; i < np; i += nthr) {
         const uint32_t key = keys[i];
         if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255], 1);
@@ -328,6 +337,7 @@ __device__ __forceinline__ void select_image(
 
   // ---- ordered compaction into S and T ------------------------------------------------------
   int eq_base = 0, sel_base = 0;
+  #pragma unroll 1
   for (int base = 0; base < np; base += nthr) {
     const int i = base + tid;
     const bool valid = i < np;
@@ -353,7 +363,9 @@ __device__ __forceinline__ void select_image(
       }
     }
   }
+  #pragma unroll 1
   for (int i = tid; i < d.n_cls; i += nthr) kept_idx[d.out_row0 + i] = i;
+  #pragma unroll 1
   for (int i = tid; i < d.n_tail; i += nthr)
     kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
 }

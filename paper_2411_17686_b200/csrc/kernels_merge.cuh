@@ -25,6 +25,7 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
                                                  const int* lsrc, const float* lw, int k0, int k1,
                                                  int v0, int nvec) {
   constexpr int E = VecTraits<T>::E;
+  #pragma unroll 1
   for (int k = k0; k < k1; k += 4) {
     uint4 u[4][MVB];
     float a[4];
@@ -89,6 +90,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
   if (tid == 0) n_heavy = 0;
   // input row of every output row (CLS / preserved token / trailing text row), prefetched
+  #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
     const int orow = w.r0 + r;
     int srow;
@@ -183,6 +185,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   __syncthreads();
 
   // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
+  #pragma unroll 1
   for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
     uint4 u[4][MVB];
 #pragma unroll
@@ -214,6 +217,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   }
 
   // ---- rows with a few sources: one warp per row --------------------------------------------------
+  #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
     const int orow = w.r0 + r;
     T* dst = out + (size_t)(d.out_row0 + orow) * D;
@@ -228,6 +232,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       float wsum = 0.f;
       for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
       const float den = 1.0f + wsum;
+      #pragma unroll 1
       for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
         float acc[MVB][E];
 #pragma unroll
@@ -277,6 +282,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   // sources of its one vector in list order, eight source rows in flight ---------------------
   const int nh = n_heavy;
   const int nblk = (nvec + 31) / 32;
+  #pragma unroll 1
   for (int it = warp; it < nh * nblk; it += 8) {
     const int li = heavy_rows[it / nblk];
     const int v = (it % nblk) * 32 + lane;
@@ -290,6 +296,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const float den = 1.0f + wsum;
     float acc[E];
     unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
+    #pragma unroll 1
     for (int k = 0; k < n; k += 8) {
       uint4 u[8];
       float a[8];
