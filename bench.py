@@ -103,11 +103,32 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def shard_seed(rank: int) -> int:
+    """Every rank reduces its own batch of B images (weak scaling): the generator seed differs
+    per rank, nothing is exchanged between ranks on the data path."""
+    return 2000 + rank
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Elapsed device time of the slowest rank (all_reduce MAX over the process group)."""
+    if world <= 1:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_images_per_s(ms_per_step: float, world: int) -> float:
+    """Whole-job throughput: all ranks' images per step over the slowest rank's step time."""
+    return world * B / (ms_per_step * 1e-3)
+
+
 def make_instances(rank: int):
     """One generated batch, laid out N_INSTANCES times with the image order rotated, so every
     step reads and writes memory that is not in L2 from the step before."""
     from paper_2411_17686_b200 import synth
-    batch = synth.make_v_batch(2000 + rank, B, GH, GW, D, H, KEEP, "bf16", True, 1.5, name="c2")
+    batch = synth.make_v_batch(shard_seed(rank), B, GH, GW, D, H, KEEP, "bf16", True, 1.5, name="c2")
     return batch
 
 
@@ -181,12 +202,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     barrier()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_per_step = ms / args.steps
-    value = world * B / (ms_per_step * 1e-3)
+    value = aggregate_images_per_s(ms_per_step, world)
 
     if rank != 0:
         return None
