@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       const int b0 = beg[li];
       float wsum = 0.f;
       for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
-      const float den = 1.0f + wsum;
+      const float inv_den = 1.0f / (1.0f + wsum);   // one division per row, then multiplies
       #pragma unroll 1
       for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
         float acc[MVB][E];
@@ -246,7 +246,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
           const int v = v0 + 32 * b;
           if (v < nvec) {
 #pragma unroll
-            for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] / den;
+            for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] * inv_den;
             reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
           }
         }
@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
     float wsum = 0.f;
     for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
-    const float den = 1.0f + wsum;
+    const float inv_den = 1.0f / (1.0f + wsum);
     float acc[E];
     unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
     #pragma unroll 1
@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       }
     }
 #pragma unroll
-    for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
+    for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
     reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
   }
 }
