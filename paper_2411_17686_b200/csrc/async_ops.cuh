@@ -39,6 +39,13 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
+// Programmatic dependent launch.  grid_dep_wait() returns once every grid this one depends on has
+// completed and its writes are visible (a no-op for a launch without the attribute);
+// grid_dep_launch() lets the next grid in the stream start its blocks early, which then park in
+// their own grid_dep_wait().
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Arrive on `bar` and announce `bytes` of bulk-copy traffic that will complete on it.

@@ -602,6 +602,25 @@ int get_plan(ficoco_ctx* c, const PlanKey& key, long long attn_rows, cudaStream_
   return FICOCO_OK;
 }
 
+// Launch with programmatic stream serialization: the grid may be staged while the kernel before
+// it in the stream is still running; the kernel itself waits (grid_dep_wait) before it reads
+// anything that kernel wrote.
+template <class... KArgs, class... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                             Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 template <class T, int VPL>
 cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn,
                                 int attn_rows, float cA, const int* pos, int window, float coef, int penalty,
@@ -685,9 +704,11 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
-  k_correlate_umma<NS, LC><<<p->n_corr, UTHREADS, p->um_smem, st>>>(tk, D, p->d_desc, p->d_corr, c->rn,       \
-      c->S_idx, c->T_idx, c->part_val, c->part_idx, c->status, p->um_stage_bytes, p->um_a_bytes,        \
-      p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c)
+  launch_dependent(k_correlate_umma<NS, LC>, p->n_corr, UTHREADS, p->um_smem, st, tk, D,               \
+      (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
+      (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
+      p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
+      c->e_w, c->e_c)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                                  \
@@ -715,8 +736,10 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     c->launches += 1;
   }
   prof_tick(c, st, "merge_compact");
-  k_merge_scan<T><<<p->n_out, 256, 0, st>>>(tok, D, p->d_desc, p->d_out, c->S_idx, c->T_idx, c->e_tgt,
-                                            c->e_w, out_tokens);
+  const int after_correlate = p->n_corr > 0 ? 1 : 0;   // else the grid before may be the filter itself
+  launch_dependent(k_merge_scan<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+                   (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
+                   (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate);
   c->launches += 1;
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);

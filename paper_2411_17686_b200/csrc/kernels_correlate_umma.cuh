@@ -165,16 +165,22 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     acc_committed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // Everything above touches only launch-constant plan data and this CTA's own resources, so it
+  // may run while the filter grid is still finishing; the index lists and norms it wrote are
+  // read below.  The dependent (merge) grid is released only after this wait, so by the time
+  // any of its blocks starts, the filter grid is complete as well.
+  grid_dep_wait();
+  grid_dep_launch();
   if (tid < UM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
   for (int c = tid; c < UN_MAX; c += UTHREADS) {
     const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
     rowT[c] = p;
     rnT[c] = p >= 0 ? rn[d.patch0 + p] : 0.f;
-  }
-  if (warp == 4) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();

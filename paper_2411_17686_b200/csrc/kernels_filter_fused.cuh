@@ -49,6 +49,9 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   extern __shared__ __align__(128) unsigned char fs_raw[];
   __shared__ uint64_t full_bar[F_MAXSTAGE], empty_bar[F_MAXSTAGE];
   __shared__ SelectShared sel_sh;
+  // All CTAs of this grid are co-resident, so the next grid may be staged right away: its blocks
+  // take over SMs as blocks of this grid exit and park until this grid has completed.
+  grid_dep_launch();
   __shared__ int won[F_MAXWON];
   __shared__ int nwon, failed;
 

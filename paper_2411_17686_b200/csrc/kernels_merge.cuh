@@ -67,7 +67,8 @@ template <class T>
 __global__ void __launch_bounds__(256) k_merge_scan(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
-    const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out) {
+    const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out,
+    int index_before_wait) {
   constexpr int E = VecTraits<T>::E;
   __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
   __shared__ int lsrc[MLIST];
@@ -89,6 +90,10 @@ __global__ void __launch_bounds__(256) k_merge_scan(
 
   if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
   if (tid == 0) n_heavy = 0;
+  // When the grid before this one is a correlate grid, the filter grid (which wrote T_idx) had
+  // completed before this grid could start, so the row lookup and prefetch may overlap that
+  // grid's tail; otherwise wait first.
+  if (!index_before_wait) grid_dep_wait();
   // input row of every output row (CLS / preserved token / trailing text row), prefetched
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
@@ -100,6 +105,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     if (lane == 0) srow_s[r] = srow;
     prefetch_row(tokens + (size_t)(d.row0 + srow) * D, row_bytes, lane);
   }
+  if (index_before_wait) grid_dep_wait();
   __syncthreads();
   // file the entries that hit this CTA's rows.  Up to 1024 entries per image every thread looks
   // at no more than four, keeps its matches in registers and needs one pass; larger images
