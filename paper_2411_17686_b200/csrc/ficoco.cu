@@ -6,6 +6,7 @@
 #include <string.h>
 
 #include <new>
+#include <mutex>
 #include <vector>
 
 #include "../../include/ficoco.h"
@@ -66,7 +67,72 @@ struct Plan {
   std::vector<ImgDesc> h_desc;
 };
 
+// ---- what the last step on a stream wrote ------------------------------------------------------
+// The filter grid of a step may start under the tail of the merge grid of the step launched
+// before it on the same stream.  That is only sound when the new step does not read what the
+// older one is still writing, so the output spans of the last step are remembered per
+// (device, stream), over all contexts of the process; a step whose inputs touch them, or whose
+// stream has no record, is launched fully serialized.
+struct Span {
+  const char* lo = nullptr;
+  const char* hi = nullptr;
+};
+inline Span span_of(const void* ptr, size_t bytes) {
+  Span s;
+  if (ptr != nullptr && bytes > 0) { s.lo = (const char*)ptr; s.hi = s.lo + bytes; }
+  return s;
+}
+inline bool spans_overlap(const Span& a, const Span& b) {
+  return a.lo != nullptr && b.lo != nullptr && a.lo < b.hi && b.lo < a.hi;
+}
+constexpr int N_TAILS = 16, N_SPANS = 4;
+struct StreamTail {
+  bool used = false;
+  int device = 0;
+  cudaStream_t st = nullptr;
+  Span out[N_SPANS];
+  unsigned long long stamp = 0;
+};
+std::mutex g_tail_mu;
+StreamTail g_tail[N_TAILS];
+unsigned long long g_tail_clock = 0;
+
+bool inputs_clear_of_last_outputs(int device, cudaStream_t st, const Span* in, int n_in) {
+  std::lock_guard<std::mutex> lk(g_tail_mu);
+  for (int i = 0; i < N_TAILS; ++i) {
+    const StreamTail& t = g_tail[i];
+    if (!t.used || t.device != device || t.st != st) continue;
+    for (int a = 0; a < n_in; ++a)
+      for (int b = 0; b < N_SPANS; ++b)
+        if (spans_overlap(in[a], t.out[b])) return false;
+    return true;
+  }
+  return false;
+}
+
+void record_last_outputs(int device, cudaStream_t st, const Span* out, int n_out) {
+  std::lock_guard<std::mutex> lk(g_tail_mu);
+  int slot = -1;
+  for (int i = 0; i < N_TAILS && slot < 0; ++i)
+    if (g_tail[i].used && g_tail[i].device == device && g_tail[i].st == st) slot = i;
+  if (slot < 0) {
+    slot = 0;
+    for (int i = 0; i < N_TAILS; ++i) {
+      if (!g_tail[i].used) { slot = i; break; }
+      if (g_tail[i].stamp < g_tail[slot].stamp) slot = i;
+    }
+  }
+  StreamTail& t = g_tail[slot];
+  t.used = true;
+  t.device = device;
+  t.st = st;
+  t.stamp = ++g_tail_clock;
+  for (int b = 0; b < N_SPANS; ++b) t.out[b] = b < n_out ? out[b] : Span();
+}
+
 }  // namespace
+
+__global__ void k_launch_probe() {}
 
 struct ficoco_ctx {
   int device = 0;
@@ -98,6 +164,7 @@ struct ficoco_ctx {
   int* img_cnt = nullptr;   // 2 * max_batch per-image piece counters of the fused filter kernel
   int num_sms = 0;
   bool coop_ok = false;
+  bool coop_pdl_ok = false;  // a cooperative grid may also be a programmatic dependent
   char* plan_slots = nullptr;
   size_t slot_bytes = 0;
   size_t off_rows = 0, off_corr = 0, off_out = 0, off_ctaf = 0;
@@ -250,6 +317,24 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
     v = 0;
     cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, device);
     c->coop_ok = v != 0;
+    // Does the runtime take a cooperative launch that also carries programmatic stream
+    // serialization?  One empty grid answers it; a refusal only turns the overlap off.
+    if (c->coop_ok) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(1);
+      cfg.blockDim = dim3(32);
+      cudaLaunchAttribute at[2];
+      at[0].id = cudaLaunchAttributeCooperative;
+      at[0].val.cooperative = 1;
+      at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      at[1].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = at;
+      cfg.numAttrs = 2;
+      const cudaError_t pe = cudaLaunchKernelEx(&cfg, k_launch_probe);
+      const cudaError_t se = cudaDeviceSynchronize();
+      c->coop_pdl_ok = pe == cudaSuccess && se == cudaSuccess;
+      if (!c->coop_pdl_ok) cudaGetLastError();
+    }
   }
   c->cap_rows = (int)(MAX_CHUNKS * B);
   if (c->cap_rows < c->num_sms + (int)B + 8) c->cap_rows = c->num_sms + (int)B + 8;
@@ -624,17 +709,20 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size
 template <class T, int VPL>
 cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn,
                                 int attn_rows, float cA, const int* pos, int window, float coef, int penalty,
-                                int* kept_idx, int* pos_out, float* scores_out, cudaStream_t st) {
+                                int* kept_idx, int* pos_out, float* scores_out, bool overlap_prev,
+                                cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p->f_grid);
   cfg.blockDim = dim3(F_THREADS);
   cfg.dynamicSmemBytes = p->f_smem;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeCooperative;
   at[0].val.cooperative = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = (c->coop_pdl_ok && overlap_prev) ? 2 : 1;
   return cudaLaunchKernelEx(&cfg, k_filter_fused<T, VPL>, tok, D, (const ImgDesc*)p->d_desc,
                             (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
@@ -659,11 +747,21 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
+  const size_t in_rows = (size_t)p->tot_patch + (size_t)p->key.batch * (p->key.has_cls + (p->key.mode == 1 ? p->key.n_text : 0));
+  const Span in_spans[3] = {span_of(tok, in_rows * D * sizeof(T)),
+                            span_of(attn, (size_t)attn_rows * p->tot_patch * sizeof(float)),
+                            span_of(pos, (size_t)p->tot_patch * sizeof(int))};
+  const Span out_spans[N_SPANS] = {span_of(out_tokens, (size_t)p->tot_out_rows * D * sizeof(T)),
+                                   span_of(kept_idx, (size_t)p->tot_out_rows * sizeof(int)),
+                                   span_of(pos_out, (size_t)p->tot_tgt * sizeof(int)),
+                                   span_of(scores_out, (size_t)p->tot_patch * sizeof(float))};
+  const bool overlap_prev = inputs_clear_of_last_outputs(c->device, st, in_spans, 3);
+  record_last_outputs(c->device, st, out_spans, N_SPANS);
   if (p->fused) {
     prof_tick(c, st, "filter_fused");
     cudaError_t fe;
 #define FICOCO_FUSED_GO(V) fe = launch_filter_fused<T, V>(c, p, tok, D, attn, attn_rows, cA, pos, window, coef, \
-                                                          penalty, kept_idx, pos_out, scores_out, st)
+                                                          penalty, kept_idx, pos_out, scores_out, overlap_prev, st)
     if (vpl <= 1) FICOCO_FUSED_GO(1);
     else if (vpl <= 2) FICOCO_FUSED_GO(2);
     else if (vpl <= 4) FICOCO_FUSED_GO(4);

@@ -277,6 +277,10 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
 
   // selections this CTA won (the ring is idle now and serves as work area)
   if (failed) return;
+  // Up to here the kernel wrote only scratch that no grid but a filter or correlate grid reads,
+  // and those of the step before were complete before this grid could start.  The index lists
+  // and outputs written below are read by the merge grid of the step before: wait for it.
+  grid_dep_wait();
   const int nw = nwon;
   for (int k = 0; k < nw; ++k) {
     const int img = won[k];

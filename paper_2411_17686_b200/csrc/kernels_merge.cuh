@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     prefetch_row(tokens + (size_t)(d.row0 + srow) * D, row_bytes, lane);
   }
   if (index_before_wait) grid_dep_wait();
+  grid_dep_launch();   // correlate is complete: the next step's filter may stream its rows under our tail
   __syncthreads();
   // file the entries that hit this CTA's rows.  Up to 1024 entries per image every thread looks
   // at no more than four, keeps its matches in registers and needs one pass; larger images

@@ -139,6 +139,40 @@ def test_run_to_run_determinism_and_host_entry_point(ctx):
     assert np.array_equal(binding.to_numpy(d.kept_idx), binding.to_numpy(hh.kept_idx))
 
 
+def test_back_to_back_steps_without_sync(ctx):
+    """Steps queued on one stream with no host synchronisation between them: a step fed
+    straight from the outputs of the step before it, and an independent step right behind
+    (whose first grid may start under the tail of the step before).  Every result must be
+    bit-identical to the same chain run with a device synchronisation after every call."""
+    nb, g, heads = 16, 24, 4
+    batch = synth.make_v_batch(91, nb, g, g, 512, heads, g * g // 2, "bf16", True, 1.5)
+    pk = packing.pack_v(batch, DEV)
+    prm = parity.params_to_abi(fo.Params(), True)
+    gen = torch.Generator().manual_seed(5)
+    k1, k2 = g * g // 2, g * g // 4
+    attn2 = torch.softmax(1.5 * torch.randn(nb, heads, k1, generator=gen), -1).reshape(-1).to(DEV)
+
+    def chain(sync):
+        r1 = ctx.ficoco_v_reduce(pk.tokens, pk.attn, k1, g, g, heads, params=prm, **pk.call_kwargs())
+        if sync:
+            torch.cuda.synchronize()
+        r2 = ctx.ficoco_v_reduce(r1.out_tokens, attn2, k2, g, g, heads, n_tokens=1 + k1, pos=r1.pos_out,
+                                 params=prm)
+        if sync:
+            torch.cuda.synchronize()
+        r3 = ctx.ficoco_v_reduce(pk.tokens, pk.attn, k1, g, g, heads, params=prm, **pk.call_kwargs())
+        torch.cuda.synchronize()
+        assert ctx.ficoco_status() == 0
+        return [binding.to_numpy(t) for r in (r1, r2, r3) for t in (r.out_tokens, r.kept_idx, r.pos_out)]
+
+    ref = chain(True)
+    assert np.array_equal(ref[0], ref[6]) and np.array_equal(ref[1], ref[7])
+    for rep in range(12):
+        got = chain(False)
+        for i, (a, b) in enumerate(zip(ref, got)):
+            assert np.array_equal(a, b), f"repetition {rep}: array {i} differs from the synchronised chain"
+
+
 def test_canaries_around_outputs(ctx):
     """Nothing is written outside the documented output extents."""
     batch = synth.workload(4, small=True)
