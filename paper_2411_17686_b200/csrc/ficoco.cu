@@ -29,6 +29,10 @@ constexpr int TARGET_CTAS = 2 * 148;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// host-buffer entry points: image groups pipelined over upload / kernels / download
+constexpr int HOST_MAX_GROUPS = 8;
+constexpr size_t HOST_GROUP_BYTES = 8u << 20;   // at least this many token bytes per group
+
 struct PlanKey {
   int mode;  // 0 = V, 1 = L
   int dtype, batch, dim, n_text, has_cls, max_targets;
@@ -187,6 +191,8 @@ struct ficoco_ctx {
   char* hs_dev = nullptr;
   size_t hs_dev_bytes = 0;
   cudaStream_t hs_stream = nullptr;
+  cudaStream_t hs_run = nullptr, hs_out = nullptr;   // kernels / downloads of the host entry points
+  cudaEvent_t hs_ev[2 * HOST_MAX_GROUPS] = {};
 };
 
 #define CUDA_TRY(ctx, expr)                                  \
@@ -416,6 +422,10 @@ extern "C" int ficoco_destroy(ficoco_ctx* c) {
   if (c->h_stage) cudaFreeHost(c->h_stage);
   if (c->hs_dev) cudaFree(c->hs_dev);
   if (c->hs_stream) cudaStreamDestroy(c->hs_stream);
+  if (c->hs_run) cudaStreamDestroy(c->hs_run);
+  if (c->hs_out) cudaStreamDestroy(c->hs_out);
+  for (int i = 0; i < 2 * HOST_MAX_GROUPS; ++i)
+    if (c->hs_ev[i]) cudaEventDestroy(c->hs_ev[i]);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return FICOCO_OK;
@@ -1005,6 +1015,10 @@ namespace {
 
 int ensure_staging(ficoco_ctx* c, size_t dev_bytes) {
   if (!c->hs_stream) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->hs_stream, cudaStreamNonBlocking));
+  if (!c->hs_run) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->hs_run, cudaStreamNonBlocking));
+  if (!c->hs_out) CUDA_TRY(c, cudaStreamCreateWithFlags(&c->hs_out, cudaStreamNonBlocking));
+  for (int i = 0; i < 2 * HOST_MAX_GROUPS; ++i)
+    if (!c->hs_ev[i]) CUDA_TRY(c, cudaEventCreateWithFlags(&c->hs_ev[i], cudaEventDisableTiming));
   if (dev_bytes > c->hs_dev_bytes) {
     if (c->hs_dev) { CUDA_TRY(c, cudaDeviceSynchronize()); cudaFree(c->hs_dev); c->hs_dev = nullptr; }
     CUDA_TRY(c, cudaMalloc((void**)&c->hs_dev, dev_bytes));
@@ -1030,13 +1044,19 @@ extern "C" int ficoco_v_reduce_host(ficoco_ctx* c, const ficoco_v_args* h, const
   if (h->dtype != FICOCO_FP32 && h->dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
   const int cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
   const size_t es = h->dtype == FICOCO_BF16 ? 2 : 4;
-  long long rows = 0, patches = 0, orows = 0, kept = 0;
-  for (int b = 0; b < h->batch; ++b) {
+  const int B = h->batch;
+  // prefix sums over images: input rows, patch tokens, output rows, preserved tokens
+  std::vector<long long> p_rows(B + 1, 0), p_patch(B + 1, 0), p_orow(B + 1, 0), p_kept(B + 1, 0);
+  for (int b = 0; b < B; ++b) {
     const int n = h->seqlens ? h->seqlens[b] : h->n_tokens;
     const int k = h->keep[h->n_keep == 1 ? 0 : b];
     if (n < cls + 1 || k < 0 || k > n - cls) return FICOCO_ERR_KEEP_RANGE;
-    rows += n; patches += n - cls; orows += cls + k; kept += k;
+    p_rows[b + 1] = p_rows[b] + n;
+    p_patch[b + 1] = p_patch[b] + n - cls;
+    p_orow[b + 1] = p_orow[b] + cls + k;
+    p_kept[b + 1] = p_kept[b] + k;
   }
+  const long long rows = p_rows[B], patches = p_patch[B], orows = p_orow[B], kept = p_kept[B];
   if (rows > c->max_tokens) return FICOCO_ERR_WORKSPACE;
   CUDA_TRY(c, cudaSetDevice(c->device));
   const size_t b_tok = (size_t)rows * h->dim * es, b_attn = (size_t)patches * h->heads * 4;
@@ -1049,7 +1069,6 @@ extern "C" int ficoco_v_reduce_host(ficoco_ctx* c, const ficoco_v_args* h, const
   int rc = ensure_staging(c, total);
   if (rc) return rc;
   Carver dv(c->hs_dev);
-  ficoco_v_args a = *h;
   char* d_tok = dv.take<char>(b_tok);
   char* d_attn = dv.take<char>(b_attn);
   char* d_pos = dv.take<char>(b_pos);
@@ -1057,21 +1076,85 @@ extern "C" int ficoco_v_reduce_host(ficoco_ctx* c, const ficoco_v_args* h, const
   char* d_kidx = dv.take<char>(b_kidx);
   char* d_po = dv.take<char>(b_posout);
   char* d_sc = dv.take<char>(b_sc);
-  cudaStream_t st = c->hs_stream;
-  CUDA_TRY(c, cudaMemcpyAsync(d_tok, h->tokens, b_tok, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(c, cudaMemcpyAsync(d_attn, h->attn, b_attn, cudaMemcpyHostToDevice, st));
-  if (h->pos) CUDA_TRY(c, cudaMemcpyAsync(d_pos, h->pos, b_pos, cudaMemcpyHostToDevice, st));
-  a.tokens = d_tok; a.attn = (const float*)d_attn; a.pos = h->pos ? (const int*)d_pos : nullptr;
-  a.out_tokens = d_out; a.kept_idx = (int*)d_kidx;
-  a.pos_out = h->pos_out ? (int*)d_po : nullptr;
-  a.scores_out = h->scores_out ? (float*)d_sc : nullptr;
-  rc = ficoco_v_reduce(c, &a, prm, st);
+
+  // Images are independent, so the batch goes through in groups of images: the upload of a
+  // group, the kernels of the group before it and the download of the one before that run at
+  // the same time on three streams (PCIe carries both directions at once).  Every group has its
+  // own slice of the staging area, so nothing is reused while in flight.
+  int n_groups = (int)(b_tok / HOST_GROUP_BYTES);
+  if (n_groups > HOST_MAX_GROUPS) n_groups = HOST_MAX_GROUPS;
+  if (n_groups > B) n_groups = B;
+  if (n_groups < 1) n_groups = 1;
+  cudaStream_t s_in = c->hs_stream, s_run = c->hs_run, s_out = c->hs_out;
+  if (n_groups == 1) s_run = s_out = s_in;
+  const size_t row_b = (size_t)h->dim * es;
+  int launches = 0;
+  rc = FICOCO_OK;
+  auto group_begin = [&](int g) { return (int)((long long)B * g / n_groups); };
+  // all uploads first: they depend on nothing, and queued ahead of everything else they never
+  // sit behind a download that is itself waiting for kernels
+  for (int g = 0; g < n_groups && rc == FICOCO_OK; ++g) {
+    const int b0 = group_begin(g), b1 = group_begin(g + 1);
+    const size_t o_tok = (size_t)p_rows[b0] * row_b, n_tok = (size_t)(p_rows[b1] - p_rows[b0]) * row_b;
+    const size_t o_at = (size_t)p_patch[b0] * h->heads * 4, n_at = (size_t)(p_patch[b1] - p_patch[b0]) * h->heads * 4;
+    const size_t o_ps = (size_t)p_patch[b0] * 4, n_ps = (size_t)(p_patch[b1] - p_patch[b0]) * 4;
+    cudaError_t e = cudaMemcpyAsync(d_tok + o_tok, (const char*)h->tokens + o_tok, n_tok, cudaMemcpyHostToDevice, s_in);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(d_attn + o_at, (const char*)h->attn + o_at, n_at, cudaMemcpyHostToDevice, s_in);
+    if (e == cudaSuccess && h->pos)
+      e = cudaMemcpyAsync(d_pos + o_ps, (const char*)h->pos + o_ps, n_ps, cudaMemcpyHostToDevice, s_in);
+    if (e == cudaSuccess && n_groups > 1) e = cudaEventRecord(c->hs_ev[2 * g], s_in);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; }
+  }
+  for (int g = 0; g < n_groups && rc == FICOCO_OK; ++g) {
+    const int b0 = group_begin(g), b1 = group_begin(g + 1);
+    const size_t o_tok = (size_t)p_rows[b0] * row_b;
+    const size_t o_at = (size_t)p_patch[b0] * h->heads * 4;
+    const size_t o_ps = (size_t)p_patch[b0] * 4, n_ps = (size_t)(p_patch[b1] - p_patch[b0]) * 4;
+    const size_t o_out = (size_t)p_orow[b0] * row_b, n_out = (size_t)(p_orow[b1] - p_orow[b0]) * row_b;
+    const size_t o_ki = (size_t)p_orow[b0] * 4, n_ki = (size_t)(p_orow[b1] - p_orow[b0]) * 4;
+    const size_t o_po = (size_t)p_kept[b0] * 4, n_po = (size_t)(p_kept[b1] - p_kept[b0]) * 4;
+    cudaError_t e = cudaSuccess;
+    if (n_groups > 1) e = cudaStreamWaitEvent(s_run, c->hs_ev[2 * g], 0);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; break; }
+    ficoco_v_args a = *h;
+    a.batch = b1 - b0;
+    a.tokens = d_tok + o_tok;
+    a.attn = (const float*)(d_attn + o_at);
+    a.pos = h->pos ? (const int*)(d_pos + o_ps) : nullptr;
+    if (h->seqlens) a.seqlens = h->seqlens + b0;
+    if (h->n_keep != 1) { a.keep = h->keep + b0; a.n_keep = b1 - b0; }
+    if (h->n_grid != 1) { a.grid_h = h->grid_h + b0; a.grid_w = h->grid_w + b0; a.n_grid = b1 - b0; }
+    a.out_tokens = d_out + o_out;
+    a.kept_idx = (int*)(d_kidx + o_ki);
+    a.pos_out = h->pos_out ? (int*)(d_po + o_po) : nullptr;
+    a.scores_out = h->scores_out ? (float*)(d_sc + o_ps) : nullptr;
+    rc = ficoco_v_reduce(c, &a, prm, s_run);
+    if (rc) break;
+    launches += c->launches;
+    if (n_groups > 1) {
+      e = cudaEventRecord(c->hs_ev[2 * g + 1], s_run);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, c->hs_ev[2 * g + 1], 0);
+    }
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync((char*)h->out_tokens + o_out, d_out + o_out, n_out, cudaMemcpyDeviceToHost, s_out);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync((char*)h->kept_idx + o_ki, d_kidx + o_ki, n_ki, cudaMemcpyDeviceToHost, s_out);
+    if (e == cudaSuccess && h->pos_out)
+      e = cudaMemcpyAsync((char*)h->pos_out + o_po, d_po + o_po, n_po, cudaMemcpyDeviceToHost, s_out);
+    if (e == cudaSuccess && h->scores_out)
+      e = cudaMemcpyAsync((char*)h->scores_out + o_ps, d_sc + o_ps, n_ps, cudaMemcpyDeviceToHost, s_out);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; }
+  }
+  // drain all three streams whatever happened, so that no copy outlives the call
+  const cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(s_run),
+                    e3 = cudaStreamSynchronize(s_out);
   if (rc) return rc;
-  CUDA_TRY(c, cudaMemcpyAsync(h->out_tokens, d_out, b_out, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(c, cudaMemcpyAsync(h->kept_idx, d_kidx, b_kidx, cudaMemcpyDeviceToHost, st));
-  if (h->pos_out) CUDA_TRY(c, cudaMemcpyAsync(h->pos_out, d_po, b_posout, cudaMemcpyDeviceToHost, st));
-  if (h->scores_out) CUDA_TRY(c, cudaMemcpyAsync(h->scores_out, d_sc, b_sc, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(c, cudaStreamSynchronize(st));
+  if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+    c->last_cuda = (int)(e1 != cudaSuccess ? e1 : e2 != cudaSuccess ? e2 : e3);
+    return FICOCO_ERR_CUDA;
+  }
+  c->launches = launches;
   return FICOCO_OK;
 }
 

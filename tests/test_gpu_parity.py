@@ -173,6 +173,33 @@ def test_back_to_back_steps_without_sync(ctx):
             assert np.array_equal(a, b), f"repetition {rep}: array {i} differs from the synchronised chain"
 
 
+@pytest.mark.parametrize("idx", [2, 4])
+def test_host_entry_point_in_image_groups(ctx, idx):
+    """Host-buffer call on a batch large enough to be cut into image groups (uploads, kernels
+    and downloads overlapped): every output equals the device-buffer call on the same bytes.
+    Workload 4 is ragged with per-image keep / grid arrays, workload 2 uniform."""
+    batch = synth.workload(idx)
+    pk = packing.pack_v(batch, DEV)
+    prm = parity.params_to_abi(fo.Params(), batch.has_cls)
+    keep = pk.keep if idx == 4 else pk.keep[0]
+    gh, gw = (pk.grid_h, pk.grid_w) if idx == 4 else (pk.grid_h[0], pk.grid_w[0])
+    d = ctx.ficoco_v_reduce(pk.tokens, pk.attn, keep, gh, gw, pk.heads, params=prm, want_scores=True,
+                            **pk.call_kwargs())
+    torch.cuda.synchronize()
+    ph = packing.pack_v(batch, None, pin=True)
+    pos_out = torch.empty(d.pos_out.shape, dtype=torch.int32).pin_memory()
+    scores = torch.empty(d.scores.shape, dtype=torch.float32).pin_memory()
+    h = ctx.ficoco_v_reduce_host(ph.tokens, ph.attn, keep, gh, gw, ph.heads, params=prm, pos_out=pos_out,
+                                 scores_out=scores, **ph.call_kwargs())
+    assert np.array_equal(binding.to_numpy(d.out_tokens), binding.to_numpy(h.out_tokens))
+    assert np.array_equal(binding.to_numpy(d.kept_idx), binding.to_numpy(h.kept_idx))
+    assert np.array_equal(binding.to_numpy(d.pos_out), pos_out.numpy())
+    # a group is planned on its own, so the column sums fold in another order: scores agree
+    # to rounding, the decisions taken from them are the same
+    np.testing.assert_allclose(scores.numpy(), binding.to_numpy(d.scores), rtol=1e-4, atol=1e-7)
+    assert ctx.ficoco_status() == 0
+
+
 def test_canaries_around_outputs(ctx):
     """Nothing is written outside the documented output extents."""
     batch = synth.workload(4, small=True)
