@@ -248,9 +248,20 @@ __device__ __noinline__ void select_image(
 
   for (int i = tid; i < nwin; i += nthr) win[i] = 0ull;
   #pragma unroll 1
-  for (int i = tid; i < np; i += nthr) {
-    sc[i] = __ldcg(s_raw + d.patch0 + i);
-    pp[i] = pos ? pos[d.patch0 + i] : i;
+  for (int i0 = tid; i0 < np; i0 += 4 * nthr) {    // four tokens' loads in flight per thread
+    float a[4];
+    int q[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = i0 + j * nthr;
+      a[j] = i < np ? __ldcg(s_raw + d.patch0 + i) : 0.f;
+      q[j] = (i < np && pos) ? pos[d.patch0 + i] : i;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int i = i0 + j * nthr;
+      if (i < np) { sc[i] = a[j]; pp[i] = q[j]; }
+    }
   }
   cta_sync(bar, nthr);
 

@@ -27,12 +27,53 @@ constexpr int F_THREADS = 544;    // + one producer warp
 constexpr int F_MAXSTAGE = 16;
 constexpr int F_MAXWON = 32;      // pieces per CTA (and therefore selections it can win)
 constexpr int F_POLL_LIMIT = 1 << 20;
-constexpr int F_P2ROWS = 3;       // rows a warp keeps in flight in pass 2
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+
+// The mean direction m (one float per column) is kept in shared memory so that a warp reads it
+// without bank conflicts: with 8 columns per 16-byte vector, floats 0-3 of vector v live in plane
+// A at 4v and floats 4-7 in plane B at 4(nvec + v); with 4 columns per vector there is one plane.
+template <int E>
+__device__ __forceinline__ int msum_slot(int c, int nvec) {
+  const int v = c / E, e = c % E;
+  return (e < 4 ? 0 : 4 * nvec) + 4 * v + (e & 3);
+}
+
+// Dot products of R rows (16-byte vectors u[r][k], vector lane + 32k of the row) with m, summed
+// over the warp.  m is read once for all R rows.
+template <class T, int VPL, int R>
+__device__ __forceinline__ void score_rows(const uint4 (&u)[R][VPL], const float* msum, int nvec, int lane,
+                                           float (&dot)[R]) {
+  constexpr int E = VecTraits<T>::E;
+#pragma unroll
+  for (int r = 0; r < R; ++r) dot[r] = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int v = lane + 32 * k;
+    const int vv = v < nvec ? v : 0;
+    float m[E];
+    const float4 ma = *reinterpret_cast<const float4*>(msum + 4 * vv);
+    m[0] = ma.x; m[1] = ma.y; m[2] = ma.z; m[3] = ma.w;
+    if (E == 8) {
+      const float4 mb = *reinterpret_cast<const float4*>(msum + 4 * (nvec + vv));
+      m[E - 4] = mb.x; m[E - 3] = mb.y; m[E - 2] = mb.z; m[E - 1] = mb.w;
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      float f[E];
+      unpack(u[r][k], f, (const T*)nullptr);
+      float t = 0.f;
+#pragma unroll
+      for (int e = 0; e < E; ++e) t = fmaf(f[e], m[e], t);
+      dot[r] += t;
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < R; ++r) dot[r] = warp_sum(dot[r]);
 }
 
 template <class T, int VPL>
@@ -46,6 +87,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     int* __restrict__ kept_idx, int* __restrict__ pos_out, unsigned* __restrict__ status,
     int nstage, int max_piece) {
   constexpr int E = VecTraits<T>::E;
+  constexpr int F_P2B = VPL <= 4 ? 2 : 1;   // rows a warp scores together in pass 2 (and has in flight from L2)
   extern __shared__ __align__(128) unsigned char fs_raw[];
   __shared__ uint64_t full_bar[F_MAXSTAGE], empty_bar[F_MAXSTAGE];
   __shared__ SelectShared sel_sh;
@@ -187,16 +229,24 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       for (int ww = 0; ww < FFOLD; ++ww) t += fold[(size_t)ww * D + c];
       pout[c] = t;
     }
-    __threadfence();
     cta_sync(1, F_NCONS);
-    if (tid == 0) atomicAdd(&cnt[w.img], 1);
+    if (tid == 0) {          // the barrier orders the CTA's stores before this one fence (cumulative)
+      __threadfence();
+      atomicAdd(&cnt[w.img], 1);
+    }
   }
   if (!ok && lane == 0) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
 
-  // pass 2: scores; the rows are L2-resident now and are read with plain loads
+  // pass 2: scores.  The last `nstage` row groups of pass 1 are still in the ring and are read
+  // from there (only when every wait of pass 1 succeeded); the older ones are L2-resident and
+  // are read with plain loads.
+  const int first_kept = ok ? seq - nstage : seq;   // groups numbered >= this are in shared memory
+  int seq2 = 0;
   for (int pi = p_begin; pi < p_end; ++pi) {
     const WorkItem w = pieces[pi];
     const ImgDesc d = desc[w.img];
+    const int seq_piece = seq2;                     // number of this piece's first group
+    seq2 += (w.nrows + FROWS - 1) / FROWS;
     if (tid == 0) {
       bool in = false;
       for (int it = 0; it < F_POLL_LIMIT && !in; ++it) {
@@ -224,50 +274,72 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
 #pragma unroll
         for (int k = 0; k < 8; ++k) t += q[k];
       }
-      msum[c] = t;
+      msum[msum_slot<E>(c, nvec)] = t;
     }
     cta_sync(1, F_NCONS);
     const float inv_np = 1.0f / (float)d.np;
     const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D;
-    for (int r0 = warp; r0 < w.nrows; r0 += FWARPS * F_P2ROWS) {
-      uint4 u[F_P2ROWS][VPL];
+    // This warp owns line `warp` of every 16-row group of the piece.  Groups numbered below
+    // g_res were overwritten in the ring and come from L2; the others are still in shared memory.
+    const int G = (w.nrows + FROWS - 1) / FROWS;
+    const int g_res = min(G, max(0, first_kept - seq_piece));
+    // norms of the warp's rows, lane l holding the one of group l
+    const int row_l = lane * FROWS + warp;
+    const float rn_l = (lane < G && row_l < w.nrows) ? __ldcg(rn + d.patch0 + w.r0 + row_l) : 0.f;
+    auto finish_row = [&](int g, float dot) {      // dot already summed over the warp
+      const int r = g * FROWS + warp;
+      const float rnv = g < 32 ? __shfl_sync(0xFFFFFFFFu, rn_l, g) : __ldcg(rn + d.patch0 + w.r0 + r);
+      if (lane == 0 && r < w.nrows)
+        s_raw[d.patch0 + w.r0 + r] = cA * (dot * rnv * inv_np) - (1.0f - cA) * a_s[r];
+    };
+    uint4 ub[F_P2B][VPL];
+    auto load_batch = [&](int g0) {
 #pragma unroll
-      for (int j = 0; j < F_P2ROWS; ++j) {
-        const int r = r0 + j * FWARPS;
+      for (int jb = 0; jb < F_P2B; ++jb) {
+        const int r = (g0 + jb) * FROWS + warp;
+        const bool on = g0 + jb < g_res && r < w.nrows;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
           const int v = lane + 32 * k;
-          u[j][k] = (r < w.nrows && v < nvec) ? ldg16(base + (size_t)r * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+          ub[jb][k] = (on && v < nvec) ? ldg16(base + (size_t)r * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
         }
       }
+    };
+    load_batch(0);
+    // the rows in the ring are scored while the first batch from L2 is in flight
+    #pragma unroll 1
+    for (int g0 = g_res; g0 < G; g0 += F_P2B) {
+      uint4 us[F_P2B][VPL];
 #pragma unroll
-      for (int j = 0; j < F_P2ROWS; ++j) {
-        const int r = r0 + j * FWARPS;
-        float dk[VPL];
+      for (int jb = 0; jb < F_P2B; ++jb) {
+        const int g = g0 + jb;
+        const bool on = g < G && g * FROWS + warp < w.nrows;
+        const unsigned char* rp =
+            ring + (size_t)((seq_piece + g) % nstage) * stage_bytes + (size_t)warp * row_bytes;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
           const int v = lane + 32 * k;
-          float f[E];
-          unpack(u[j][k], f, (const T*)nullptr);
-          const float* m = msum + (size_t)(v < nvec ? v : 0) * E;
-          float t = 0.f;
-#pragma unroll
-          for (int e = 0; e < E; ++e) t = fmaf(f[e], m[e], t);
-          dk[k] = t;
-        }
-        float dot = 0.f;
-#pragma unroll
-        for (int k = 0; k < VPL; ++k) dot += dk[k];
-        dot = warp_sum(dot);
-        if (lane == 0 && r < w.nrows) {
-          const float v_i = dot * __ldcg(rn + d.patch0 + w.r0 + r) * inv_np;
-          s_raw[d.patch0 + w.r0 + r] = cA * v_i - (1.0f - cA) * a_s[r];
+          us[jb][k] = (on && v < nvec) ? *reinterpret_cast<const uint4*>(rp + (size_t)v * 16) : make_uint4(0, 0, 0, 0);
         }
       }
+      float dot[F_P2B];
+      score_rows<T, VPL, F_P2B>(us, msum, nvec, lane, dot);
+#pragma unroll
+      for (int jb = 0; jb < F_P2B; ++jb)
+        if (g0 + jb < G) finish_row(g0 + jb, dot[jb]);
     }
-    __threadfence();
+    #pragma unroll 1
+    for (int g0 = 0; g0 < g_res; g0 += F_P2B) {
+      float dot[F_P2B];
+      score_rows<T, VPL, F_P2B>(ub, msum, nvec, lane, dot);
+#pragma unroll
+      for (int jb = 0; jb < F_P2B; ++jb)
+        if (g0 + jb < g_res) finish_row(g0 + jb, dot[jb]);
+      if (g0 + F_P2B < g_res) load_batch(g0 + F_P2B);
+    }
     cta_sync(1, F_NCONS);
     if (tid == 0) {
+      __threadfence();
       const int old = atomicAdd(&cnt[B + w.img], 1);
       if (old == d.n_chunks - 1 && nwon < F_MAXWON) won[nwon++] = w.img;
       __threadfence();
