@@ -23,7 +23,7 @@ namespace {
 
 constexpr int N_PLANS = 8;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
-constexpr int OUT_ROWS_PER_CTA = 32;  // == MROWS of the merge kernel
+constexpr int OUT_ROWS_PER_CTA = 16;  // <= MROWS of the merge kernel
 constexpr int NSPLIT_MAX = 16;
 constexpr int TARGET_CTAS = 2 * 148;
 

@@ -4,6 +4,7 @@
 
 namespace ficoco {
 
+constexpr int MHUB = 8;        // source rows a lane has in flight for a hub row
 constexpr int MROWS = 32;      // output rows per CTA (four per warp)
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
 constexpr int MHEAVY = 4;      // rows with more sources than this are split into 32-vector blocks over the warps
@@ -286,7 +287,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   if (!fits) return;
 
   // ---- hub rows: (row, block of 32 vectors) items dealt to the warps; each lane sums all the
-  // sources of its one vector in list order, eight source rows in flight ---------------------
+  // sources of its one vector in list order, MHUB source rows in flight ---------------------
   const int nh = n_heavy;
   const int nblk = (nvec + 31) / 32;
   #pragma unroll 1
@@ -304,17 +305,17 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     float acc[E];
     unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
     #pragma unroll 1
-    for (int k = 0; k < n; k += 8) {
-      uint4 u[8];
-      float a[8];
+    for (int k = 0; k < n; k += MHUB) {
+      uint4 u[MHUB];
+      float a[MHUB];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < MHUB; ++j) {
         const bool on = k + j < n;
         a[j] = on ? lw[b0 + k + j] : 0.f;
         u[j] = on ? ldg16(pbase + (size_t)lsrc[b0 + k + j] * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < MHUB; ++j) {
         float f[E];
         unpack(u[j], f, (const T*)nullptr);
 #pragma unroll
