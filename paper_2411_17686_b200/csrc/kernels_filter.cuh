@@ -220,11 +220,10 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
 // positions are read from global memory once and kept there with the keys and window bids.
 // ---------------------------------------------------------------------------------------
 __host__ __device__ inline size_t select_work_bytes(int np, int nwin) {
-  return (size_t)np * 12 + 8 + (size_t)nwin * 8;
+  return (size_t)np * 12 + 8 + (size_t)nwin * 8 + 16 + 4 * 256 * sizeof(int);
 }
 
 struct SelectShared {
-  int hist[256];
   int warp_tot[33];
   uint32_t prefix;
   int remaining;
@@ -243,9 +242,12 @@ __device__ __noinline__ void select_image(
   const int nwc = (d.gw + window - 1) / window;
   const int nwr = (d.gh + window - 1) / window;
   const int nwin = penalty ? nwc * nwr : 0;
+  // [4][256], one histogram per digit, 16-byte aligned
+  int* hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(win + nwin) + 15) & ~(uintptr_t)15);
 
   #pragma unroll 1
-
+  for (int i = tid; i < 4 * 256; i += nthr) hist[i] = 0;
+  #pragma unroll 1
   for (int i = tid; i < nwin; i += nthr) win[i] = 0ull;
   #pragma unroll 1
   for (int i0 = tid; i0 < np; i0 += 4 * nthr) {    // four tokens' loads in flight per thread
@@ -295,36 +297,42 @@ __device__ __noinline__ void select_image(
   cta_sync(bar, nthr);
 
   // ---- radix select: key of the n_src-th largest ------------------------------------------
+  // Two barriers per digit: count, then the first warp finds the digit's bin; every digit has a
+  // histogram of its own, zeroed up front.
   const int k = d.n_src;
   uint32_t thr = 0;       // threshold key
   int need_eq = 0;        // how many keys equal to thr are selected (lowest indices)
   if (k > 0 && k < np) {
-    if (tid == 0) { sh.prefix = 0; sh.remaining = k; }
-    uint32_t mask = 0;
+    const int lane = tid & 31;
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k;
     #pragma unroll 1
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
-      if (tid < 256) sh.hist[tid] = 0;
-      cta_sync(bar, nthr);
-      const uint32_t prefix = sh.prefix;
+      int* h = hist + 256 * pass;
       #pragma unroll 1
       for (int i = tid; i < np; i += nthr) {
         const uint32_t key = keys[i];
-        if ((key & mask) == prefix) atomicAdd(&sh.hist[(key >> shift) & 255], 1);
+        if ((key & mask) == prefix) atomicAdd(&h[(key >> shift) & 255], 1);
       }
       cta_sync(bar, nthr);
       if (tid < 32) {
-        // lane l owns bins 255-8l .. 248-8l (descending); find where the running count
-        // from the top reaches `remaining`
-        const int remaining = sh.remaining;
+        // lane l owns bins 255-8l .. 248-8l (descending); find where the running count from
+        // the top reaches `remaining`
         int c[8], tot = 0;
+        {
+          const int4 lo = *reinterpret_cast<const int4*>(h + 248 - 8 * lane);
+          const int4 hi = *reinterpret_cast<const int4*>(h + 252 - 8 * lane);
+          c[0] = hi.w; c[1] = hi.z; c[2] = hi.y; c[3] = hi.x;
+          c[4] = lo.w; c[5] = lo.z; c[6] = lo.y; c[7] = lo.x;
+        }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = sh.hist[255 - 8 * tid - j]; tot += c[j]; }
+        for (int j = 0; j < 8; ++j) tot += c[j];
         int inc = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-          if (tid >= o) inc += n;
+          if (lane >= o) inc += n;
         }
         const int before = inc - tot;
         if (before < remaining && inc >= remaining) {
@@ -332,38 +340,47 @@ __device__ __noinline__ void select_image(
 #pragma unroll
           for (int j = 0; j < 8; ++j) {
             if (cum < remaining && cum + c[j] >= remaining) {
-              sh.prefix = prefix | ((uint32_t)(255 - 8 * tid - j) << shift);
+              sh.prefix = prefix | ((uint32_t)(255 - 8 * lane - j) << shift);
               sh.remaining = remaining - cum;
             }
             cum += c[j];
           }
         }
       }
-      mask |= 0xFFu << shift;
       cta_sync(bar, nthr);
+      prefix = sh.prefix;
+      remaining = sh.remaining;
+      mask |= 0xFFu << shift;
     }
-    thr = sh.prefix;
-    need_eq = sh.remaining;
+    thr = prefix;
+    need_eq = remaining;
   }
 
   // ---- ordered compaction into S and T ------------------------------------------------------
-  int eq_base = 0, sel_base = 0;
-  #pragma unroll 1
-  for (int base = 0; base < np; base += nthr) {
-    const int i = base + tid;
-    const bool valid = i < np;
-    const uint32_t key = valid ? keys[i] : 0u;
-    bool gt, eq;
-    if (k <= 0) { gt = false; eq = false; }
-    else if (k >= np) { gt = valid; eq = false; }
-    else { gt = valid && key > thr; eq = valid && key == thr; }
+  // Each thread takes a run of consecutive tokens; one block scan over packed counts
+  // (greater-than in the high half, equal in the low half) places every run.
+  {
+    const int ipt = (np + nthr - 1) / nthr;
+    const int i_lo = min(np, tid * ipt), i_hi = min(np, i_lo + ipt);
+    int n_gt = 0, n_eq = 0;
+    #pragma unroll 1
+    for (int i = i_lo; i < i_hi; ++i) {
+      const uint32_t key = keys[i];
+      if (k >= np) ++n_gt;
+      else if (k > 0) { n_gt += key > thr ? 1 : 0; n_eq += key == thr ? 1 : 0; }
+    }
     int tot;
-    const int eq_rank = eq_base + block_exclusive_scan(eq ? 1 : 0, sh.warp_tot, &tot, bar, nthr);
-    eq_base += tot;
-    const bool sel = gt || (eq && eq_rank < need_eq);
-    const int sel_rank = sel_base + block_exclusive_scan(sel ? 1 : 0, sh.warp_tot, &tot, bar, nthr);
-    sel_base += tot;
-    if (valid) {
+    const int packed = block_exclusive_scan((n_gt << 16) | n_eq, sh.warp_tot, &tot, bar, nthr);
+    int gt_before = packed >> 16, eq_before = packed & 0xFFFF;
+    #pragma unroll 1
+    for (int i = i_lo; i < i_hi; ++i) {
+      const uint32_t key = keys[i];
+      bool gt, eq;
+      if (k <= 0) { gt = false; eq = false; }
+      else if (k >= np) { gt = true; eq = false; }
+      else { gt = key > thr; eq = key == thr; }
+      const bool sel = gt || (eq && eq_before < need_eq);
+      const int sel_rank = gt_before + min(eq_before, need_eq);   // selected tokens before i
       if (sel) {
         S_idx[d.src0 + sel_rank] = i;
       } else {
@@ -372,6 +389,8 @@ __device__ __noinline__ void select_image(
         kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
         if (pos_out) pos_out[d.tgt0 + tp] = pp[i];
       }
+      gt_before += gt ? 1 : 0;
+      eq_before += eq ? 1 : 0;
     }
   }
   #pragma unroll 1
