@@ -397,6 +397,9 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
     cudaFuncSetAttribute(k_correlate_umma<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<3, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<4, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<6, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<6, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma<6, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
   }
   {
     const int fmax = 221 * 1024;
@@ -446,12 +449,11 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = p->max_list = 0;
   p->need_finalize = false;
   p->umma = key.mode == 0 && key.dtype == FICOCO_BF16 && key.dim % UKB == 0;
-  const int tile_rows_max = p->umma ? UM : CBM;       // source rows per correlate CTA
+  int tile_rows_max = p->umma ? UM : CBM;             // source rows per correlate CTA (decided below)
   const int col_granule = p->umma ? 16 : CBN;
   int um_a_rows = 8, um_cols = 16;
 
   // first pass: sizes
-  long long base_strips = 0;
   for (int b = 0; b < B; ++b) {
     ImgDesc& d = p->h_desc[b];
     const int ntok = key.ntok[b];
@@ -483,7 +485,6 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     d.list_len = L;
     d.frac = frac;
     if (L > p->max_list) p->max_list = L;
-    if (L > 0) base_strips += (d.n_src + tile_rows_max - 1) / tile_rows_max;
   }
   // ---- fused filter kernel: piece size and feasibility -------------------------------------
   const int esz = key.dtype == FICOCO_BF16 ? 2 : 4;
@@ -508,11 +509,52 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     f_rc = (count(rc1) <= c->num_sms && rc1 * 10 <= rc0 * 16) ? rc1 : rc0;
   }
 
+  // ---- correlate tiling ---------------------------------------------------------------------
+  // A CTA gathers (tile rows + split columns) token rows per k-block from L2, which is what
+  // bounds the stage.  Tiles of up to 256 rows (two MMA sub-tiles sharing one column tile) cut
+  // that traffic but need the whole SM; tiles of up to 128 rows let two CTAs share an SM.
+  // Both are costed as (waves x rows gathered per CTA x CTAs per SM) and the cheaper one is used.
+  struct CorrChoice { int tile_rows, want_split; long long load; };
+  auto cost_corr = [&](int rows_max, int ctas_per_sm) {
+    CorrChoice ch{rows_max, 1, 0};
+    long long strips = 0;
+    for (int b = 0; b < B; ++b)
+      if (p->h_desc[b].list_len > 0) strips += (p->h_desc[b].n_src + rows_max - 1) / rows_max;
+    if (strips == 0) return ch;
+    const long long slots = (long long)c->num_sms * ctas_per_sm;
+    long long ws = slots / strips;
+    if (ws < 1) ws = 1;
+    if (ws > NSPLIT_MAX) ws = NSPLIT_MAX;
+    ch.want_split = (int)ws;
+    long long n_ctas = 0, max_rows = 0;
+    for (int b = 0; b < B; ++b) {
+      const ImgDesc& d = p->h_desc[b];
+      if (d.list_len == 0) continue;
+      int ns = ch.want_split;
+      const int max_by_cols = (d.n_tgt + col_granule - 1) / col_granule;
+      if (ns > max_by_cols) ns = max_by_cols;
+      int cps = ((d.n_tgt + ns - 1) / ns + col_granule - 1) / col_granule * col_granule;
+      if (p->umma && cps > UN_MAX) cps = UN_MAX;
+      ns = (d.n_tgt + cps - 1) / cps;
+      const int ntile = (d.n_src + rows_max - 1) / rows_max;
+      const int trows = ((d.n_src + ntile - 1) / ntile + 7) / 8 * 8;
+      n_ctas += (long long)ntile * ns;
+      if (trows + cps > max_rows) max_rows = trows + cps;
+    }
+    const long long waves = (n_ctas + slots - 1) / slots;
+    const long long per_sm = n_ctas < slots ? (n_ctas + c->num_sms - 1) / c->num_sms : ctas_per_sm;
+    ch.load = waves * max_rows * per_sm;
+    return ch;
+  };
   int want_split = 1;
-  if (base_strips > 0) {
-    want_split = (int)(TARGET_CTAS / base_strips);
-    if (want_split < 1) want_split = 1;
-    if (want_split > NSPLIT_MAX) want_split = NSPLIT_MAX;
+  {
+    CorrChoice best = cost_corr(tile_rows_max, 2);
+    if (p->umma) {
+      const CorrChoice wide = cost_corr(UM * UM_SUB, 1);
+      if (wide.load > 0 && wide.load * 10 < best.load * 9) best = wide;   // only for a clear gain
+    }
+    tile_rows_max = best.tile_rows;
+    want_split = best.want_split;
   }
 
   for (int b = 0; b < B; ++b) {
@@ -626,14 +668,19 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     // shared-memory ring of the tensor-core correlate: prefer a size that lets two CTAs share an SM
     p->um_a_bytes = um_a_rows * 128;
     p->um_stage_bytes = p->um_a_bytes + um_cols * 128;
+    const int n_sub = (um_a_rows + UM - 1) / UM;       // row sub-tiles (MMAs per k-step) of the largest tile
     p->um_tmem_cols = 32;
-    while (p->um_tmem_cols < um_cols) p->um_tmem_cols *= 2;
-    const size_t slack = 1024 + (p->um_stage_bytes < UM * 128 ? UM * 128 - p->um_stage_bytes : 0);
+    while (p->um_tmem_cols < n_sub * um_cols) p->um_tmem_cols *= 2;
+    if (p->um_tmem_cols > 512) return FICOCO_ERR_UNSUPPORTED;
+    // every MMA reads 128 A rows: behind the last stage there must be room for the rows past the tile
+    const size_t a_span = (size_t)n_sub * UM * 128;
+    const size_t slack = 1024 + ((size_t)p->um_stage_bytes < a_span ? a_span - p->um_stage_bytes : 0);
     p->um_nstage = 0;
-    for (int ns = 4; ns >= 2 && !p->um_nstage; --ns)
+    // (a CTA that takes more than half of TMEM has the SM to itself anyway: use the deepest ring)
+    for (int ns = 4; ns >= 2 && !p->um_nstage && p->um_tmem_cols <= 256; --ns)
       if ((size_t)ns * p->um_stage_bytes + slack <= 106 * 1024) p->um_nstage = ns;
-    for (int ns = 4; ns >= 2 && !p->um_nstage; --ns)
-      if ((size_t)ns * p->um_stage_bytes + slack <= 220 * 1024) p->um_nstage = ns;
+    for (int ns = 6; ns >= 2 && !p->um_nstage; --ns)
+      if (ns != 5 && (size_t)ns * p->um_stage_bytes + slack <= 220 * 1024) p->um_nstage = ns;
     if (!p->um_nstage) return FICOCO_ERR_UNSUPPORTED;
     p->um_smem = (size_t)p->um_nstage * p->um_stage_bytes + slack;
     // the epilogue helpers hand their lists back through the ring
@@ -819,7 +866,8 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       c->e_w, c->e_c)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
-    if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                                  \
+    if (p->um_nstage == 6) FICOCO_UMMA_LAUNCH(6, LC);                                                  \
+    else if (p->um_nstage == 4) FICOCO_UMMA_LAUNCH(4, LC);                                             \
     else if (p->um_nstage == 3) FICOCO_UMMA_LAUNCH(3, LC);                                             \
     else FICOCO_UMMA_LAUNCH(2, LC);                                                                    \
   } while (0)

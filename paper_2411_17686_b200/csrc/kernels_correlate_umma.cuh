@@ -21,7 +21,8 @@
 
 namespace ficoco {
 
-constexpr int UM = 128;          // accumulator rows per CTA
+constexpr int UM = 128;          // accumulator rows per MMA (one TMEM lane each)
+constexpr int UM_SUB = 2;        // row sub-tiles per CTA: up to 256 discarded tokens share one gathered column tile
 constexpr int UN_MAX = 256;      // accumulator columns per CTA
 constexpr int UKB = 64;          // bf16 elements per k-block (one 128-byte swizzle row)
 constexpr int UTHREADS = 288;    // warps 0-3 gather + epilogue, warp 4 MMA, warps 5-8 epilogue helpers
@@ -144,7 +145,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
-  __shared__ int rowS[UM], rowT[UN_MAX];
+  __shared__ int rowS[UM * UM_SUB], rowT[UN_MAX];
   __shared__ float rnT[UN_MAX];
   __shared__ int failed, acc_committed, is_last;
 
@@ -156,10 +157,11 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   const int ncols = min(d.n_tgt, col_begin + d.cols_per_split) - col_begin;   // 1..256
   const int n_pad = (ncols + 15) & ~15;
   const int nkb = D / UKB;
+  const int nsub = (w.nrows + UM - 1) / UM;       // 1 or 2; sub-tile s accumulates in TMEM columns [s * n_pad, (s + 1) * n_pad)
   const uint32_t ring = (smem_u32(um_raw) + 1023u) & ~1023u;
 
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full_bar[s], 128); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full_bar[s], 256); mbar_init(&empty_bar[s], 1); }
     mbar_init(&acc_bar, 1);
     failed = 0;
     acc_committed = 0;
@@ -176,7 +178,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   // any of its blocks starts, the filter grid is complete as well.
   grid_dep_wait();
   grid_dep_launch();
-  if (tid < UM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
+  if (tid < UM * UM_SUB) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
   for (int c = tid; c < UN_MAX; c += UTHREADS) {
     const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
     rowT[c] = p;
@@ -187,10 +189,31 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
 
-  if (warp < 4) {
-    // ---------------- producer: gather rows, 16 bytes per thread per copy -------------------
-    const int chunk = tid & 7;          // 16-byte chunk inside the 128-byte row
-    const int rsub = tid >> 3;          // 0..15
+  if (warp != 4) {
+    // ---------------- producers (all eight epilogue warps): gather rows, 16 bytes per copy -------
+    // Thread pt copies chunk (pt & 7) of rows (pt >> 3) + 32 i of the A tile and of the B tile.
+    // Row offsets stay in registers and the swizzled destination advances by a constant
+    // (32 rows = 4 KB), so a copy costs an add and the cp.async itself.
+    const int pt = warp < 4 ? tid : tid - 32;
+    const int chunk = pt & 7;
+    const int rsub = pt >> 3;           // 0..31
+    uint32_t offA[UM * UM_SUB / 32], offB[UN_MAX / 32];
+    uint32_t onA = 0, onB = 0;
+#pragma unroll
+    for (int i = 0; i < UM * UM_SUB / 32; ++i) {
+      const int r = rsub + 32 * i;
+      const bool on = r < w.nrows;
+      offA[i] = on ? (uint32_t)rowS[r] * (uint32_t)D : 0u;
+      onA |= on ? 1u << i : 0u;
+    }
+#pragma unroll
+    for (int i = 0; i < UN_MAX / 32; ++i) {
+      const int r = rsub + 32 * i;
+      const bool on = r < ncols;
+      offB[i] = on ? (uint32_t)rowT[r] * (uint32_t)D : 0u;
+      onB |= on ? 1u << i : 0u;
+    }
+    const uint32_t dsw = (uint32_t)((rsub >> 3) * 1024 + (rsub & 7) * 128 + ((chunk ^ (rsub & 7)) << 4));
     const __nv_bfloat16* tbase = tokens + (size_t)(d.row0 + d.n_cls) * D + chunk * 8;
     bool ok = true;
     // a stage is published LAG iterations after its copies were issued; LAG < NSTAGE - 1 leaves
@@ -201,15 +224,15 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
         const int s = kb % NSTAGE;
         if (kb >= NSTAGE && ok) ok = mbar_wait(&empty_bar[s], ((kb / NSTAGE) - 1) & 1);
         if (ok) {
-          const uint32_t a0 = ring + (uint32_t)s * stage_bytes;
+          const uint32_t a0 = ring + (uint32_t)s * stage_bytes + dsw;
           const uint32_t b0 = a0 + (uint32_t)a_bytes;
           const __nv_bfloat16* src = tbase + (size_t)kb * UKB;
-          for (int r = rsub; r < w.nrows; r += 16)
-            cp_async16(a0 + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4),
-                       src + (size_t)rowS[r] * D);
-          for (int r = rsub; r < ncols; r += 16)
-            cp_async16(b0 + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4),
-                       src + (size_t)rowT[r] * D);
+#pragma unroll
+          for (int i = 0; i < UM * UM_SUB / 32; ++i)
+            if (onA >> i & 1u) cp_async16(a0 + i * 4096, src + offA[i]);
+#pragma unroll
+          for (int i = 0; i < UN_MAX / 32; ++i)
+            if (onB >> i & 1u) cp_async16(b0 + i * 4096, src + offB[i]);
         }
       }
       cp_async_commit();
@@ -223,86 +246,90 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     }
     cp_async_wait<0>();
     if (!ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
-
-    // ---------------- epilogue: lane = accumulator row ---------------------------------------
     bool acc_ok = ok && mbar_wait(&acc_bar, 0);
     if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
-    __threadfence_block();
-    asm volatile("bar.arrive 2, 256;" ::: "memory");     // releases the helper warps
     tc_fence_after();
-    const int row = tid;                               // TMEM lane == accumulator row
-    const bool row_valid = row < w.nrows;
-    const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
+   if (warp < 4) {
+    // ---------------- epilogue: lane = accumulator row ---------------------------------------
     // this warp scans the lower half of the columns, its helper warp (same TMEM lanes) the
     // upper half; the helper's list comes back through the (now idle) operand ring
-    float v[LCAP];
-    int ix[LCAP];
     const int c_mid = ((n_pad / 16 + 1) / 2) * 16;
-    if (acc_ok) epilogue_scan<LCAP>(tmem_base + ((uint32_t)(warp * 32) << 16), 0, c_mid, ncols, col_begin, rs, rnT,
-                                    row_valid, L, v, ix);
-    else {
+    #pragma unroll 1
+    for (int sub = 0; sub < nsub; ++sub) {
+      const int row = sub * UM + tid;                  // TMEM lane == accumulator row of the sub-tile
+      const bool row_valid = row < w.nrows;
+      const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
+      float v[LCAP];
+      int ix[LCAP];
+      if (acc_ok && sub * UM + warp * 32 < w.nrows)
+        epilogue_scan<LCAP>(tmem_base + (uint32_t)(sub * n_pad) + ((uint32_t)(warp * 32) << 16), 0, c_mid, ncols,
+                            col_begin, rs, rnT, row_valid, L, v, ix);
+      else {
 #pragma unroll
-      for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-    }
-    cta_sync(1, 256);                                  // helper lists are in shared memory
-    {
-      const float* hv = reinterpret_cast<const float*>(um_raw + (ring - smem_u32(um_raw)));
-      const int* hi = reinterpret_cast<const int*>(hv + UM * LCAP);
+        for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+      }
+      cta_sync(1, 256);                                // helper lists of this sub-tile are in shared memory
+      {
+        const float* hv = reinterpret_cast<const float*>(um_raw + (ring - smem_u32(um_raw)));
+        const int* hi = reinterpret_cast<const int*>(hv + UM * LCAP);
 #pragma unroll
-      for (int e = 0; e < LCAP; ++e) {
-        if (e < L) {
-          float cv = hv[row * LCAP + e];
-          int ci = hi[row * LCAP + e];
-          bool shift = ci == INT_MAX;                  // empty helper slot: nothing to insert
-          if (!shift) {
-            shift = false;
+        for (int e = 0; e < LCAP; ++e) {
+          if (e < L) {
+            float cv = hv[tid * LCAP + e];
+            int ci = hi[tid * LCAP + e];
+            bool shift = ci == INT_MAX;                // empty helper slot: nothing to insert
+            if (!shift) {
+              shift = false;
 #pragma unroll
-            for (int k = 0; k < LCAP; ++k)
-              if (k < L && (shift || toplist_better(cv, ci, v[k], ix[k]))) {
-                const float tv = v[k]; const int ti = ix[k];
-                v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
-                shift = true;
-              }
+              for (int k = 0; k < LCAP; ++k)
+                if (k < L && (shift || toplist_better(cv, ci, v[k], ix[k]))) {
+                  const float tv = v[k]; const int ti = ix[k];
+                  v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+                  shift = true;
+                }
+            }
           }
         }
       }
-    }
-    if (row_valid) {
-      const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
+      if (row_valid) {
+        const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + row) * d.nsplit + w.aux) * L;
 #pragma unroll
-      for (int k = 0; k < LCAP; ++k)
-        if (k < L) {
-          part_val[o + k] = v[k];
-          part_idx[o + k] = ix[k] == INT_MAX ? -1 : ix[k];
-        }
+        for (int k = 0; k < LCAP; ++k)
+          if (k < L) {
+            part_val[o + k] = v[k];
+            part_idx[o + k] = ix[k] == INT_MAX ? -1 : ix[k];
+          }
+      }
+      if (sub + 1 < nsub) cta_sync(1, 256);            // the helpers may reuse the hand-over area
     }
-  } else if (warp > 4) {
+   } else {
     // ---------------- epilogue helpers: upper half of the columns --------------------------------
-    // sleep on hardware barrier 2 until the gather warps have seen the accumulator complete
-    // (polling the mbarrier from here would take issue slots from the gather warps)
-    cta_sync(2, 256);
-    bool acc_ok = !failed;
-    acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);
-    tc_fence_after();
     const int grp = warp & 3;                          // TMEM lanes this warp may read
-    const int row = grp * 32 + lane;
-    const bool row_valid = row < w.nrows;
-    const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
-    float v[LCAP];
-    int ix[LCAP];
     const int c_mid = ((n_pad / 16 + 1) / 2) * 16;
-    if (acc_ok) epilogue_scan<LCAP>(tmem_base + ((uint32_t)(grp * 32) << 16), c_mid, n_pad, ncols, col_begin, rs,
-                                    rnT, row_valid, L, v, ix);
-    else {
-#pragma unroll
-      for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
-    }
     float* hv = reinterpret_cast<float*>(um_raw + (ring - smem_u32(um_raw)));
     int* hi = reinterpret_cast<int*>(hv + UM * LCAP);
+    #pragma unroll 1
+    for (int sub = 0; sub < nsub; ++sub) {
+      const int lrow = grp * 32 + lane;
+      const int row = sub * UM + lrow;
+      const bool row_valid = row < w.nrows;
+      const float rs = row_valid ? rn[d.patch0 + rowS[row]] : 0.f;
+      float v[LCAP];
+      int ix[LCAP];
+      if (acc_ok && sub * UM + grp * 32 < w.nrows)
+        epilogue_scan<LCAP>(tmem_base + (uint32_t)(sub * n_pad) + ((uint32_t)(grp * 32) << 16), c_mid, n_pad, ncols,
+                            col_begin, rs, rnT, row_valid, L, v, ix);
+      else {
 #pragma unroll
-    for (int k = 0; k < LCAP; ++k) { hv[row * LCAP + k] = v[k]; hi[row * LCAP + k] = ix[k]; }
-    cta_sync(1, 256);
+        for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+      }
+#pragma unroll
+      for (int k = 0; k < LCAP; ++k) { hv[lrow * LCAP + k] = v[k]; hi[lrow * LCAP + k] = ix[k]; }
+      cta_sync(1, 256);
+      if (sub + 1 < nsub) cta_sync(1, 256);
+    }
+   }
   } else {
     // ---------------- MMA issuer (one lane) ---------------------------------------------------
     if (lane == 0) {
@@ -316,9 +343,14 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
         const uint32_t a0 = ring + (uint32_t)s * stage_bytes;
         const uint64_t ad = umma_smem_desc(a0), bd = umma_smem_desc(a0 + (uint32_t)a_bytes);
 #pragma unroll
-        for (int k4 = 0; k4 < UKB / 16; ++k4)
+        for (int k4 = 0; k4 < UKB / 16; ++k4) {
           umma_bf16(tmem_base, ad + (uint64_t)(k4 * 2), bd + (uint64_t)(k4 * 2), idesc,
                     (kb > 0 || k4 > 0) ? 1u : 0u);
+          // second row sub-tile: A rows 128.. (UM * 128 bytes further, in 16-byte units), same B
+          if (nsub > 1)
+            umma_bf16(tmem_base + (uint32_t)n_pad, ad + (uint64_t)(UM * 128 / 16) + (uint64_t)(k4 * 2),
+                      bd + (uint64_t)(k4 * 2), idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+        }
         umma_commit(&empty_bar[s]);      // frees the stage once these MMAs have read it
       }
       if (ok) { umma_commit(&acc_bar); acc_committed = 1; }   // accumulator complete
