@@ -1,12 +1,16 @@
 // Correlate stage on the 5th-generation tensor cores (bf16 tokens).
 //
-// One CTA owns up to 128 discarded tokens (rows of the accumulator, one TMEM lane each) and
-// one column split (<= 256 preserved tokens) of one image:
-//   warps 0-3  gather the token rows with 16-byte cp.async into a ring of 128B-swizzled,
+// One CTA owns a tile of discarded tokens (rows of the accumulator, one TMEM lane each) and
+// one column split (<= 256 preserved tokens) of one image.  A tile has up to 128 rows, or up
+// to 256 as two sub-tiles that share the gathered column tile and accumulate in adjacent TMEM
+// column ranges:
+//   warps 0-3, 5-8  gather the token rows with 16-byte cp.async into a ring of 128B-swizzled,
 //              K-major shared-memory tiles (64 bf16 of the hidden dimension per stage);
 //   warp  4    allocates TMEM and issues tcgen05.mma (M = 128, N = columns rounded to 16,
-//              K = 16 per instruction, fp32 accumulation of exact bf16 products);
-//   warps 0-3  afterwards read their 32 TMEM lanes back with tcgen05.ld, scale by
+//              K = 16 per instruction, fp32 accumulation of exact bf16 products), one per
+//              sub-tile and k-step;
+//   warps 0-3, 5-8  afterwards read TMEM lanes back with tcgen05.ld (warps 0-3 the lower half
+//              of the columns, warps 5-8 the upper half of the same lanes), scale by
 //              rn_i * rn_j to cosines and keep each row's L <= LCAP largest entries in registers.
 // Rows / columns past the valid range are never loaded: their shared memory is garbage that
 // only reaches accumulator rows / columns the epilogue ignores.
@@ -25,7 +29,7 @@ constexpr int UM = 128;          // accumulator rows per MMA (one TMEM lane each
 constexpr int UM_SUB = 2;        // row sub-tiles per CTA: up to 256 discarded tokens share one gathered column tile
 constexpr int UN_MAX = 256;      // accumulator columns per CTA
 constexpr int UKB = 64;          // bf16 elements per k-block (one 128-byte swizzle row)
-constexpr int UTHREADS = 288;    // warps 0-3 gather + epilogue, warp 4 MMA, warps 5-8 epilogue helpers
+constexpr int UTHREADS = 288;    // warps 0-3 and 5-8 gather + epilogue, warp 4 MMA
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -131,7 +135,7 @@ __device__ __forceinline__ void epilogue_scan(uint32_t tmem_lane, int c_lo, int 
 }
 
 // Dynamic shared memory: [1024-aligned] ring of NSTAGE stages, each an A tile (a_bytes: the
-// valid source rows rounded up to 8, x 128 B) followed by a B tile (column rows x 128 B).  The
+// valid source rows rounded up to 8, x 128 B) followed by a B tile (column rows x 128 B).  An
 // MMA always reads 128 A rows; rows past a_bytes alias the B tile (or the slack the host adds
 // behind the ring) and only feed accumulator rows that are never read.
 template <int NSTAGE, int LCAP>
@@ -250,7 +254,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
     tc_fence_after();
-   if (warp < 4) {
+    if (warp < 4) {
     // ---------------- epilogue: lane = accumulator row ---------------------------------------
     // this warp scans the lower half of the columns, its helper warp (same TMEM lanes) the
     // upper half; the helper's list comes back through the (now idle) operand ring
@@ -303,7 +307,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       }
       if (sub + 1 < nsub) cta_sync(1, 256);            // the helpers may reuse the hand-over area
     }
-   } else {
+    } else {
     // ---------------- epilogue helpers: upper half of the columns --------------------------------
     const int grp = warp & 3;                          // TMEM lanes this warp may read
     const int c_mid = ((n_pad / 16 + 1) / 2) * 16;
@@ -329,7 +333,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       cta_sync(1, 256);
       if (sub + 1 < nsub) cta_sync(1, 256);
     }
-   }
+    }
   } else {
     // ---------------- MMA issuer (one lane) ---------------------------------------------------
     if (lane == 0) {
