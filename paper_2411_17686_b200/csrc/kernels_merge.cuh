@@ -120,14 +120,23 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   if (tp_hi > tp_lo) {
     if (one_pass) {
 #pragma unroll
+      int t4[4];
+#pragma unroll
       for (int i = 0; i < 4; ++i) {
+        // target, source and weight are fetched together: a source fetched only for the matches
+        // would add a second round trip to L2
         const int e = tid + 256 * i;
-        const int t = e < n_ent ? e_tgt[d.ent0 + e] : -1;
+        const bool on = e < n_ent;
+        t4[i] = on ? e_tgt[d.ent0 + e] : -1;
+        st_src[i] = on ? S_idx[d.src0 + e / L] : 0;
+        st_w[i] = on ? e_w[d.ent0 + e] : 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int t = t4[i];
         if (t >= tp_lo && t < tp_hi) {
           st_row[i] = t - tp_lo;
           st_slot[i] = atomicAdd(&cnt[t - tp_lo], 1);
-          st_src[i] = S_idx[d.src0 + e / L];
-          st_w[i] = e_w[d.ent0 + e];
         }
       }
     } else {
