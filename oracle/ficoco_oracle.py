@@ -13,6 +13,7 @@ Each function names the passage of the paper it follows:
   * Eq. 2: self-preserving compression and the weights alpha_ij
   * Sec. "Task-Aware Improvements for FiCoCo-L": s^l and C^l
   * Algorithm 1 / Algorithm 2: order of the steps, output = X without the rows of S
+  * Appendix "Implementation of the Equivalent Token": a^Eq from the key states
 
 Readings taken where the paper is silent (all listed in the design notes):
   * the token-token relation A_{i,j} between two vision tokens is the cosine similarity
@@ -112,6 +113,25 @@ def vision_redundancy(R: np.ndarray) -> np.ndarray:
 def head_mean(attn: np.ndarray) -> np.ndarray:
     """Average a per-head quantity over heads (axis 0)."""
     return attn.astype(np.float64).sum(axis=0) / attn.shape[0]
+
+
+def equivalent_token(keys: np.ndarray, n_cls: int) -> np.ndarray:
+    """Appendix "Implementation of the Equivalent Token": the stand-in for the CLS attention
+    when the encoder has no CLS token.  keys: [T, H, d] key states of one image, token-major
+    (bf16 bit patterns or floats).  M = mean over the H heads; P = the patch rows of M (the
+    first n_cls rows are left out); mu = mean of P; a_i = -cos(mu, P_i).
+    Reading (the paper does not say): a zero mu or a zero P_i gives a_i = 0."""
+    K = widen(keys)
+    M = K.mean(axis=1)                       # [T, d]
+    P = M[n_cls:]
+    mu = P.mean(axis=0)
+    out = np.zeros(P.shape[0], dtype=np.float64)
+    n_mu = np.sqrt(np.dot(mu, mu))
+    for i in range(P.shape[0]):
+        n_i = np.sqrt(np.dot(P[i], P[i]))
+        if n_mu > 0.0 and n_i > 0.0:
+            out[i] = -np.dot(mu, P[i]) / (n_mu * n_i)
+    return out
 
 
 def score_v(v: np.ndarray, a_cls: np.ndarray, lam: float) -> np.ndarray:

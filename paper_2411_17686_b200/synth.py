@@ -242,6 +242,22 @@ def make_l_batch(seed: int, batch: int, n_vision: int, n_text: int, dim: int, he
     return LBatch(dtype, dim, heads, n_vision, n_text, toks, attn, [keep] * batch, name)
 
 
+def make_keys(seed: int, n_tokens: List[int], heads: int, head_dim: int, dtype: str = "bf16",
+              common: float = 0.5) -> List[np.ndarray]:
+    """Key states for the no-CLS equivalent token, one [T, H, d] array per image (token-major,
+    as a key projection writes them).  Every entry is N(0, 1) plus a per-image direction shared
+    by all tokens and heads (scale `common`), so that the cosines with the mean key spread over
+    a range instead of hovering around zero."""
+    out = []
+    for b, t in enumerate(n_tokens):
+        r = rng_for(seed, b, 7)
+        k = r.standard_normal((t, heads, head_dim))
+        shared = r.standard_normal(head_dim)
+        gain = r.uniform(0.0, 2.0, size=(t, 1, 1))          # how much of it each token carries
+        out.append(_store(k + common * gain * shared[None, None, :], dtype))
+    return out
+
+
 def regenerate_attention(batch: VBatch, seed: int, step: int, logit_std: float) -> None:
     """Replace the attention of every image by fresh per-head softmax weights over its
     currently alive patches (used between the steps of a progressive schedule)."""

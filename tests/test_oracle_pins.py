@@ -303,3 +303,66 @@ def test_edge_counts():
     assert r.out.shape[0] == 1 and np.array_equal(r.out[0], tok[0])
     r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 1, True)       # one target takes it all
     assert r.out.shape[0] == 2 and all(j.tolist() == [0] for j in r.J if j.size)
+
+
+# ---------------------------------------------------------------------------
+# equivalent token (appendix "Implementation of the Equivalent Token")
+# ---------------------------------------------------------------------------
+
+def _eq_token_loops(keys, n_cls):
+    """Scalar-loop transcription of the appendix equations (independent of the checker)."""
+    T, H, d = keys.shape
+    M = [[sum(float(keys[t, h, o]) for h in range(H)) / H for o in range(d)] for t in range(T)]
+    P = M[n_cls:]
+    mu = [sum(P[i][o] for i in range(len(P))) / len(P) for o in range(d)]
+    n_mu = sum(x * x for x in mu) ** 0.5
+    out = []
+    for row in P:
+        n_r = sum(x * x for x in row) ** 0.5
+        out.append(-sum(a * b for a, b in zip(mu, row)) / (n_mu * n_r))
+    return np.array(out)
+
+
+def test_equivalent_token_closed_forms():
+    # identical patch keys: every cosine with their mean is 1, so a = -1
+    k = np.tile(np.array([[[0.3, -1.2, 2.0]]], dtype=np.float32), (5, 2, 1))
+    np.testing.assert_allclose(fo.equivalent_token(k, 0), -1.0, atol=1e-12)
+    # two orthogonal patch keys of equal length: cos(mean, each) = 1/sqrt(2)
+    k = np.zeros((2, 1, 2), dtype=np.float32)
+    k[0, 0] = [2, 0]
+    k[1, 0] = [0, 2]
+    np.testing.assert_allclose(fo.equivalent_token(k, 0), -1.0 / np.sqrt(2.0), atol=1e-12)
+    # P = [3u, -u]: the mean is u, so the first token is aligned (a = -1), the second opposed (a = +1)
+    u = np.array([0.6, -0.8, 0.0], dtype=np.float32)
+    k = np.stack([3 * u, -u])[:, None, :]
+    np.testing.assert_allclose(fo.equivalent_token(k.astype(np.float32), 0), [-1.0, 1.0], atol=1e-7)
+    # a zero patch key (reading: a = 0) next to ordinary ones
+    k = np.array([[[0.0, 0.0]], [[1.0, 0.0]], [[1.0, 1.0]]], dtype=np.float32)
+    a = fo.equivalent_token(k, 0)
+    assert a[0] == 0.0 and a[1] < 0.0 and a[2] < 0.0
+
+
+def test_equivalent_token_invariants_and_loops():
+    keys = synth.make_keys(11, [9], 3, 5, "fp32")[0]
+    a = fo.equivalent_token(keys, 1)
+    assert a.shape == (8,) and np.all(np.abs(a) <= 1.0 + 1e-12)
+    np.testing.assert_allclose(a, _eq_token_loops(keys, 1), atol=1e-12)
+    # the CLS row takes no part; a common positive scale changes nothing
+    k2 = keys.copy()
+    k2[0] = 123.0
+    np.testing.assert_allclose(fo.equivalent_token(k2, 1), a, atol=1e-12)
+    np.testing.assert_allclose(fo.equivalent_token((4.0 * keys).astype(np.float32), 1), a, atol=1e-6)
+    # heads enter only through their mean: one head holding that mean gives the same result
+    m = keys.astype(np.float64).mean(axis=1, keepdims=True)
+    np.testing.assert_allclose(fo.equivalent_token(m.astype(np.float32), 1), a, atol=1e-6)
+    # without the CLS exclusion the first row would be scored too
+    assert fo.equivalent_token(keys, 0).shape == (9,)
+    # a planted mistake (mean taken over all rows, CLS included) must not survive the loops pin
+    M = keys.astype(np.float64).mean(axis=1)
+    mu_wrong = M.mean(axis=0)
+    wrong = -(M[1:] @ mu_wrong) / (np.linalg.norm(M[1:], axis=1) * np.linalg.norm(mu_wrong))
+    assert np.max(np.abs(wrong - _eq_token_loops(keys, 1))) > 1e-3
+    # bf16 storage is widened exactly
+    kb = synth.make_keys(12, [6], 2, 4, "bf16")[0]
+    kf = synth.bf16_bits_to_f32(kb)
+    np.testing.assert_allclose(fo.equivalent_token(kb, 0), fo.equivalent_token(kf, 0), atol=0)
