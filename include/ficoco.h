@@ -225,6 +225,26 @@ int ficoco_profile_read(ficoco_ctx* ctx, int index, char* name, int name_cap, do
                         long long* launches);
 
 /*
+ * Equivalent token for encoders without a CLS token (appendix "Implementation of the Equivalent
+ * Token"): M = mean of the key states over the heads, mu = mean of M over the image's patch
+ * tokens, a_i = -cos(mu, M_i) for every patch token i.  The result stands in for the CLS
+ * attention of Eq. 1: pass it to ficoco_v_reduce as `attn` with heads = 1.
+ *
+ * keys: device, token-major [rows, heads, head_dim] (the layout a key projection writes: one
+ * contiguous row of heads * head_dim elements per token), fp32 or bf16, images packed one after
+ * the other like `tokens`; a row must be a multiple of 16 bytes.  seqlens: host int32[batch]
+ * rows per image (CLS row included when has_cls != 0), or NULL when every image has n_tokens
+ * rows.  a_eq: device fp32, one value per patch token, packed in the same order (CLS rows left
+ * out).  A patch key or a mean of zero length gives 0.
+ * One thread-block cluster of 8 CTAs works on an image and keeps the head-mean keys of its
+ * tokens in shared memory, which bounds an image at 8 * floor(200 KB / (4 * head_dim)) patch
+ * tokens (6400 at head_dim 64); more returns FICOCO_ERR_UNSUPPORTED.  Nothing is allocated and
+ * no context is needed; work is enqueued on cuda_stream and the call does not synchronise.
+ */
+int ficoco_equivalent_token(const void* keys, int dtype, int batch, int n_tokens, const int* seqlens,
+                            int heads, int head_dim, int has_cls, float* a_eq, void* cuda_stream);
+
+/*
  * Allocation-free vision-aware redundancy.  (The paper has no counterpart to this entry
  * point: it exists for callers of this library that are not allowed to allocate.)
  *

@@ -32,6 +32,7 @@ EXPORTS = [
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
     "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
+    "ficoco_equivalent_token",
 ]
 
 
@@ -83,6 +84,8 @@ def load_library() -> C.CDLL:
     lib.ficoco_last_cuda_error.argtypes = [C.c_void_p]
     lib.ficoco_default_params.argtypes = [C.POINTER(ficoco_params)]
     lib.ficoco_default_params.restype = None
+    lib.ficoco_equivalent_token.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int,
+                                            C.c_int, C.c_int, C.c_void_p, C.c_void_p]
     lib.ficoco_v_reduce.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_l_reduce.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_v_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params)]
@@ -356,6 +359,34 @@ def ficoco_vision_redundancy_noalloc(tokens, n_tokens: int, has_cls: bool = True
                                               v_out.data_ptr(), C.c_void_p(stream))
     _check(None, rc)
     return v_out
+
+
+def ficoco_equivalent_token(keys, heads: int, head_dim: int, *, n_tokens: int = 0, seqlens=None,
+                            has_cls: bool = False, a_eq=None, stream: Optional[int] = None):
+    """a^Eq of the no-CLS variant.  ``keys``: cuda tensor [rows, heads * head_dim] (token-major
+    key states, images packed); ``seqlens``: rows per image, or None with ``n_tokens`` given.
+    Returns the cuda fp32 tensor of one value per patch token (allocated with torch when
+    ``a_eq`` is not passed); use it as ``attn`` with ``heads = 1`` in ficoco_v_reduce."""
+    import torch
+    lib = load_library()
+    cls = 1 if has_cls else 0
+    if seqlens is not None:
+        sl, batch = _int_array(seqlens)
+        patches = int(sl.sum()) - cls * batch
+        sl_ptr = sl.ctypes.data
+    else:
+        sl, batch = None, keys.shape[0] // n_tokens
+        patches = batch * (n_tokens - cls)
+        sl_ptr = None
+    if a_eq is None:
+        a_eq = torch.empty((patches,), dtype=torch.float32, device=keys.device)
+    if stream is None:
+        stream = torch.cuda.current_stream(keys.device).cuda_stream
+    rc = lib.ficoco_equivalent_token(C.c_void_p(keys.data_ptr()), _dtype_code(keys), batch, n_tokens,
+                                     C.c_void_p(sl_ptr), heads, head_dim, cls, C.c_void_p(a_eq.data_ptr()),
+                                     C.c_void_p(stream))
+    _check(None, rc)
+    return a_eq
 
 
 # ----------------------------------------------------------------------------------------

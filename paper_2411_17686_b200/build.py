@@ -9,7 +9,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libficoco.so")
-SOURCES = ["ficoco.cu", "noalloc.cu"]
+SOURCES = ["ficoco.cu", "noalloc.cu", "equivalent_token.cu"]
 
 
 def _nvcc() -> str:

@@ -25,7 +25,6 @@ constexpr int N_PLANS = 8;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
 constexpr int OUT_ROWS_PER_CTA = 16;  // <= MROWS of the merge kernel
 constexpr int NSPLIT_MAX = 16;
-constexpr int TARGET_CTAS = 2 * 148;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -119,7 +119,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   for (int i = 0; i < 4; ++i) st_row[i] = -1;
   if (tp_hi > tp_lo) {
     if (one_pass) {
-#pragma unroll
       int t4[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
