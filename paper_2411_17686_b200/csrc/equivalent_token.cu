@@ -4,7 +4,7 @@
 //
 // One thread-block cluster of 8 CTAs per image.  CTA r owns a contiguous eighth of the image's
 // patch tokens; their key rows are contiguous in memory (token-major layout), so one producer
-// lane streams them with 16-row bulk copies (TMA) through an mbarrier ring while 8 consumer
+// lane streams them with 8-row bulk copies (TMA) through an mbarrier ring while 8 consumer
 // warps reduce each row over its heads.  The head-mean keys stay in shared memory, so the keys
 // are read from HBM exactly once; the only exchange between the CTAs of an image is their
 // partial column sums (head_dim floats each), read from the peers' shared memory between two
@@ -28,12 +28,12 @@ using namespace ficoco;
 namespace {
 
 constexpr int EQ_CLUSTER = 8;          // CTAs per image
-constexpr int EQ_ROWS = 16;            // key rows per ring stage (two per consumer warp)
+constexpr int EQ_ROWS = 8;             // key rows per ring stage (one per consumer warp)
 constexpr int EQ_WARPS = 8;            // consumer warps
 constexpr int EQ_THREADS = 32 * (EQ_WARPS + 1);
-constexpr int EQ_MAX_STAGE = 4;
+constexpr int EQ_MAX_STAGE = 6;
 constexpr int EQ_MAX_BATCH_RAGGED = 256;
-constexpr int EQ_MAX_HEAD_DIM = 256;   // eight columns per lane
+constexpr int EQ_MAX_HEAD_DIM = 256;   // four pairs of columns per lane
 constexpr size_t EQ_SMEM_LIMIT = 220 * 1024;
 
 // first row of every image of a ragged batch (kernel parameter space; no device allocation)
@@ -41,9 +41,11 @@ struct EqOffsets {
   int row0[EQ_MAX_BATCH_RAGGED + 1];
 };
 
-__device__ __forceinline__ float load_key(const float* p) { return *p; }
-__device__ __forceinline__ float load_key(const __nv_bfloat16* p) {
-  return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short*>(p)) << 16);
+// two adjacent columns of one head
+__device__ __forceinline__ float2 load_key2(const float* p) { return *reinterpret_cast<const float2*>(p); }
+__device__ __forceinline__ float2 load_key2(const __nv_bfloat16* p) {
+  const uint32_t u = *reinterpret_cast<const uint32_t*>(p);
+  return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
 }
 
 // Dynamic shared memory: ring [nstage][EQ_ROWS][heads * dk] of T | Ms [tpc_max][dk] |
@@ -88,7 +90,7 @@ __global__ void __launch_bounds__(EQ_THREADS, 2) k_equivalent_token(
 
   const int ngroups = (nt + EQ_ROWS - 1) / EQ_ROWS;
   if (warp == EQ_WARPS) {
-    // ---------------- producer: 16-row bulk copies into the ring -------------------------------
+    // ---------------- producer: bulk copies of EQ_ROWS rows into the ring -------------------------------
     if (lane == 0) {
       const unsigned char* base =
           reinterpret_cast<const unsigned char*>(keys + (size_t)(row0 + n_cls + t_lo) * row_elems);
@@ -121,15 +123,28 @@ __global__ void __launch_bounds__(EQ_THREADS, 2) k_equivalent_token(
           const T* rp = reinterpret_cast<const T*>(ring + (size_t)s * stage_bytes + (size_t)rr * row_bytes);
           float ss = 0.f;
 #pragma unroll
-          for (int j = 0; j < EQ_MAX_HEAD_DIM / 32; ++j) {
-            const int o = lane + 32 * j;
+          for (int j = 0; j < EQ_MAX_HEAD_DIM / 64; ++j) {
+            const int o = 2 * (lane + 32 * j);           // this lane's pair of columns
             if (o < dk) {
-              float m = 0.f;
-              for (int h = 0; h < heads; ++h) m += load_key(rp + h * dk + o);
-              m *= inv_h;
-              Ms[(size_t)t * dk + o] = m;
-              col[j] += m;
-              ss = fmaf(m, m, ss);
+              // four running sums, so that the loads of four heads are in flight together
+              float2 m0 = make_float2(0.f, 0.f), m1 = m0, m2 = m0, m3 = m0;
+              int h = 0;
+              for (; h + 4 <= heads; h += 4) {
+                const float2 k0 = load_key2(rp + (h + 0) * dk + o), k1 = load_key2(rp + (h + 1) * dk + o);
+                const float2 k2 = load_key2(rp + (h + 2) * dk + o), k3 = load_key2(rp + (h + 3) * dk + o);
+                m0.x += k0.x; m0.y += k0.y; m1.x += k1.x; m1.y += k1.y;
+                m2.x += k2.x; m2.y += k2.y; m3.x += k3.x; m3.y += k3.y;
+              }
+              for (; h < heads; ++h) {
+                const float2 k0 = load_key2(rp + h * dk + o);
+                m0.x += k0.x; m0.y += k0.y;
+              }
+              const float mx = ((m0.x + m1.x) + (m2.x + m3.x)) * inv_h;
+              const float my = ((m0.y + m1.y) + (m2.y + m3.y)) * inv_h;
+              *reinterpret_cast<float2*>(Ms + (size_t)t * dk + o) = make_float2(mx, my);
+              col[2 * j] += mx;
+              col[2 * j + 1] += my;
+              ss = fmaf(mx, mx, fmaf(my, my, ss));
             }
           }
           ss = warp_sum(ss);
@@ -141,9 +156,9 @@ __global__ void __launch_bounds__(EQ_THREADS, 2) k_equivalent_token(
     }
     if (!ok) failed = 1;
 #pragma unroll
-    for (int j = 0; j < EQ_MAX_HEAD_DIM / 32; ++j) {
-      const int o = lane + 32 * j;
-      if (o < dk) csum[warp * dk + o] = col[j];
+    for (int j = 0; j < EQ_MAX_HEAD_DIM / 64; ++j) {
+      const int o = 2 * (lane + 32 * j);
+      if (o < dk) { csum[warp * dk + o] = col[2 * j]; csum[warp * dk + o + 1] = col[2 * j + 1]; }
     }
   }
   __syncthreads();
@@ -215,7 +230,7 @@ extern "C" int ficoco_equivalent_token(const void* keys, int dtype, int batch, i
   const size_t es = dtype == FICOCO_BF16 ? 2 : 4;
   const size_t row_bytes = (size_t)heads * head_dim * es;
   if (row_bytes % 16 != 0 || ((uintptr_t)keys & 15) != 0) return FICOCO_ERR_INVALID_ARG;
-  if (head_dim > EQ_MAX_HEAD_DIM) return FICOCO_ERR_UNSUPPORTED;
+  if (head_dim > EQ_MAX_HEAD_DIM || head_dim % 2 != 0) return FICOCO_ERR_UNSUPPORTED;
   EqOffsets offs;
   offs.row0[0] = 0;
   int max_np = 0;
