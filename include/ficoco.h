@@ -237,9 +237,12 @@ int ficoco_profile_read(ficoco_ctx* ctx, int index, char* name, int name_cap, do
  * rows.  a_eq: device fp32, one value per patch token, packed in the same order (CLS rows left
  * out).  A patch key or a mean of zero length gives 0.
  * One thread-block cluster of 8 CTAs works on an image and keeps the head-mean keys of its
- * tokens in shared memory, which bounds an image at 8 * floor(200 KB / (4 * head_dim)) patch
- * tokens (6400 at head_dim 64); more returns FICOCO_ERR_UNSUPPORTED.  Nothing is allocated and
- * no context is needed; work is enqueued on cuda_stream and the call does not synchronise.
+ * tokens in shared memory: an eighth of the image's patch tokens times 4 * head_dim bytes, plus
+ * two staging buffers of 8 key rows, must fit in 220 KB (about 5000 patch tokens per image at
+ * 16 heads of 64 bf16); a longer image, head_dim > 256 or odd, or a ragged batch of more than
+ * 256 images returns FICOCO_ERR_UNSUPPORTED.  Nothing is allocated and no context is needed;
+ * work is enqueued on cuda_stream and the call does not synchronise.  Should a bounded
+ * device-side wait run out, the affected tokens read NaN.
  */
 int ficoco_equivalent_token(const void* keys, int dtype, int batch, int n_tokens, const int* seqlens,
                             int heads, int head_dim, int has_cls, float* a_eq, void* cuda_stream);
