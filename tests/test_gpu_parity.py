@@ -200,6 +200,25 @@ def test_host_entry_point_in_image_groups(ctx, idx):
     assert ctx.ficoco_status() == 0
 
 
+def test_pairwise_correlation_gap_from_inspection(ctx):
+    """The paper's diagnostic for choosing K (Sec. "Correlation-based Information Recycling"):
+    top-1 minus top-2 correlation of every discarded token.  With the adaptive threshold the
+    library keeps each row's two (or more) largest correlations, so the gap can be read from
+    the inspection arrays; it must match the checker's full correlation rows."""
+    batch = synth.workload(2, small=True)
+    gaps.repair_v(batch)
+    p = fo.Params()
+    _, results = parity.run_and_compare_v(ctx, batch, p, DEV, what="gap")
+    cc = ctx.ficoco_inspect("corr_c")
+    s0 = 0
+    for r in results:
+        order = np.argsort(r.S)
+        for k, si in enumerate(order):
+            row = np.sort(r.C[si])[::-1]
+            np.testing.assert_allclose(cc[s0 + k, 0] - cc[s0 + k, 1], row[0] - row[1], rtol=0, atol=3e-5)
+        s0 += r.S.shape[0]
+
+
 def test_canaries_around_outputs(ctx):
     """Nothing is written outside the documented output extents."""
     batch = synth.workload(4, small=True)
