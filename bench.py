@@ -132,6 +132,92 @@ def make_instances(rank: int):
     return batch
 
 
+def other_workloads(binding, packing, ctx, insts, prm, stream, dev) -> dict:
+    """Device times of the other configurations (not the headline metric): the whole progressive
+    schedule of the headline batch (576 -> 288 -> 144 -> 64, every step fed from the one before,
+    one CUDA graph over the 8 buffer sets) and one reduce step of the other four workloads
+    (their inputs are reused every step, so the smaller ones are L2-warm)."""
+    import torch
+    from paper_2411_17686_b200 import synth
+    out = {}
+    n = 1 + GH * GW
+    k2, k3 = KEEP // 2, 64
+    g = torch.Generator().manual_seed(7)
+    attn2 = torch.softmax(1.5 * torch.randn(B, H, KEEP, generator=g), -1).reshape(-1).to(dev)
+    attn3 = torch.softmax(1.5 * torch.randn(B, H, k2, generator=g), -1).reshape(-1).to(dev)
+    o2 = torch.empty((B * (1 + k2), D), dtype=torch.bfloat16, device=dev)
+    o3 = torch.empty((B * (1 + k3), D), dtype=torch.bfloat16, device=dev)
+    i2 = torch.empty((B * (1 + k2),), dtype=torch.int32, device=dev)
+    i3 = torch.empty((B * (1 + k3),), dtype=torch.int32, device=dev)
+    p2 = torch.empty((B * k2,), dtype=torch.int32, device=dev)
+    p3 = torch.empty((B * k3,), dtype=torch.int32, device=dev)
+
+    def chain(i):
+        it = insts[i % N_INSTANCES]
+        s = stream.cuda_stream
+        ctx.ficoco_v_reduce(it["tokens"], it["attn"], KEEP, GH, GW, H, n_tokens=n, pos=it["pos"], params=prm,
+                            out_tokens=it["out"], kept_idx=it["kidx"], pos_out=it["pout"], stream=s)
+        ctx.ficoco_v_reduce(it["out"], attn2, k2, GH, GW, H, n_tokens=1 + KEEP, pos=it["pout"], params=prm,
+                            out_tokens=o2, kept_idx=i2, pos_out=p2, stream=s)
+        ctx.ficoco_v_reduce(o2, attn3, k3, GH, GW, H, n_tokens=1 + k2, pos=p2, params=prm,
+                            out_tokens=o3, kept_idx=i3, pos_out=p3, stream=s)
+
+    with torch.cuda.stream(stream):
+        chain(0)
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr, stream=stream):
+        for i in range(N_INSTANCES):
+            chain(i)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        gr.replay()
+        e0.record(stream)
+        for _ in range(5):
+            gr.replay()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (5 * N_INSTANCES)
+    out["c2 schedule 576->288->144->64"] = {"us_per_schedule": us, "images_per_s": B / (us * 1e-6)}
+
+    for idx, label in ((1, "c1: 1 x 577 x 1024 fp32, discard 64"), (3, "c3 step 1: 8 x 2881 x 1024 bf16, 2880 -> 1440"),
+                       (4, "c4: 16 ragged images x 1280 bf16, keep 1/9"), (5, "c5: FiCoCo-L 16 x (576+64) x 4096 bf16, 576 -> 64")):
+        wl = synth.workload(idx)
+        rows = sum(int(t.shape[0]) for t in wl.tokens)
+        c2 = binding.Context(max_tokens=rows, max_dim=wl.dim, max_batch=len(wl.tokens),
+                             max_text=getattr(wl, "n_text", 0), device=torch.device(dev).index)
+        try:
+            if idx == 5:
+                pk = packing.pack_l(wl, dev)
+                pp = binding.make_params(has_cls=False)
+                res = c2.ficoco_l_reduce(pk.tokens, pk.attn_t2v, pk.keep, pk.n_vision, pk.n_text, pk.heads, params=pp,
+                                         stream=stream.cuda_stream)
+                step = lambda: c2.ficoco_l_reduce(pk.tokens, pk.attn_t2v, pk.keep, pk.n_vision, pk.n_text, pk.heads,
+                                                  params=pp, out_tokens=res.out_tokens, kept_idx=res.kept_idx,
+                                                  stream=stream.cuda_stream)
+            else:
+                pk = packing.pack_v(wl, dev)
+                pp = binding.make_params(has_cls=wl.has_cls)
+                res = c2.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=pp,
+                                         stream=stream.cuda_stream, **pk.call_kwargs())
+                step = lambda: c2.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads,
+                                                  params=pp, out_tokens=res.out_tokens, kept_idx=res.kept_idx,
+                                                  pos_out=res.pos_out, stream=stream.cuda_stream, **pk.call_kwargs())
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    step()
+                e0.record(stream)
+                for _ in range(20):
+                    step()
+                e1.record(stream)
+            torch.cuda.synchronize()
+            assert c2.ficoco_status(stream.cuda_stream) == 0
+            out[label] = {"us_per_step": e0.elapsed_time(e1) * 1e3 / 20, "images": len(wl.tokens), "token_rows": rows}
+        finally:
+            c2.close()
+    return out
+
+
 def run_ours(args, rank: int, world: int, local_rank: int):
     import torch
     from paper_2411_17686_b200 import binding, build, packing
@@ -257,6 +343,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                "workload": "32 x 577 tokens x 16 heads x 64 bf16 keys, 4 buffers cycled"}
     del eq_keys
 
+    extras = other_workloads(binding, packing, ctx, insts, prm, stream, dev) if args.extras else None
+
     # end to end through the host-buffer entry point (pinned host tensors, copies inside)
     hp = packing.pack_v(batch, None, pin=True)
     out_h = torch.empty((B * (1 + KEEP), D), dtype=torch.bfloat16).pin_memory()
@@ -283,6 +371,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "tokens_per_s": value * n,
         "clocks": clocks,
         "equivalent_token": eq_info,
+        "other_workloads": extras,
         "e2e": {"value": world * B / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps},
         "gpu_launches": launches_per_step * args.steps,
@@ -396,6 +485,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", dest="graph", action="store_false")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
+    ap.add_argument("--no-extras", dest="extras", action="store_false",
+                    help="skip the schedule / other-workload timings that follow the headline measurement")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
