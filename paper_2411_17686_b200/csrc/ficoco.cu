@@ -447,7 +447,10 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
   p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = p->max_list = 0;
   p->need_finalize = false;
-  p->umma = key.mode == 0 && key.dtype == FICOCO_BF16 && key.dim % UKB == 0;
+  // tensor-core correlate: bf16 tokens, hidden size a multiple of 64.  FiCoCo-L adds its text term
+  // in the epilogue from weights staged in shared memory, 2 KB per text token for the largest tile.
+  p->umma = key.dtype == FICOCO_BF16 && key.dim % UKB == 0 &&
+            (key.mode == 0 || (size_t)key.n_text * 2048 + 1024 + (size_t)UM * KCAP * 8 <= 220 * 1024);
   int tile_rows_max = p->umma ? UM : CBM;             // source rows per correlate CTA (decided below)
   const int col_granule = p->umma ? 16 : CBN;
   int um_a_rows = 8, um_cols = 16;
@@ -685,8 +688,12 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       if (ns != 5 && (size_t)ns * p->um_stage_bytes + slack <= 220 * 1024) p->um_nstage = ns;
     if (!p->um_nstage) return FICOCO_ERR_UNSUPPORTED;
     p->um_smem = (size_t)p->um_nstage * p->um_stage_bytes + slack;
-    // the epilogue helpers hand their lists back through the ring
-    if (p->um_smem < 1024 + (size_t)UM * KCAP * 8) p->um_smem = 1024 + (size_t)UM * KCAP * 8;
+    // the epilogue halves hand their lists over through the ring; FiCoCo-L also stages the head-mean
+    // text->vision weights of a tile's rows and columns there
+    size_t epi = 1024 + (size_t)UM * KCAP * 8;
+    if (key.mode == 1) epi += (size_t)key.n_text * ((size_t)n_sub * UM + (size_t)((um_cols + 15) / 16 * 16)) * 4;
+    if (p->um_smem < epi) p->um_smem = epi;
+    if (p->um_smem > 220 * 1024) return FICOCO_ERR_UNSUPPORTED;
   }
 
   char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
@@ -857,7 +864,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   c->launches += 2;
   }
   if (p->n_corr > 0) {
-    if (p->umma && tmean == nullptr && sizeof(T) == 2) {
+    if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
@@ -865,7 +872,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
       (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
       p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-      c->e_w, c->e_c)
+      c->e_w, c->e_c, tmean, M, p->max_np, gamma)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 6) FICOCO_UMMA_LAUNCH(6, LC);                                                  \

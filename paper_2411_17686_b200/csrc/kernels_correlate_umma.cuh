@@ -98,10 +98,14 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
 // once a value is placed the rest of the list shifts down; '>' keeps the lower column first
 // among equal values because columns arrive in ascending order.
 // v / ix: descending list, -inf / INT_MAX in empty slots.  Warp-collective (tcgen05.ld).
+// FiCoCo-L adds the text-bridged term: tS (this row's text->vision weights, element k at
+// tS[k * s_stride]) and tT ([M][t_stride], one row per text token over the CTA's columns) sit in
+// shared memory; C = gamma * cosine + t_scale * sum_k tS_k tT_kc.  tT == nullptr: FiCoCo-V.
 template <int LCAP>
 __device__ __forceinline__ void epilogue_scan(uint32_t tmem_lane, int c_lo, int c_hi, int ncols, int col_begin,
                                               float rs, const float* rnT, bool row_valid, int L,
-                                              float (&v)[LCAP], int (&ix)[LCAP]) {
+                                              float (&v)[LCAP], int (&ix)[LCAP], const float* tS, int s_stride,
+                                              const float* tT, int t_stride, int M, float gamma, float t_scale) {
 #pragma unroll
   for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
   const int cmax = row_valid ? min(ncols, c_hi) : 0;
@@ -109,11 +113,29 @@ __device__ __forceinline__ void epilogue_scan(uint32_t tmem_lane, int c_lo, int 
   for (int c0 = c_lo; c0 < c_hi; c0 += 16) {
     uint32_t r[16];
     tmem_ld16_issue(tmem_lane + (uint32_t)c0, r);
+    float tx[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) tx[j] = 0.f;
+    if (tT != nullptr) {
+      #pragma unroll 1
+      for (int k = 0; k < M; ++k) {
+        const float a = tS[(size_t)k * s_stride];
+        const float4* q = reinterpret_cast<const float4*>(tT + (size_t)k * t_stride + c0);
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4) {
+          const float4 t4 = q[j4];
+          tx[4 * j4 + 0] = fmaf(a, t4.x, tx[4 * j4 + 0]);
+          tx[4 * j4 + 1] = fmaf(a, t4.y, tx[4 * j4 + 1]);
+          tx[4 * j4 + 2] = fmaf(a, t4.z, tx[4 * j4 + 2]);
+          tx[4 * j4 + 3] = fmaf(a, t4.w, tx[4 * j4 + 3]);
+        }
+      }
+    }
     tmem_ld_wait();
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
       const int c = c0 + j;
-      float cv = (rs * rnT[c]) * __uint_as_float(r[j]);
+      float cv = gamma * ((rs * rnT[c]) * __uint_as_float(r[j])) + t_scale * tx[j];
       if (!(c < cmax)) cv = -CUDART_INF_F;           // also drops NaN-free padding columns
       int ci = col_begin + c;
       bool ins = false;
@@ -145,7 +167,8 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
     int stage_bytes, int a_bytes, int tmem_cols, int* __restrict__ img_done, int* __restrict__ corr_cnt,
-    float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
+    float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
+    const float* __restrict__ tmean, int M, int NV, float gamma) {
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
@@ -254,6 +277,26 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
     tc_fence_after();
+    // FiCoCo-L: the head-mean text->vision weights of this tile's columns and rows go into the idle
+    // ring, behind the area the two epilogue halves use to hand over their lists
+    const int rows_pad = nsub * UM;
+    float* tT = nullptr;
+    float* tSb = nullptr;
+    const float t_scale = tmean != nullptr ? (1.0f - gamma) / (float)M : 0.f;
+    if (tmean != nullptr) {
+      tT = reinterpret_cast<float*>(um_raw + (ring - smem_u32(um_raw)) + (size_t)UM * LCAP * 8);
+      tSb = tT + (size_t)M * n_pad;
+      const float* tb = tmean + (size_t)w.img * M * NV;
+      for (int i = pt; i < M * n_pad; i += 256) {
+        const int k = i / n_pad, cc = i - k * n_pad;
+        tT[i] = cc < ncols ? __ldg(tb + (size_t)k * NV + rowT[cc]) : 0.f;
+      }
+      for (int i = pt; i < M * rows_pad; i += 256) {
+        const int k = i / rows_pad, rr = i - k * rows_pad;
+        tSb[i] = rr < w.nrows ? __ldg(tb + (size_t)k * NV + rowS[rr]) : 0.f;
+      }
+      cta_sync(1, 256);
+    }
     if (warp < 4) {
     // ---------------- epilogue: lane = accumulator row ---------------------------------------
     // this warp scans the lower half of the columns, its helper warp (same TMEM lanes) the
@@ -268,7 +311,8 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       int ix[LCAP];
       if (acc_ok && sub * UM + warp * 32 < w.nrows)
         epilogue_scan<LCAP>(tmem_base + (uint32_t)(sub * n_pad) + ((uint32_t)(warp * 32) << 16), 0, c_mid, ncols,
-                            col_begin, rs, rnT, row_valid, L, v, ix);
+                            col_begin, rs, rnT, row_valid, L, v, ix, tSb + row, rows_pad, tT, n_pad, M, gamma,
+                            t_scale);
       else {
 #pragma unroll
         for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
@@ -323,7 +367,8 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       int ix[LCAP];
       if (acc_ok && sub * UM + grp * 32 < w.nrows)
         epilogue_scan<LCAP>(tmem_base + (uint32_t)(sub * n_pad) + ((uint32_t)(grp * 32) << 16), c_mid, n_pad, ncols,
-                            col_begin, rs, rnT, row_valid, L, v, ix);
+                            col_begin, rs, rnT, row_valid, L, v, ix, tSb + row, rows_pad, tT, n_pad, M, gamma,
+                            t_scale);
       else {
 #pragma unroll
         for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
