@@ -1,4 +1,5 @@
-// Correlate stage on the 5th-generation tensor cores (bf16 tokens).
+// Correlate stage on the 5th-generation tensor cores (bf16 tokens; FiCoCo-V, and FiCoCo-L with its
+// text-bridged term added in the epilogue).
 //
 // One CTA owns a tile of discarded tokens (rows of the accumulator, one TMEM lane each) and
 // one column split (<= 256 preserved tokens) of one image.  A tile has up to 128 rows, or up
