@@ -46,6 +46,17 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Counter updates that publish (release) and, for the second one, also observe (acquire) at GPU
+// scope in one round trip.  Called by one thread after a CTA barrier: the barrier orders the other
+// threads' stores before it, and the release makes them visible with the count.
+__device__ __forceinline__ void red_release_add(int* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int atom_acq_rel_add(int* p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Arrive on `bar` and announce `bytes` of bulk-copy traffic that will complete on it.

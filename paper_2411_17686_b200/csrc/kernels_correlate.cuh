@@ -2,6 +2,7 @@
 #pragma once
 #include <limits.h>
 #include <math_constants.h>
+#include "async_ops.cuh"
 #include "common.cuh"
 
 namespace ficoco {
@@ -299,12 +300,12 @@ __device__ __forceinline__ void correlate_tail(
     const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
     int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem) {
-  __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int old = atomicAdd(&tile_done[tile], 1);
+    // publishes this CTA's partial lists and, for the split that arrives last, observes the others'
+    const int old = atom_acq_rel_add(&tile_done[tile], 1);
     const int last = old == d.nsplit - 1;
-    if (last) { __threadfence(); tile_done[tile] = 0; }
+    if (last) tile_done[tile] = 0;
     *is_last_smem = last;
   }
   __syncthreads();

@@ -230,10 +230,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       pout[c] = t;
     }
     cta_sync(1, F_NCONS);
-    if (tid == 0) {          // the barrier orders the CTA's stores before this one fence (cumulative)
-      __threadfence();
-      atomicAdd(&cnt[w.img], 1);
-    }
+    if (tid == 0) red_release_add(&cnt[w.img], 1);   // pairs with the ld.acquire poll of pass 2
   }
   if (!ok && lane == 0) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
 
@@ -339,10 +336,9 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     }
     cta_sync(1, F_NCONS);
     if (tid == 0) {
-      __threadfence();
-      const int old = atomicAdd(&cnt[B + w.img], 1);
+      // release this piece's scores, and (for the CTA that arrives last) acquire everyone else's
+      const int old = atom_acq_rel_add(&cnt[B + w.img], 1);
       if (old == d.n_chunks - 1 && nwon < F_MAXWON) won[nwon++] = w.img;
-      __threadfence();
     }
   }
   cta_sync(1, F_NCONS);
