@@ -15,7 +15,7 @@ Each function names the passage of the paper it follows:
   * Algorithm 1 / Algorithm 2: order of the steps, output = X without the rows of S
   * Appendix "Implementation of the Equivalent Token": a^Eq from the key states
 
-Readings taken where the paper is silent (all listed in the design notes):
+Readings taken where the paper is silent:
   * the token-token relation A_{i,j} between two vision tokens is the cosine similarity
     R = X_hat X_hat^T of the layer's hidden states (the paper itself uses cosine
     similarity in place of attention for encoders without CLS, Appendix
