@@ -10,15 +10,6 @@ constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shar
 constexpr int MHEAVY = 4;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
-__device__ __forceinline__ void prefetch_l1(const void* p) {
-  asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
-}
-// Lanes of a warp touch every 128-byte line of one token row.
-__device__ __forceinline__ void prefetch_row(const void* row, int row_bytes, int lane) {
-  for (int o = lane * 128; o < row_bytes; o += 32 * 128)
-    prefetch_l1(reinterpret_cast<const unsigned char*>(row) + o);
-}
-
 // acc[b][.] += sum over list entries [k0, k1) of alpha * x, for the MVB vectors v0 + 32 b of
 // each row; source rows are fetched four at a time so that 4 * MVB loads are in flight per lane.
 template <class T>
@@ -55,10 +46,11 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
 
 // Compress + compact.  No per-target lists are built in global memory.  A CTA owns up to 32
 // consecutive output rows of one image (warp w: rows w, w + 8, w + 16, w + 24).
-//   1. every warp resolves the input row of its output rows and prefetches those rows into L1;
+//   1. every warp resolves the input row of its output rows (L1 prefetches of the rows were tried:
+//      they never produced L1 hits and cost 1.7 us per step, so there are none);
 //   2. meanwhile the CTA scans the image's (source -> target) entries twice (count, then fill)
 //      to file those that hit its rows into per-row lists in shared memory (token index,
-//      alpha), prefetching the source rows, and orders every list by token index so that the
+//      alpha), and orders every list by token index so that the
 //      fp32 sums have one fixed order and no atomics touch floats;
 //   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
 //      rows with few sources by their own warp; hub rows are cut into blocks of 32 vectors that
@@ -82,7 +74,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = D / E;
-  const int row_bytes = D * (int)sizeof(T);
   const int L = d.list_len;
   const int tp_lo = max(w.r0 - d.n_cls, 0);
   const int tp_hi = min(w.r0 + w.nrows - d.n_cls, d.n_tgt);
@@ -92,10 +83,10 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
   if (tid == 0) n_heavy = 0;
   // When the grid before this one is a correlate grid, the filter grid (which wrote T_idx) had
-  // completed before this grid could start, so the row lookup and prefetch may overlap that
+  // completed before this grid could start, so the row lookup may overlap that
   // grid's tail; otherwise wait first.
   if (!index_before_wait) grid_dep_wait();
-  // input row of every output row (CLS / preserved token / trailing text row), prefetched
+  // input row of every output row (CLS / preserved token / trailing text row)
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
     const int orow = w.r0 + r;
@@ -104,7 +95,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
     else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
     if (lane == 0) srow_s[r] = srow;
-    prefetch_row(tokens + (size_t)(d.row0 + srow) * D, row_bytes, lane);
   }
   if (index_before_wait) grid_dep_wait();
   grid_dep_launch();   // correlate is complete: the next step's filter may stream its rows under our tail
@@ -170,8 +160,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
           const int slot = beg[st_row[i]] + st_slot[i];
           tsrc[slot] = st_src[i];
           tw[slot] = st_w[i];
-          const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)st_src[i] * D);
-          for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
         }
     } else {
       for (int e = tid; e < n_ent; e += 256) {
@@ -181,8 +169,6 @@ __global__ void __launch_bounds__(256) k_merge_scan(
           const int si = S_idx[d.src0 + e / L];
           tsrc[slot] = si;
           tw[slot] = e_w[d.ent0 + e];
-          const unsigned char* xr = reinterpret_cast<const unsigned char*>(pbase + (size_t)si * D);
-          for (int o = 0; o < row_bytes; o += 128) prefetch_l1(xr + o);
         }
       }
     }
