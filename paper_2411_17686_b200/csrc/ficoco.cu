@@ -23,7 +23,7 @@ namespace {
 
 constexpr int N_PLANS = 8;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
-constexpr int OUT_ROWS_PER_CTA = 16;  // <= MROWS of the merge kernel
+constexpr int OUT_ROWS_PER_CTA = MROWS_CTA;  // the merge kernel's copy batches are sized for it
 constexpr int NSPLIT_MAX = 16;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -5,7 +5,9 @@
 namespace ficoco {
 
 constexpr int MHUB = 8;        // source rows a lane has in flight for a hub row
-constexpr int MROWS = 32;      // output rows per CTA (four per warp)
+constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the per-row arrays)
+constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
+constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
 constexpr int MHEAVY = 4;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
@@ -189,9 +191,9 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
   #pragma unroll 1
   for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
-    uint4 u[4][MVB];
+    uint4 u[MCOPY][MVB];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < MCOPY; ++j) {
       const int r = warp + 8 * j;
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       }
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < MCOPY; ++j) {
       const int r = warp + 8 * j;
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
