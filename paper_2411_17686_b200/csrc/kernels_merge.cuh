@@ -9,7 +9,7 @@ constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the 
 constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
 constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
-constexpr int MHEAVY = 4;      // rows with more sources than this are split into 32-vector blocks over the warps
+constexpr int MHEAVY = 2;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
 // acc[b][.] += sum over list entries [k0, k1) of alpha * x, for the MVB vectors v0 + 32 b of
