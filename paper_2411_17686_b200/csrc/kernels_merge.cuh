@@ -4,7 +4,7 @@
 
 namespace ficoco {
 
-constexpr int MHUB = 8;        // source rows a lane has in flight for a hub row
+constexpr int MHUB = 4;        // source rows a lane has in flight for a hub row
 constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the per-row arrays)
 constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
 constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
