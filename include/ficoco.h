@@ -68,7 +68,11 @@ enum ficoco_error {
 
 enum ficoco_flags {
   FICOCO_HAS_CLS = 1u,           /* row 0 of every image is a CLS token: never scored, always kept */
-  FICOCO_LOCAL_PENALTY = 2u      /* apply the local penalty (FiCoCo-V default) */
+  FICOCO_LOCAL_PENALTY = 2u,     /* apply the local penalty (FiCoCo-V default) */
+  FICOCO_AVERAGE_COMPRESSION = 4u /* ablation "average compression" (Sec. "Ablation Study", Compress:
+                                    the features are averaged directly): every alpha_ij of Eq. 2
+                                    is 1, so a preserved token becomes the plain mean of itself
+                                    and the discarded tokens sent to it; J_i is unchanged */
 };
 
 /* Hyper-parameters; defaults are the paper's (Sec. "Implementation Details"):

@@ -27,6 +27,8 @@ Readings taken where the paper is silent:
   * weights use max(C, 0) (cosine can be negative, attention cannot); a discarded token
     whose positive mass is zero is pruned;
   * all preserved tokens are updated at once from the pre-update X;
+  * "average compression" (ablation tables; "directly averaging the features") keeps J_i as
+    it is and sets every alpha_ij to 1, whatever the sign of C_ij;
   * for FiCoCo-L the supplied text->vision block t (head mean, M x N) is used for both
     the task term (1/M) sum_k t[k,i] and the text-bridged term (1/M) sum_k t[k,i] t[k,j]
     (main-text equations, which carry the 1/M that Algorithm 2 omits).
@@ -57,6 +59,7 @@ class Params:
     window: int = 2            # local-penalty window side
     local_penalty: bool = True
     max_targets: Optional[int] = None  # None: token-adaptive K (paper); 0: pruning; k>0: fixed K
+    average_compression: bool = False  # ablation "average compression": every alpha_ij = 1
 
 
 # ----------------------------------------------------------------------------
@@ -211,7 +214,11 @@ def quantile_threshold(row: np.ndarray, eps: float) -> float:
 
 def targets_and_weights(C: np.ndarray, p: Params) -> Tuple[List[np.ndarray], List[np.ndarray], np.ndarray]:
     """Per discarded token i: J_i = {j : C_ij >= tau_i} (as column positions in T) and
-    alpha_ij = C+_ij / sum_{j in J_i} C+_ij (Eq. 2).  Returns (J, alpha, tau)."""
+    alpha_ij = C+_ij / sum_{j in J_i} C+_ij (Eq. 2).  Returns (J, alpha, tau).
+
+    With p.average_compression (the "average compression" row of the ablation tables, which
+    Sec. "Ablation Study" describes as directly averaging the features) every alpha_ij is 1,
+    so Eq. 2 turns into the plain mean of a preserved token and the tokens sent to it."""
     ns, nt = C.shape
     J: List[np.ndarray] = []
     A: List[np.ndarray] = []
@@ -228,6 +235,8 @@ def targets_and_weights(C: np.ndarray, p: Params) -> Tuple[List[np.ndarray], Lis
             order = np.argsort(-row, kind="stable")[:k]
             tau[i] = row[order[-1]]
             j = np.sort(order)
+        if p.average_compression:
+            J.append(j.astype(np.int64)); A.append(np.ones(j.shape[0])); continue
         cpos = np.maximum(row[j], 0.0)
         den = cpos.sum()
         if den <= 1e-12:

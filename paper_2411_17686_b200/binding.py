@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libficoco.so")
 
 FICOCO_FP32, FICOCO_BF16 = 0, 1
-FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY = 1, 2
+FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY, FICOCO_AVERAGE_COMPRESSION = 1, 2, 4
 KCAP = 16
 
 INSPECT = {
@@ -109,11 +109,12 @@ def ficoco_default_params() -> ficoco_params:
 
 
 def make_params(lam=0.35, beta=0.6, gamma=0.6, eps=0.998, penalty_coef=2.0, window=2,
-                max_targets=-1, has_cls=True, local_penalty=True) -> ficoco_params:
+                max_targets=-1, has_cls=True, local_penalty=True, average_compression=False) -> ficoco_params:
     p = ficoco_params()
     p.lambda_, p.beta, p.gamma, p.eps, p.penalty_coef = lam, beta, gamma, eps, penalty_coef
     p.window, p.max_targets = window, -1 if max_targets is None else max_targets
-    p.flags = (FICOCO_HAS_CLS if has_cls else 0) | (FICOCO_LOCAL_PENALTY if local_penalty else 0)
+    p.flags = ((FICOCO_HAS_CLS if has_cls else 0) | (FICOCO_LOCAL_PENALTY if local_penalty else 0) |
+               (FICOCO_AVERAGE_COMPRESSION if average_compression else 0))
     return p
 
 

@@ -34,6 +34,7 @@ struct ImgDesc {
   int corr_items;  // correlate work items (CTAs) of this image
   int chunk0;      // first row chunk (column-sum partials)
   int n_chunks;
+  int avg;         // 1: every alpha_ij is 1 ("average compression" ablation)
   long long attn0; // offset (floats) of this image's attention block
 };
 

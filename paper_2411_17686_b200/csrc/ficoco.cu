@@ -34,12 +34,12 @@ constexpr size_t HOST_GROUP_BYTES = 8u << 20;   // at least this many token byte
 
 struct PlanKey {
   int mode;  // 0 = V, 1 = L
-  int dtype, batch, dim, n_text, has_cls, max_targets;
+  int dtype, batch, dim, n_text, has_cls, max_targets, avg;
   double eps;
   std::vector<int> ntok, keep, gh, gw;
   bool operator==(const PlanKey& o) const {
     return mode == o.mode && dtype == o.dtype && batch == o.batch && dim == o.dim &&
-           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets &&
+           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets && avg == o.avg &&
            eps == o.eps && ntok == o.ntok && keep == o.keep && gh == o.gh && gw == o.gw;
   }
 };
@@ -486,6 +486,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     }
     d.list_len = L;
     d.frac = frac;
+    d.avg = key.avg;
     if (L > p->max_list) p->max_list = L;
   }
   // ---- fused filter kernel: piece size and feasibility -------------------------------------
@@ -944,6 +945,7 @@ extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const fico
   key.mode = 0; key.dtype = a->dtype; key.batch = a->batch; key.dim = a->dim; key.n_text = 0;
   key.has_cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
   key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
+  key.avg = (prm->flags & FICOCO_AVERAGE_COMPRESSION) ? 1 : 0;
   key.eps = prm->eps;
   key.ntok.resize(a->batch); key.keep.resize(a->batch); key.gh.resize(a->batch); key.gw.resize(a->batch);
   for (int b = 0; b < a->batch; ++b) {
@@ -984,6 +986,7 @@ extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const fico
   key.mode = 1; key.dtype = a->dtype; key.batch = a->batch; key.dim = a->dim; key.n_text = a->n_text;
   key.has_cls = 0;
   key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
+  key.avg = (prm->flags & FICOCO_AVERAGE_COMPRESSION) ? 1 : 0;
   key.eps = prm->eps;
   key.ntok.assign(a->batch, a->n_vision + a->n_text);
   key.keep.resize(a->batch);

@@ -265,7 +265,7 @@ __device__ __forceinline__ void finalize_source(
       if (ix[k] != INT_MAX && v[k] >= tau) { ++nj; den += fmaxf(v[k], 0.f); } else open = false;
     }
   }
-  if (!(den > 1e-12f)) nj = 0;
+  if (!d.avg && !(den > 1e-12f)) nj = 0;
   corr_cnt[o] = nj;
   tau_out[o] = tau;
   const size_t eb = (size_t)d.ent0 + (size_t)s * L;
@@ -273,7 +273,7 @@ __device__ __forceinline__ void finalize_source(
   for (int k = 0; k < LC; ++k) {
     if (k < L) {
       e_tgt[eb + k] = k < nj ? ix[k] : -1;
-      e_w[eb + k] = k < nj ? fmaxf(v[k], 0.f) / den : 0.f;
+      e_w[eb + k] = k < nj ? (d.avg ? 1.0f : fmaxf(v[k], 0.f) / den) : 0.f;
       e_c[eb + k] = v[k];
     }
   }

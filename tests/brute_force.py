@@ -105,3 +105,14 @@ def _correlate_compress(P, S, T, corr, eps, s_raw, s):
         wsum[j] = w
     return {"s_raw": s_raw, "s": s, "S": S, "T": T, "J": J, "alpha": alpha, "merged": merged,
             "wsum": wsum, "C": C}
+
+
+def group_means(P, S, T, J):
+    """'Average compression' written as what it means, not through Eq. 2: every preserved token j
+    becomes the arithmetic mean of the group made of itself and the discarded tokens that chose it.
+    P: rows (lists of floats); S, T: token indices; J: dict discarded token -> list of targets."""
+    out = {}
+    for j in T:
+        members = [j] + [i for i in S if j in J[i]]
+        out[j] = [math.fsum(P[m][d] for m in members) / len(members) for d in range(len(P[0]))]
+    return out

@@ -22,7 +22,8 @@ def params_to_abi(p: fo.Params, has_cls: bool):
     return binding.make_params(lam=p.lam, beta=p.beta, gamma=p.gamma, eps=p.eps,
                                penalty_coef=p.penalty_coef, window=p.window,
                                max_targets=-1 if p.max_targets is None else p.max_targets,
-                               has_cls=has_cls, local_penalty=p.local_penalty)
+                               has_cls=has_cls, local_penalty=p.local_penalty,
+                               average_compression=p.average_compression)
 
 
 def _widen(a: np.ndarray) -> np.ndarray:

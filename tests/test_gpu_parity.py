@@ -66,7 +66,10 @@ def test_small_progressive_schedule(ctx, idx):
     fo.Params(window=3, penalty_coef=1.5),
     fo.Params(window=1),
     fo.Params(lam=0.8),
-], ids=["nopenalty", "eps097", "eps1", "prune", "fixedK2", "win3", "win1", "lam08"])
+    fo.Params(average_compression=True),            # ablation: features averaged directly
+    fo.Params(eps=0.97, average_compression=True),
+    fo.Params(max_targets=1, average_compression=True),
+], ids=["nopenalty", "eps097", "eps1", "prune", "fixedK2", "win3", "win1", "lam08", "avg", "avg-eps097", "avg-K1"])
 def test_variants(ctx, p):
     batch = synth.make_v_batch(77, 3, 13, 11, 192, 5, 80, "bf16", True, 1.2)
     gaps.repair_v(batch, p)
@@ -107,7 +110,8 @@ def test_fp32_wide_rows(ctx):
 
 
 def test_l_variants(ctx):
-    for p in (fo.Params(gamma=1.0), fo.Params(beta=0.9), fo.Params(eps=0.9), fo.Params(max_targets=0)):
+    for p in (fo.Params(gamma=1.0), fo.Params(beta=0.9), fo.Params(eps=0.9), fo.Params(max_targets=0),
+              fo.Params(eps=0.9, average_compression=True)):
         batch = synth.make_l_batch(82, 2, 100, 9, 256, 3, 30, "bf16", scale=1.0 / 16)
         gaps.repair_l(batch, p)
         parity.run_and_compare_l(ctx, batch, p, DEV, what="l-variant")

@@ -258,6 +258,42 @@ def test_merge_invariants():
     np.testing.assert_allclose(rs.out, same[:25], rtol=1e-6)
 
 
+def test_average_compression_is_the_group_mean():
+    """Ablation 'average compression' (features averaged directly): same S, T, J_i as the default,
+    every weight 1, merged rows equal to the plain mean of each group (scalar-loop routine that
+    does not go through Eq. 2), rows of size-1 groups untouched, and the count-weighted mass
+    identity sum_j |group_j| out_j = sum_{j in T} x_j + sum_i |J_i| x_i."""
+    for seed, eps, kfix in ((6, 0.7, None), (7, 0.998, None), (8, 0.998, 2)):
+        batch = tiny_v(seed)
+        tok, attn = batch.tokens[0], batch.attn[0]
+        P = tok[1:].astype(np.float64)
+        base = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 9, True, fo.Params(eps=eps, max_targets=kfix))
+        r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 9, True,
+                               fo.Params(eps=eps, max_targets=kfix, average_compression=True))
+        assert r.S.tolist() == base.S.tolist() and r.T.tolist() == base.T.tolist()
+        Tl, Sl = r.T.tolist(), r.S.tolist()
+        J = {}
+        for k, i in enumerate(Sl):
+            assert r.J[k].tolist() == base.J[k].tolist()
+            assert r.alpha[k].tolist() == [1.0] * len(r.J[k])
+            J[i] = [Tl[jj] for jj in r.J[k].tolist()]
+        means = bf.group_means(P.tolist(), Sl, Tl, J)
+        sizes = {j: 1 + sum(1 for i in Sl if j in J[i]) for j in Tl}
+        assert max(sizes.values()) > 1
+        for jj, j in enumerate(Tl):
+            np.testing.assert_allclose(r.out[1 + jj].astype(np.float64), means[j], rtol=2e-7, atol=1e-7)
+            if sizes[j] == 1:
+                assert np.array_equal(r.out[1 + jj], tok[1 + j])
+        merged, wsum = fo.compress(P, r.S, r.T, r.J, r.alpha)
+        assert wsum.tolist() == [float(sizes[j] - 1) for j in Tl]
+        lhs = ((1.0 + wsum)[:, None] * merged).sum(axis=0)
+        rhs = P[Tl].sum(axis=0) + sum(len(J[i]) * P[i] for i in Sl)
+        np.testing.assert_allclose(lhs, rhs, atol=1e-10)
+        # the default weights differ from 1 somewhere, so the two variants really differ
+        if kfix is None and eps < 0.9:
+            assert not np.array_equal(r.out, base.out)
+
+
 def test_untouched_rows_keep_their_bits_and_bf16_rounding():
     batch = synth.make_v_batch(28, 2, 8, 8, 64, 2, 40, "bf16")
     for b in range(2):
