@@ -180,6 +180,35 @@ def other_workloads(binding, packing, ctx, insts, prm, stream, dev) -> dict:
     us = e0.elapsed_time(e1) * 1e3 / (5 * N_INSTANCES)
     out["c2 schedule 576->288->144->64"] = {"us_per_schedule": us, "images_per_s": B / (us * 1e-6)}
 
+    # the same step driven by a caller-supplied relation map (fp32 [B, 576, 576], attention each
+    # token receives): the map is read once for the scores and its discarded rows once more for C;
+    # three maps and the 8 token sets are cycled so that every step starts from HBM
+    npatch = GH * GW
+    rels = [torch.softmax(4.0 * torch.randn((B, npatch, npatch), generator=g), -1).reshape(-1).to(dev)
+            for _ in range(3)]
+
+    def rel_step(i):
+        it = insts[i % N_INSTANCES]
+        ctx.ficoco_v_reduce(it["tokens"], it["attn"], KEEP, GH, GW, H, n_tokens=n, pos=it["pos"], params=prm,
+                            out_tokens=it["out"], kept_idx=it["kidx"], pos_out=it["pout"],
+                            stream=stream.cuda_stream, relation=rels[i % 3], by_column=True)
+
+    with torch.cuda.stream(stream):
+        for i in range(3):
+            rel_step(i)
+        e0.record(stream)
+        for i in range(24):
+            rel_step(i)
+        e1.record(stream)
+    torch.cuda.synchronize()
+    assert ctx.ficoco_status(stream.cuda_stream) == 0
+    rel_us = e0.elapsed_time(e1) * 1e3 / 24
+    rel_bytes = B * npatch * npatch * 4 + algorithmic_bytes()["total"]
+    out["c2 step 1 on a supplied relation map (by column)"] = {
+        "us_per_step": rel_us, "images_per_s": B / (rel_us * 1e-6), "algorithmic_bytes": rel_bytes,
+        "achieved_gbs": rel_bytes / rel_us / 1e3, "frac_of_hbm_peak": rel_bytes / rel_us / 1e3 / peaks()["hbm_gbs"]}
+    del rels
+
     for idx, label in ((1, "c1: 1 x 577 x 1024 fp32, discard 64"), (3, "c3 step 1: 8 x 2881 x 1024 bf16, 2880 -> 1440"),
                        (4, "c4: 16 ragged images x 1280 bf16, keep 1/9"), (5, "c5: FiCoCo-L 16 x (576+64) x 4096 bf16, 576 -> 64")):
         wl = synth.workload(idx)

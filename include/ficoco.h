@@ -149,6 +149,24 @@ typedef struct ficoco_v_args {
 int ficoco_v_reduce(ficoco_ctx* ctx, const ficoco_v_args* args, const ficoco_params* params,
                     void* cuda_stream);
 
+/* FiCoCo-V reduce step on a caller-supplied relation matrix: the paper's own formulation, in
+ * which every token-token quantity is read from the self-attention map A^v (Sec.
+ * "Redundancy-based Token Discard", Eq. 1 first term; Sec. "Correlation-based Information
+ * Recycling", C = A^v) instead of from the cosine similarity of the hidden states.
+ *   relation  : device fp32, 4-byte aligned; image b's [Np_b, Np_b] block (row = query token,
+ *               column = key token, alive patch tokens only, no CLS row or column) starts at
+ *               sum_{b' < b} Np_b'^2 floats.  Read only; the caller keeps ownership.
+ *   by_column : 0: v_i = (1/Np) sum_j A[i, j], Eq. 1 as printed (a constant for a row-stochastic
+ *               softmax map); non-zero: v_i = (1/Np) sum_j A[j, i], the attention token i receives,
+ *               as the prose of that paragraph puts it.
+ * C_ij = A[S_i, T_j]; tau_i, J_i, alpha_ij, Eq. 2, the local penalty, the selection and every
+ * other argument, output and error are those of ficoco_v_reduce; the tokens only feed Eq. 2.
+ * The step runs unfused kernels (score, select, correlate, merge) and never reads the N x N block
+ * more than twice (all of it for the scores, the rows of S for C).  Asynchronous on the stream,
+ * allocates nothing. */
+int ficoco_v_reduce_relation(ficoco_ctx* ctx, const ficoco_v_args* args, const float* relation,
+                             int by_column, const ficoco_params* params, void* cuda_stream);
+
 /*
  * FiCoCo-L reduce step (Algorithm 2) for a batch of decoder sequences of equal shape.
  * Each sequence has n_vision vision rows followed by n_text text rows.  Vision rows are

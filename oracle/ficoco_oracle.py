@@ -287,11 +287,19 @@ class StepResult:
 
 def ficoco_v_reduce(tokens: np.ndarray, attn: np.ndarray, pos: Optional[np.ndarray],
                     grid: Tuple[int, int], keep: int, has_cls: bool = True,
-                    p: Optional[Params] = None) -> StepResult:
+                    p: Optional[Params] = None, relation: Optional[np.ndarray] = None,
+                    by_column: bool = False) -> StepResult:
     """One FiCoCo-V reduce step on one image (Algorithm 1).
 
     tokens [c+Np, D]; attn [H, Np]; pos [Np] grid positions (None = identity);
-    keep = N^T preserved patch tokens."""
+    keep = N^T preserved patch tokens.
+
+    relation: optional [Np, Np] map A^v over the patch tokens (row = query).  When given it is
+    used wherever the paper writes A^v: the first term of Eq. 1 is (1/N) sum_j A_{i,j} as
+    printed, or with by_column (1/N) sum_j A_{j,i}, the attention token i receives (the prose
+    of the same paragraph; for a row-stochastic softmax map the printed sum is the constant
+    1/N), and C_ij = A_{S_i, T_j} (Sec. "Correlation-based Information Recycling").  The
+    tokens then only feed Eq. 2."""
     p = p or Params()
     c = 1 if has_cls else 0
     X = widen(tokens)
@@ -304,8 +312,13 @@ def ficoco_v_reduce(tokens: np.ndarray, attn: np.ndarray, pos: Optional[np.ndarr
     n_src = npatch - keep
 
     # Stage 1: Filter
-    R = cosine_relation(P)
-    v = vision_redundancy(R)
+    if relation is None:
+        R = cosine_relation(P)
+        v = vision_redundancy(R)
+    else:
+        R = np.asarray(relation, dtype=np.float64)
+        assert R.shape == (npatch, npatch)
+        v = vision_redundancy(R.T if by_column else R)
     a = head_mean(attn)
     s_raw = score_v(v, a, p.lam)
     s = local_penalty(s_raw, pos, grid, p.window, p.penalty_coef) if p.local_penalty else s_raw.copy()

@@ -157,6 +157,42 @@ def repair_v(batch, p: Optional[fo.Params] = None, max_iter: int = 40, seed: int
     return log
 
 
+def repair_v_relation(batch, rels: List[np.ndarray], by_column: bool, p: Optional[fo.Params] = None,
+                      max_iter: int = 60, seed: int = 11) -> List[str]:
+    """repair_v for the relation mode (rels[b]: fp32 [Np, Np] map of image b, changed in place).
+    Window and boundary margins are repaired through the attention columns as in repair_v; a
+    correlation row that is too close to its threshold gets that discarded token's row of the map
+    rescaled entry by entry by a few per cent."""
+    p = p or fo.Params()
+    log: List[str] = []
+    for b in range(batch.batch):
+        for it in range(max_iter):
+            res = fo.ficoco_v_reduce(batch.tokens[b], batch.attn[b], batch.pos[b], batch.grid[b],
+                                     batch.keep[b], batch.has_cls, p, relation=rels[b], by_column=by_column)
+            m = margins(res, batch.pos[b].astype(np.int64), batch.grid[b], p, p.local_penalty)
+            if ok(m):
+                break
+            rng = np.random.Generator(np.random.Philox(key=[seed, (b << 16) | it]))
+            if m.win_gap < WIN_GAP:
+                for (_win, second) in m.win_pairs:
+                    d = (2.0 * WIN_GAP + 1e-6 * rng.random()) / (1.0 - p.lam)
+                    batch.attn[b][:, second] += np.float32(d)
+                    log.append(f"img {b} it {it}: window runner-up {second} attn += {d:.3e}")
+            elif m.sel_gap < SEL_GAP:
+                for lower, d in _band(res, m, rng, 1.0 - p.lam):
+                    batch.attn[b][:, lower] += np.float32(d)
+                    log.append(f"img {b} it {it}: boundary token {lower} attn += {d:.3e}")
+            else:
+                for i in m.bad_rows:
+                    row = int(res.S[i])
+                    f = 1.0 + 0.05 * rng.standard_normal(rels[b].shape[1])
+                    rels[b][row] = (rels[b][row].astype(np.float64) * np.abs(f)).astype(np.float32)
+                    log.append(f"img {b} it {it}: rescaled relation row {row}")
+        else:
+            raise RuntimeError(f"image {b}: margins not repaired after {max_iter} iterations: {m}")
+    return log
+
+
 def repair_l(batch, p: Optional[fo.Params] = None, max_iter: int = 40, seed: int = 7) -> List[str]:
     """Same for a synthetic LBatch (no windows; the score's attention term is the text->vision
     column mean, moved by raising that column for every head and text row)."""

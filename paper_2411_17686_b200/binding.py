@@ -32,7 +32,7 @@ EXPORTS = [
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
     "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
-    "ficoco_equivalent_token",
+    "ficoco_equivalent_token", "ficoco_v_reduce_relation",
 ]
 
 
@@ -88,6 +88,8 @@ def load_library() -> C.CDLL:
                                             C.c_int, C.c_int, C.c_void_p, C.c_void_p]
     lib.ficoco_v_reduce.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_l_reduce.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params), C.c_void_p]
+    lib.ficoco_v_reduce_relation.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.c_void_p, C.c_int,
+                                             C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_v_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params)]
     lib.ficoco_l_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params)]
     lib.ficoco_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
@@ -179,10 +181,13 @@ class Context:
     def ficoco_v_reduce(self, tokens, attn, keep, grid_h, grid_w, heads: int, *, n_tokens: int = 0,
                         seqlens=None, pos=None, params: Optional[ficoco_params] = None,
                         out_tokens=None, kept_idx=None, pos_out=None, scores_out=None,
-                        want_scores: bool = False, stream: Optional[int] = None) -> VResult:
+                        want_scores: bool = False, stream: Optional[int] = None,
+                        relation=None, by_column: bool = False) -> VResult:
         """tokens: cuda tensor [rows, D]; attn: cuda fp32 tensor (packed per image [H, Np]);
         keep / grid_h / grid_w: int or per-image list; seqlens: per-image rows incl. CLS or
-        None with n_tokens given.  Output tensors are allocated with torch when not passed."""
+        None with n_tokens given.  Output tensors are allocated with torch when not passed.
+        relation: optional cuda fp32 tensor, the images' [Np, Np] relation blocks one after the
+        other; when given the call goes to ficoco_v_reduce_relation."""
         import torch
         p = params or ficoco_default_params()
         cls = 1 if (p.flags & FICOCO_HAS_CLS) else 0
@@ -217,7 +222,11 @@ class Context:
         a.n_grid, a.n_keep = n_gh, n_keep
         if stream is None:
             stream = torch.cuda.current_stream(dev).cuda_stream
-        _check(self.h, self.lib.ficoco_v_reduce(self.h, C.byref(a), C.byref(p), C.c_void_p(stream)))
+        if relation is not None:
+            _check(self.h, self.lib.ficoco_v_reduce_relation(self.h, C.byref(a), _ptr(relation), int(by_column),
+                                                             C.byref(p), C.c_void_p(stream)))
+        else:
+            _check(self.h, self.lib.ficoco_v_reduce(self.h, C.byref(a), C.byref(p), C.c_void_p(stream)))
         return VResult(out_tokens, kept_idx, pos_out, scores_out, out_rows)
 
     def ficoco_l_reduce(self, tokens, attn_t2v, keep, n_vision: int, n_text: int, heads: int, *,

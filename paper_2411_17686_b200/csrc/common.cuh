@@ -36,6 +36,7 @@ struct ImgDesc {
   int n_chunks;
   int avg;         // 1: every alpha_ij is 1 ("average compression" ablation)
   long long attn0; // offset (floats) of this image's attention block
+  long long rel0;  // offset (floats) of this image's [Np, Np] relation block (relation mode)
 };
 
 struct WorkItem {

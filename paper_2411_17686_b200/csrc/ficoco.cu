@@ -16,6 +16,7 @@
 #include "kernels_filter.cuh"
 #include "kernels_filter_fused.cuh"
 #include "kernels_merge.cuh"
+#include "kernels_relation.cuh"
 
 using namespace ficoco;
 
@@ -35,11 +36,12 @@ constexpr size_t HOST_GROUP_BYTES = 8u << 20;   // at least this many token byte
 struct PlanKey {
   int mode;  // 0 = V, 1 = L
   int dtype, batch, dim, n_text, has_cls, max_targets, avg;
+  int rel = 0;  // 0: cosine relation of the tokens; 1 / 2: caller-supplied relation, by row / by column
   double eps;
   std::vector<int> ntok, keep, gh, gw;
   bool operator==(const PlanKey& o) const {
     return mode == o.mode && dtype == o.dtype && batch == o.batch && dim == o.dim &&
-           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets && avg == o.avg &&
+           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets && avg == o.avg && rel == o.rel &&
            eps == o.eps && ntok == o.ntok && keep == o.keep && gh == o.gh && gw == o.gw;
   }
 };
@@ -444,13 +446,14 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   const int tail = key.mode == 1 ? key.n_text : 0;
   p->h_desc.assign(B, ImgDesc());
   std::vector<WorkItem> rows, corr, outw;
-  long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0;
+  long long row0 = 0, patch0 = 0, out0 = 0, src0 = 0, tgt0 = 0, ent0 = 0, part0 = 0, chunk0 = 0, rel0 = 0;
   p->max_np = p->max_tgt = p->max_src = p->max_rc = p->max_nwin_cells = p->max_list = 0;
   p->need_finalize = false;
   // tensor-core correlate: bf16 tokens, hidden size a multiple of 64.  FiCoCo-L adds its text term
   // in the epilogue from weights staged in shared memory, 2 KB per text token for the largest tile.
   p->umma = key.dtype == FICOCO_BF16 && key.dim % UKB == 0 &&
             (key.mode == 0 || (size_t)key.n_text * 2048 + 1024 + (size_t)UM * KCAP * 8 <= 220 * 1024);
+  if (key.rel) p->umma = false;                       // C is read from the supplied matrix, not contracted
   int tile_rows_max = p->umma ? UM : CBM;             // source rows per correlate CTA (decided below)
   const int col_granule = p->umma ? 16 : CBN;
   int um_a_rows = 8, um_cols = 16;
@@ -493,7 +496,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   const int esz = key.dtype == FICOCO_BF16 ? 2 : 4;
   const int f_nvec = key.dim / (16 / esz);
   p->f_vpl = (f_nvec + 31) / 32;
-  p->fused = c->coop_ok && p->f_vpl <= 8;
+  p->fused = c->coop_ok && p->f_vpl <= 8 && !key.rel;
   int f_rc = 0;
   if (p->fused) {
     long long total = 0;
@@ -568,6 +571,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     d.row0 = (int)row0; d.patch0 = (int)patch0; d.out_row0 = (int)out0;
     d.src0 = (int)src0; d.tgt0 = (int)tgt0; d.ent0 = (int)ent0; d.part0 = (int)part0;
     d.attn0 = 0;  // set by the caller-specific code below
+    d.rel0 = rel0;
+    rel0 += (long long)d.np * d.np;
     // row chunks (fused filter: equal pieces of at most f_rc rows)
     int rc = (d.np + MAX_CHUNKS - 1) / MAX_CHUNKS;
     rc = (rc + 7) / 8 * 8;
@@ -810,7 +815,7 @@ template <class T>
 int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn, int attn_rows,
              float cA, const int* pos, int window, float coef, int penalty, const float* tmean, int M,
              float gamma, T* out_tokens, int* kept_idx, int* pos_out, float* scores_out,
-             cudaStream_t st) {
+             cudaStream_t st, const float* rel = nullptr) {
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
@@ -838,6 +843,12 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     if (fe != cudaSuccess) { c->last_cuda = (int)fe; return FICOCO_ERR_CUDA; }
     c->launches += 1;
   } else {
+  if (rel) {
+    prof_tick(c, st, "score_relation");
+    k_score_rel<<<p->n_rows, 256, (size_t)p->max_rc * sizeof(float), st>>>(
+        rel, p->d_desc, p->d_rows, attn, attn_rows, cA, p->key.rel == 2 ? 1 : 0, c->s_raw);
+    c->launches += 1;
+  } else {
   prof_tick(c, st, vpl <= 8 ? "colsum" : "rownorm");
   if (vpl <= 8) {
     if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
@@ -857,15 +868,22 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   prof_tick(c, st, "score");
   k_score<T><<<p->n_rows, 256, (size_t)(D + p->max_rc) * sizeof(float), st>>>(
       tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
+  c->launches += 1;
+  }
   const size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
   prof_tick(c, st, "select");
   k_select<<<p->key.batch, 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
                                                   pos_out, c->status);
-  c->launches += 2;
+  c->launches += 1;
   }
   if (p->n_corr > 0) {
-    if (p->umma && sizeof(T) == 2) {
+    if (rel) {
+      prof_tick(c, st, "correlate_relation");
+      k_correlate_rel<<<p->n_corr, 256, 0, st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val,
+                                                 c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,
+                                                 c->e_w, c->e_c);
+    } else if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
@@ -928,8 +946,9 @@ int check_common(const ficoco_params* prm, int dtype, int batch, int dim, int he
 
 }  // namespace
 
-extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm,
-                               void* cuda_stream) {
+namespace {
+int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm, void* cuda_stream,
+                  const float* rel, int rel_mode) {
   if (!c || !a) return FICOCO_ERR_INVALID_ARG;
   int rc = check_common(prm, a->dtype, a->batch, a->dim, a->heads, a->tokens, a->out_tokens);
   if (rc) return rc;
@@ -946,6 +965,7 @@ extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const fico
   key.has_cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
   key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
   key.avg = (prm->flags & FICOCO_AVERAGE_COMPRESSION) ? 1 : 0;
+  key.rel = rel_mode;
   key.eps = prm->eps;
   key.ntok.resize(a->batch); key.keep.resize(a->batch); key.gh.resize(a->batch); key.gw.resize(a->batch);
   for (int b = 0; b < a->batch; ++b) {
@@ -964,10 +984,22 @@ extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const fico
     return run_step<__nv_bfloat16>(c, p, (const __nv_bfloat16*)a->tokens, a->dim, a->attn, a->heads,
                                    (float)prm->lambda_, a->pos, prm->window, (float)prm->penalty_coef,
                                    penalty, nullptr, 0, 1.0f, (__nv_bfloat16*)a->out_tokens, a->kept_idx,
-                                   a->pos_out, a->scores_out, st);
+                                   a->pos_out, a->scores_out, st, rel);
   return run_step<float>(c, p, (const float*)a->tokens, a->dim, a->attn, a->heads, (float)prm->lambda_,
                          a->pos, prm->window, (float)prm->penalty_coef, penalty, nullptr, 0, 1.0f,
-                         (float*)a->out_tokens, a->kept_idx, a->pos_out, a->scores_out, st);
+                         (float*)a->out_tokens, a->kept_idx, a->pos_out, a->scores_out, st, rel);
+}
+}  // namespace
+
+extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm,
+                               void* cuda_stream) {
+  return v_reduce_impl(c, a, prm, cuda_stream, nullptr, 0);
+}
+
+extern "C" int ficoco_v_reduce_relation(ficoco_ctx* c, const ficoco_v_args* a, const float* relation,
+                                        int by_column, const ficoco_params* prm, void* cuda_stream) {
+  if (!relation || ((uintptr_t)relation & 3)) return FICOCO_ERR_INVALID_ARG;
+  return v_reduce_impl(c, a, prm, cuda_stream, relation, by_column ? 2 : 1);
 }
 
 extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const ficoco_params* prm,

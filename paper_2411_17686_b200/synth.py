@@ -79,6 +79,19 @@ def softmax_attention(rng: np.random.Generator, heads: int, n: int, logit_std: f
     return (e / e.sum(axis=1, keepdims=True)).astype(np.float32)
 
 
+def relation_map(rng: np.random.Generator, patches: np.ndarray, sharpness: float = 8.0,
+                 logit_std: float = 1.0) -> np.ndarray:
+    """[Np, Np] fp32 stand-in for a head-averaged self-attention map over the patch tokens:
+    row i is a softmax over sharpness * cos(x_i, x_j) + N(0, logit_std) logits, so rows sum to 1,
+    the map is not symmetric and similar tokens attend to each other."""
+    x = patches.astype(np.float64)
+    xh = x / np.sqrt((x * x).sum(axis=1, keepdims=True))
+    z = sharpness * (xh @ xh.T) + logit_std * rng.standard_normal((x.shape[0], x.shape[0]))
+    z -= z.max(axis=1, keepdims=True)
+    e = np.exp(z)
+    return (e / e.sum(axis=1, keepdims=True)).astype(np.float32)
+
+
 def causal_text_to_vision_attention(rng: np.random.Generator, heads: int, n_vision: int,
                                     n_text: int, logit_std: float = 1.0) -> np.ndarray:
     """[heads, n_text, n_vision] fp32: the vision block of a causal softmax.  Text row k

@@ -49,7 +49,8 @@ def compare_tokens(got: np.ndarray, exp: np.ndarray, wsum: np.ndarray, c: int, t
         assert np.abs(g - e).max() <= 2.0 ** -7 * max(1.0, np.abs(e).max()), what
 
 
-def compare_stages(ctx: binding.Context, results: List[fo.StepResult], n_cls: int, what: str):
+def compare_stages(ctx: binding.Context, results: List[fo.StepResult], n_cls: int, what: str,
+                   check_rn: bool = True):
     """Intermediate arrays of the last call vs the checker, image by image."""
     rn = ctx.ficoco_inspect("rnorm")
     s_raw = ctx.ficoco_inspect("score_raw")
@@ -65,7 +66,8 @@ def compare_stages(ctx: binding.Context, results: List[fo.StepResult], n_cls: in
     for b, r in enumerate(results):
         npatch, ns, nt = r.score.shape[0], r.S.shape[0], r.T.shape[0]
         tag = f"{what} image {b}"
-        np.testing.assert_allclose(rn[p0:p0 + npatch], r.rn, rtol=1e-6, err_msg=tag + " rnorm")
+        if check_rn:
+            np.testing.assert_allclose(rn[p0:p0 + npatch], r.rn, rtol=1e-6, err_msg=tag + " rnorm")
         scale = float(np.mean(np.abs(r.score_raw)))
         for got, exp, nm in ((s_raw[p0:p0 + npatch], r.score_raw, "score_raw"),
                              (s_pen[p0:p0 + npatch], r.score, "score")):
@@ -120,6 +122,36 @@ def run_and_compare_v(ctx: binding.Context, batch, p: fo.Params, device, stages:
         compare_stages(ctx, results, c, what)
         sc = binding.to_numpy(res.scores)
         assert np.array_equal(sc, ctx.ficoco_inspect("score"))
+    return res, results
+
+
+def run_and_compare_v_relation(ctx: binding.Context, batch, rels, by_column: bool, p: fo.Params, device,
+                               what: str = ""):
+    """ficoco_v_reduce_relation against the checker given the same relation blocks."""
+    import torch
+    pk = packing.pack_v(batch, device)
+    prm = params_to_abi(p, batch.has_cls)
+    rel_d = torch.from_numpy(np.concatenate([r.reshape(-1) for r in rels])).to(device)
+    res = ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm,
+                              want_scores=True, relation=rel_d, by_column=by_column, **pk.call_kwargs())
+    assert ctx.ficoco_status() == 0
+    results = [fo.ficoco_v_reduce(batch.tokens[b], batch.attn[b], batch.pos[b], batch.grid[b], batch.keep[b],
+                                  batch.has_cls, p, relation=rels[b], by_column=by_column)
+               for b in range(batch.batch)]
+    out = binding.to_numpy(res.out_tokens)
+    kidx = binding.to_numpy(res.kept_idx)
+    pout = binding.to_numpy(res.pos_out)
+    c = 1 if batch.has_cls else 0
+    r0 = k0 = 0
+    for b, r in enumerate(results):
+        nrow = res.out_rows[b]
+        assert nrow == r.out.shape[0]
+        assert np.array_equal(kidx[r0:r0 + nrow], r.kept_idx), f"{what} image {b}: kept_idx"
+        nt = r.T.shape[0]
+        assert np.array_equal(pout[k0:k0 + nt], r.pos_out), f"{what} image {b}: pos_out"
+        compare_tokens(out[r0:r0 + nrow], r.out, r.wsum, c, 0, f"{what} image {b}")
+        r0 += nrow; k0 += nt
+    compare_stages(ctx, results, c, what, check_rn=False)
     return res, results
 
 

@@ -109,6 +109,44 @@ def test_fp32_wide_rows(ctx):
     parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="fp32-wide")
 
 
+def _relations(batch, seed, stochastic=True, times_n=False):
+    c = 1 if batch.has_cls else 0
+    rels = []
+    for b in range(batch.batch):
+        r = synth.relation_map(synth.rng_for(seed, b, 21), fo.widen(batch.tokens[b])[c:])
+        if not stochastic:   # rows of different mass, so that the by-row mean is not a constant
+            r = (r * synth.rng_for(seed, b, 22).uniform(0.5, 1.5, size=(r.shape[0], 1))).astype(np.float32)
+        if times_n:          # entries of order one whatever the image size
+            r = (r * np.float32(r.shape[0])).astype(np.float32)
+        rels.append(r)
+    return rels
+
+
+@pytest.mark.parametrize("by_column", [False, True], ids=["by-row", "by-column"])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_relation_mode(ctx, by_column, dtype):
+    """Caller-supplied relation map in place of the cosine similarity: scores, S / T, target
+    sets, weights and merged rows against the checker given the same map."""
+    batch = synth.make_v_batch(90, 3, 13, 11, 192, 5, 60, dtype, True, 1.2)
+    rels = _relations(batch, 90, stochastic=by_column)
+    for p in (fo.Params(), fo.Params(eps=0.97, local_penalty=False)):
+        gaps.repair_v_relation(batch, rels, by_column, p)
+        parity.run_and_compare_v_relation(ctx, batch, rels, by_column, p, DEV, what="relation")
+
+
+def test_relation_mode_ragged_no_cls(ctx):
+    batch = synth.workload(4, small=True)
+    rels = _relations(batch, 91, times_n=True)
+    gaps.repair_v_relation(batch, rels, True)
+    parity.run_and_compare_v_relation(ctx, batch, rels, True, fo.Params(), DEV, what="relation-ragged")
+    # keep everything / keep nothing
+    for keep_all in (True, False):
+        b2 = synth.make_v_batch(92, 2, 6, 6, 64, 2, 36 if keep_all else 0, "bf16", True, 1.0)
+        r2 = _relations(b2, 92)
+        gaps.repair_v_relation(b2, r2, True)
+        parity.run_and_compare_v_relation(ctx, b2, r2, True, fo.Params(), DEV, what="relation-edge")
+
+
 def test_l_variants(ctx):
     for p in (fo.Params(gamma=1.0), fo.Params(beta=0.9), fo.Params(eps=0.9), fo.Params(max_targets=0),
               fo.Params(eps=0.9, average_compression=True)):

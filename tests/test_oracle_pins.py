@@ -294,6 +294,42 @@ def test_average_compression_is_the_group_mean():
             assert not np.array_equal(r.out, base.out)
 
 
+def test_relation_argument():
+    """The relation argument replaces A^v everywhere and nothing else: (i) given the cosine
+    similarity computed by torch it reproduces the default step; (ii) for a symmetric map the two
+    directions of the mean agree; (iii) a row-stochastic map makes the printed first term of Eq. 1
+    the constant 1/N, so the ranking is that of the attention term alone (lambda = 0); (iv) scores
+    and C against scalar loops over the map."""
+    batch = synth.make_v_batch(31, 1, 6, 6, 16, 3, 20, "fp32", True, 1.0)
+    tok, attn = batch.tokens[0], batch.attn[0]
+    P = torch.from_numpy(tok[1:].astype(np.float64))
+    R = torch.nn.functional.cosine_similarity(P[:, None, :], P[None, :, :], dim=-1).numpy()
+    p = fo.Params(eps=0.9)
+    r_def = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, p)
+    for by_col in (False, True):
+        r = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, p, relation=R, by_column=by_col)
+        np.testing.assert_allclose(r.score, r_def.score, atol=1e-13)
+        assert r.S.tolist() == r_def.S.tolist() and r.kept_idx.tolist() == r_def.kept_idx.tolist()
+        assert all(a.tolist() == b.tolist() for a, b in zip(r.J, r_def.J))
+        np.testing.assert_allclose(r.out, r_def.out, rtol=1e-6, atol=1e-7)
+    A = synth.relation_map(synth.rng_for(31, 5), tok[1:]).astype(np.float64)
+    np.testing.assert_allclose(A.sum(axis=1), 1.0, atol=1e-6)
+    pn = fo.Params(local_penalty=False)
+    r_row = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, pn, relation=A)
+    r_att = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, fo.Params(lam=0.0, local_penalty=False))
+    np.testing.assert_allclose(r_row.v, 1.0 / 36, atol=1e-8)
+    assert sorted(r_row.S.tolist()) == sorted(r_att.S.tolist())
+    r_col = fo.ficoco_v_reduce(tok, attn, None, (6, 6), 20, True, pn, relation=A, by_column=True)
+    a_mean = attn.astype(np.float64).mean(axis=0)
+    for i in range(36):
+        received = sum(A[j, i] for j in range(36)) / 36
+        assert abs(r_col.score_raw[i] - (0.35 * received - 0.65 * a_mean[i])) < 1e-12
+    for k, i in enumerate(r_col.S.tolist()):
+        for jj, j in enumerate(r_col.T.tolist()):
+            assert r_col.C[k, jj] == A[i, j]
+    assert not np.array_equal(r_col.S, r_row.S) or not np.allclose(r_col.score_raw, r_row.score_raw)
+
+
 def test_untouched_rows_keep_their_bits_and_bf16_rounding():
     batch = synth.make_v_batch(28, 2, 8, 8, 64, 2, 40, "bf16")
     for b in range(2):
