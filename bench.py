@@ -196,13 +196,20 @@ def other_workloads(binding, packing, ctx, insts, prm, stream, dev) -> dict:
     with torch.cuda.stream(stream):
         for i in range(3):
             rel_step(i)
-        e0.record(stream)
+    torch.cuda.synchronize()
+    rel_graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(rel_graph, stream=stream):
         for i in range(24):
             rel_step(i)
+    with torch.cuda.stream(stream):
+        rel_graph.replay()
+        e0.record(stream)
+        for _ in range(5):
+            rel_graph.replay()
         e1.record(stream)
     torch.cuda.synchronize()
     assert ctx.ficoco_status(stream.cuda_stream) == 0
-    rel_us = e0.elapsed_time(e1) * 1e3 / 24
+    rel_us = e0.elapsed_time(e1) * 1e3 / (5 * 24)
     rel_bytes = B * npatch * npatch * 4 + algorithmic_bytes()["total"]
     out["c2 step 1 on a supplied relation map (by column)"] = {
         "us_per_step": rel_us, "images_per_s": B / (rel_us * 1e-6), "algorithmic_bytes": rel_bytes,

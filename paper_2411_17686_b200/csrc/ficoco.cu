@@ -455,6 +455,17 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
             (key.mode == 0 || (size_t)key.n_text * 2048 + 1024 + (size_t)UM * KCAP * 8 <= 220 * 1024);
   if (key.rel) p->umma = false;                       // C is read from the supplied matrix, not contracted
   int tile_rows_max = p->umma ? UM : CBM;             // source rows per correlate CTA (decided below)
+  if (key.rel) {
+    // a warp of the relation correlate takes one discarded token at a time and is bound by the
+    // latency of its gathers: small tiles put more rows in flight (as far as the work table goes)
+    auto strips = [&](int t) {
+      long long n = 0;
+      for (int b = 0; b < B; ++b) n += (key.ntok[b] - cls - tail - key.keep[b] + t - 1) / t;
+      return n;
+    };
+    tile_rows_max = 16;
+    while (tile_rows_max < CBM && strips(tile_rows_max) + 2 * c->num_sms > c->cap_corr) tile_rows_max *= 2;
+  }
   const int col_granule = p->umma ? 16 : CBN;
   int um_a_rows = 8, um_cols = 16;
 
@@ -880,9 +891,14 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   if (p->n_corr > 0) {
     if (rel) {
       prof_tick(c, st, "correlate_relation");
-      k_correlate_rel<<<p->n_corr, 256, 0, st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val,
-                                                 c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,
-                                                 c->e_w, c->e_c);
+#define FICOCO_REL_GO(LC)                                                                              \
+  k_correlate_rel<LC><<<p->n_corr, 256, 0, st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
+                                                 c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
+                                                 c->e_w, c->e_c)
+      if (p->max_list <= 2) FICOCO_REL_GO(2);
+      else if (p->max_list <= 4) FICOCO_REL_GO(4);
+      else FICOCO_REL_GO(16);
+#undef FICOCO_REL_GO
     } else if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);

@@ -16,8 +16,9 @@ constexpr int RCOLS = 64;   // columns summed together in the by-column mode
 // s_i = cA * v_i - (1 - cA) * mean_h attn[h, i] for one row chunk of one image, with
 //   by_column == 0:  v_i = (1/Np) sum_j A[i, j]   (Eq. 1 as printed: row i of the map)
 //   by_column == 1:  v_i = (1/Np) sum_j A[j, i]   (the attention token i receives)
-// Row mode: one warp per row, four partial sums per lane.  Column mode: 64 columns x 4 row
-// phases per pass, two partial sums per thread, phases added in a fixed order.
+// Row mode: two rows per warp at a time, four partial sums per row and lane.  Column mode:
+// 64 columns x 4 row phases per pass, eight partial sums per thread (eight rows in flight),
+// phases added in a fixed order.
 __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel,
                                                    const ImgDesc* __restrict__ desc,
                                                    const WorkItem* __restrict__ work,
@@ -32,29 +33,49 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_np = 1.0f / (float)np;
   if (!by_column) {
-    for (int r = warp; r < w.nrows; r += 8) {
-      const float* row = A + (size_t)(w.r0 + r) * np;
-      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-      int j = lane;
-      for (; j + 96 < np; j += 128) {
-        s0 += __ldg(row + j); s1 += __ldg(row + j + 32); s2 += __ldg(row + j + 64); s3 += __ldg(row + j + 96);
+    // two rows per warp at a time, four partial sums per row and lane
+    for (int r = 2 * warp; r < w.nrows; r += 16) {
+      const bool two = r + 1 < w.nrows;
+      const float* row0 = A + (size_t)(w.r0 + r) * np;
+      const float* row1 = two ? row0 + np : row0;
+      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+      for (int j0 = lane; j0 < np; j0 += 128) {
+        float a[2][4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int j = j0 + 32 * q;
+          a[0][q] = j < np ? __ldg(row0 + j) : 0.f;
+          a[1][q] = j < np ? __ldg(row1 + j) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { s[0][q] += a[0][q]; s[1][q] += a[1][q]; }
       }
-      for (; j < np; j += 32) s0 += __ldg(row + j);
-      const float s = warp_sum((s0 + s1) + (s2 + s3));
-      if (lane == 0) vrow[r] = s * inv_np;
+      const float t0 = warp_sum((s[0][0] + s[0][1]) + (s[0][2] + s[0][3]));
+      const float t1 = warp_sum((s[1][0] + s[1][1]) + (s[1][2] + s[1][3]));
+      if (lane == 0) {
+        vrow[r] = t0 * inv_np;
+        if (two) vrow[r + 1] = t1 * inv_np;
+      }
     }
   } else {
     const int tx = tid & (RCOLS - 1), ty = tid / RCOLS;
     for (int c0 = 0; c0 < w.nrows; c0 += RCOLS) {
       const int c = c0 + tx;
-      float s0 = 0.f, s1 = 0.f;
+      float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       if (c < w.nrows) {
         const float* col = A + w.r0 + c;
-        int j = ty;
-        for (; j + 4 < np; j += 8) { s0 += __ldg(col + (size_t)j * np); s1 += __ldg(col + (size_t)(j + 4) * np); }
-        for (; j < np; j += 4) s0 += __ldg(col + (size_t)j * np);
+        for (int j0 = ty; j0 < np; j0 += 32) {     // rows j0, j0 + 4, ..., j0 + 28 in flight
+          float a[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int j = j0 + 4 * q;
+            a[q] = j < np ? __ldg(col + (size_t)j * np) : 0.f;
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) s8[q] += a[q];
+        }
       }
-      red[ty][tx] = s0 + s1;
+      red[ty][tx] = ((s8[0] + s8[1]) + (s8[2] + s8[3])) + ((s8[4] + s8[5]) + (s8[6] + s8[7]));
       __syncthreads();
       if (ty == 0 && c < w.nrows) vrow[c] = ((red[0][tx] + red[1][tx]) + (red[2][tx] + red[3][tx])) * inv_np;
       __syncthreads();
@@ -70,10 +91,14 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
   }
 }
 
-// C_ij = A[S_i, T_j]: a CTA owns up to 64 discarded tokens and one column split of the image's
-// preserved tokens, gathers the entries 64 columns at a time into shared memory and keeps the L
-// largest per row (value, position in T) exactly as the fp32 correlate kernel does; the partial
-// lists and the tail (tau_i, J_i, alpha_ij by the last split of the tile) are shared with it.
+// C_ij = A[S_i, T_j].  A CTA owns up to 64 discarded tokens of one image and one column split of
+// the image's preserved tokens; a warp takes one discarded token at a time.  Its lanes walk the
+// split's columns (four gathers from the token's row of the map in flight per lane), each lane
+// keeping the LC largest entries it saw (value, position in T) in registers; the warp then draws
+// the L largest of the 32 lists one by one (a shuffle tournament over the lists' heads).  The
+// partial lists and the tail (tau_i, J_i, alpha_ij by the last split of the tile) are those of
+// the fp32 correlate kernel.
+template <int LC>
 __global__ void __launch_bounds__(256) k_correlate_rel(
     const float* __restrict__ rel, const ImgDesc* __restrict__ desc, const WorkItem* __restrict__ work,
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
@@ -81,47 +106,65 @@ __global__ void __launch_bounds__(256) k_correlate_rel(
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
     float* __restrict__ e_w, float* __restrict__ e_c) {
   __shared__ int is_last;
-  __shared__ float Cs[CBM][CBN + 1];
-  __shared__ float lv[CBM][KCAP];
-  __shared__ int li[CBM][KCAP];
-  __shared__ int rowS[CBM], rowT[CBN];
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int L = d.list_len, np = d.np;
-  const int tid = threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* A = rel + d.rel0;
-  for (int i = tid; i < CBM * KCAP; i += 256) {
-    (&lv[0][0])[i] = -CUDART_INF_F;
-    (&li[0][0])[i] = INT_MAX;
-  }
-  if (tid < CBM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : 0;
+  const int* tcol = T_idx + d.tgt0;
   const int col_begin = w.aux * d.cols_per_split;
   const int col_end = min(d.n_tgt, col_begin + d.cols_per_split);
-  for (int c0 = col_begin; c0 < col_end; c0 += CBN) {
-    __syncthreads();
-    const int ncol = min(CBN, col_end - c0);
-    if (tid < CBN) rowT[tid] = tid < ncol ? T_idx[d.tgt0 + c0 + tid] : 0;
-    __syncthreads();
-    for (int i = tid; i < w.nrows * CBN; i += 256) {
-      const int r = i / CBN, c = i % CBN;
-      Cs[r][c] = c < ncol ? __ldg(A + (size_t)rowS[r] * np + rowT[c]) : 0.f;
-    }
-    __syncthreads();
-    if (tid < w.nrows) {
-      for (int c = 0; c < ncol; ++c) {
-        const float val = Cs[tid][c];
-        const int idx = c0 + c;
-        if (toplist_better(val, idx, lv[tid][L - 1], li[tid][L - 1]))
-          toplist_insert(lv[tid], li[tid], L, val, idx);
+  #pragma unroll 1
+  for (int r = warp; r < w.nrows; r += 8) {
+    const float* row = A + (size_t)S_idx[d.src0 + w.r0 + r] * np;
+    float v[LC];
+    int ix[LC];
+#pragma unroll
+    for (int k = 0; k < LC; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
+    #pragma unroll 1
+    for (int c0 = col_begin + lane; c0 < col_end; c0 += 128) {
+      float a[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int c = c0 + 32 * q;
+        a[q] = c < col_end ? __ldg(row + __ldg(tcol + c)) : -CUDART_INF_F;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float cv = a[q];
+        int ci = c0 + 32 * q;
+        if (ci >= col_end) continue;
+#pragma unroll
+        for (int k = 0; k < LC; ++k) {     // sorted insertion: the displaced entry moves down
+          if (toplist_better(cv, ci, v[k], ix[k])) {
+            const float tv = v[k]; const int ti = ix[k];
+            v[k] = cv; ix[k] = ci; cv = tv; ci = ti;
+          }
+        }
       }
     }
-  }
-  __syncthreads();
-  for (int i = tid; i < w.nrows * L; i += 256) {
-    const int r = i / L, k = i % L;
-    const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + r) * d.nsplit + w.aux) * L + k;
-    part_val[o] = lv[r][k];
-    part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
+    // the L best of the warp, best first
+    const size_t o = (size_t)d.part0 + ((size_t)(w.r0 + r) * d.nsplit + w.aux) * L;
+    #pragma unroll 1
+    for (int k = 0; k < L; ++k) {
+      float bv = v[0];
+      int bi = ix[0];
+#pragma unroll
+      for (int m = 16; m >= 1; m >>= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, m);
+        const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, m);
+        if (toplist_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      if (bi != INT_MAX && bi == ix[0]) {   // the winner's owner pops its head
+#pragma unroll
+        for (int q = 0; q + 1 < LC; ++q) { v[q] = v[q + 1]; ix[q] = ix[q + 1]; }
+        v[LC - 1] = -CUDART_INF_F; ix[LC - 1] = INT_MAX;
+      }
+      if (lane == 0) {
+        part_val[o + k] = bv;
+        part_idx[o + k] = bi == INT_MAX ? -1 : bi;
+      }
+    }
   }
   correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, tile_done, part_val, part_idx, corr_cnt, tau_out,
                        e_tgt, e_w, e_c, &is_last);
