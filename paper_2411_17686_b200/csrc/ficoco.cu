@@ -891,8 +891,11 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   if (p->n_corr > 0) {
     if (rel) {
       prof_tick(c, st, "correlate_relation");
+      int rel_cols = 1;
+      for (const ImgDesc& d : p->h_desc)
+        if (d.list_len > 0 && d.cols_per_split > rel_cols) rel_cols = d.cols_per_split;
 #define FICOCO_REL_GO(LC)                                                                              \
-  k_correlate_rel<LC><<<p->n_corr, 256, 0, st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
+  k_correlate_rel<LC><<<p->n_corr, 256, (size_t)rel_cols * sizeof(int), st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
                                                  c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
                                                  c->e_w, c->e_c)
       if (p->max_list <= 2) FICOCO_REL_GO(2);

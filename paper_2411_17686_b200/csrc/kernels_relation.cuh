@@ -16,9 +16,10 @@ constexpr int RCOLS = 64;   // columns summed together in the by-column mode
 // s_i = cA * v_i - (1 - cA) * mean_h attn[h, i] for one row chunk of one image, with
 //   by_column == 0:  v_i = (1/Np) sum_j A[i, j]   (Eq. 1 as printed: row i of the map)
 //   by_column == 1:  v_i = (1/Np) sum_j A[j, i]   (the attention token i receives)
-// Row mode: two rows per warp at a time, four partial sums per row and lane.  Column mode:
-// 64 columns x 4 row phases per pass, eight partial sums per thread (eight rows in flight),
-// phases added in a fixed order.
+// Row mode: a few rows per warp at a time, partial sums per row and lane.  Column mode: 64
+// columns per pass, the rows dealt to row phases with eight rows in flight per thread, phases
+// added in a fixed order.  Blocks whose rows start on 16-byte boundaries (Np a multiple of four)
+// are read with 16-byte loads.
 __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel,
                                                    const ImgDesc* __restrict__ desc,
                                                    const WorkItem* __restrict__ work,
@@ -26,13 +27,43 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
                                                    int by_column, float* __restrict__ s_raw) {
   extern __shared__ float vrow[];            // [rows of the largest chunk]
   __shared__ float red[4][RCOLS];
+  __shared__ float4 red4[16][16];
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int np = d.np;
   const float* A = rel + d.rel0;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float inv_np = 1.0f / (float)np;
+  // 16-byte loads when every row of the block starts on a 16-byte boundary
+  const bool vec = (np & 3) == 0 && (reinterpret_cast<uintptr_t>(A) & 15) == 0;
   if (!by_column) {
+    if (vec) {
+      // four rows per warp at a time, two 16-byte loads per row and lane in flight
+      const int nv = np >> 2;
+      for (int r = 4 * warp; r < w.nrows; r += 32) {
+        float s[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int j0 = lane; j0 < nv; j0 += 64) {
+          float4 a[4][2];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float4* row = reinterpret_cast<const float4*>(A + (size_t)(w.r0 + min(r + i, w.nrows - 1)) * np);
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int j = j0 + 32 * q;
+              a[i][q] = j < nv ? __ldg(row + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            s[i] += ((a[i][0].x + a[i][0].y) + (a[i][0].z + a[i][0].w)) + ((a[i][1].x + a[i][1].y) + (a[i][1].z + a[i][1].w));
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float t = warp_sum(s[i]);
+          if (lane == 0 && r + i < w.nrows) vrow[r + i] = t * inv_np;
+        }
+      }
+    } else {
     // two rows per warp at a time, four partial sums per row and lane
     for (int r = 2 * warp; r < w.nrows; r += 16) {
       const bool two = r + 1 < w.nrows;
@@ -56,6 +87,36 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
         vrow[r] = t0 * inv_np;
         if (two) vrow[r + 1] = t1 * inv_np;
       }
+    }
+    }
+  } else if (vec && (w.r0 & 3) == 0) {
+    // 16 groups of four columns x 16 row phases per pass, eight rows in flight per thread
+    const int tx = tid & 15, ty = tid >> 4;
+    for (int c0 = 0; c0 < w.nrows; c0 += RCOLS) {
+      const int c = c0 + 4 * tx;
+      float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c < w.nrows) {     // w.r0 + c + 3 < np because both are multiples of four
+        const float* col = A + w.r0 + c;
+        for (int j0 = ty; j0 < np; j0 += 128) {
+          float4 a[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int j = j0 + 16 * q;
+            a[q] = j < np ? __ldg(reinterpret_cast<const float4*>(col + (size_t)j * np)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int q = 0; q < 8; ++q) { s4.x += a[q].x; s4.y += a[q].y; s4.z += a[q].z; s4.w += a[q].w; }
+        }
+      }
+      red4[ty][tx] = s4;
+      __syncthreads();
+      if (tid < RCOLS && c0 + tid < w.nrows) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) t += reinterpret_cast<const float*>(&red4[k][tid >> 2])[tid & 3];
+        vrow[c0 + tid] = t * inv_np;
+      }
+      __syncthreads();
     }
   } else {
     const int tx = tid & (RCOLS - 1), ty = tid / RCOLS;
@@ -91,49 +152,56 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
   }
 }
 
-// C_ij = A[S_i, T_j].  A CTA owns up to 64 discarded tokens of one image and one column split of
-// the image's preserved tokens; a warp takes one discarded token at a time.  Its lanes walk the
-// split's columns (four gathers from the token's row of the map in flight per lane), each lane
-// keeping the LC largest entries it saw (value, position in T) in registers; the warp then draws
-// the L largest of the 32 lists one by one (a shuffle tournament over the lists' heads).  The
-// partial lists and the tail (tau_i, J_i, alpha_ij by the last split of the tile) are those of
-// the fp32 correlate kernel.
+// C_ij = A[S_i, T_j].  A CTA owns a few discarded tokens of one image and one column split of
+// the image's preserved tokens, whose token indices it first copies to shared memory; a warp then
+// takes one discarded token at a time.  Its lanes walk the split's columns, eight gathers from the
+// token's row of the map in flight per lane, each lane keeping the LC largest entries it saw
+// (value, position in T) in registers; the warp then draws the L largest of the 32 lists one by
+// one (a shuffle tournament over the lists' heads).  The partial lists and the tail (tau_i, J_i,
+// alpha_ij by the last split of the tile) are those of the fp32 correlate kernel.
+constexpr int RGATHER = 8;   // gathers a lane has in flight
+
 template <int LC>
-__global__ void __launch_bounds__(256) k_correlate_rel(
+__global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
     const float* __restrict__ rel, const ImgDesc* __restrict__ desc, const WorkItem* __restrict__ work,
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ tile_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
     float* __restrict__ e_w, float* __restrict__ e_c) {
+  extern __shared__ int tcol[];              // token index of every column of the split
   __shared__ int is_last;
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int L = d.list_len, np = d.np;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const float* A = rel + d.rel0;
-  const int* tcol = T_idx + d.tgt0;
   const int col_begin = w.aux * d.cols_per_split;
-  const int col_end = min(d.n_tgt, col_begin + d.cols_per_split);
+  const int ncol = min(d.n_tgt, col_begin + d.cols_per_split) - col_begin;
+  // the rows of this warp (two at most with the planned tiles of 16) are looked up while the
+  // column indices arrive
+  const int r_first = warp < w.nrows ? S_idx[d.src0 + w.r0 + warp] : 0;
+  for (int c = threadIdx.x; c < ncol; c += 256) tcol[c] = T_idx[d.tgt0 + col_begin + c];
+  __syncthreads();
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
-    const float* row = A + (size_t)S_idx[d.src0 + w.r0 + r] * np;
+    const float* row = A + (size_t)(r == warp ? r_first : S_idx[d.src0 + w.r0 + r]) * np;
     float v[LC];
     int ix[LC];
 #pragma unroll
     for (int k = 0; k < LC; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
     #pragma unroll 1
-    for (int c0 = col_begin + lane; c0 < col_end; c0 += 128) {
-      float a[4];
+    for (int c0 = lane; c0 < ncol; c0 += 32 * RGATHER) {
+      float a[RGATHER];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < RGATHER; ++q) {
         const int c = c0 + 32 * q;
-        a[q] = c < col_end ? __ldg(row + __ldg(tcol + c)) : -CUDART_INF_F;
+        a[q] = c < ncol ? __ldg(row + tcol[c]) : -CUDART_INF_F;
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
+      for (int q = 0; q < RGATHER; ++q) {
         float cv = a[q];
-        int ci = c0 + 32 * q;
-        if (ci >= col_end) continue;
+        int ci = col_begin + c0 + 32 * q;
+        if (c0 + 32 * q >= ncol) continue;
 #pragma unroll
         for (int k = 0; k < LC; ++k) {     // sorted insertion: the displaced entry moves down
           if (toplist_better(cv, ci, v[k], ix[k])) {
@@ -166,8 +234,8 @@ __global__ void __launch_bounds__(256) k_correlate_rel(
       }
     }
   }
-  correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, tile_done, part_val, part_idx, corr_cnt, tau_out,
-                       e_tgt, e_w, e_c, &is_last);
+  correlate_tail<LC>(d, w, (int)blockIdx.x - w.aux, tile_done, part_val, part_idx, corr_cnt, tau_out,
+                     e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco

@@ -134,6 +134,15 @@ def test_relation_mode(ctx, by_column, dtype):
         parity.run_and_compare_v_relation(ctx, batch, rels, by_column, p, DEV, what="relation")
 
 
+@pytest.mark.parametrize("by_column", [False, True], ids=["by-row", "by-column"])
+def test_relation_mode_rows_on_16_byte_boundaries(ctx, by_column):
+    """Np a multiple of four: the score kernel reads the map with 16-byte loads."""
+    batch = synth.make_v_batch(93, 2, 12, 12, 128, 3, 50, "bf16", True, 1.0)
+    rels = _relations(batch, 93, stochastic=by_column)
+    gaps.repair_v_relation(batch, rels, by_column)
+    parity.run_and_compare_v_relation(ctx, batch, rels, by_column, fo.Params(), DEV, what="relation-vec")
+
+
 def test_relation_mode_ragged_no_cls(ctx):
     batch = synth.workload(4, small=True)
     rels = _relations(batch, 91, times_n=True)
