@@ -883,7 +883,8 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   }
   const size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
   prof_tick(c, st, "select");
-  k_select<<<p->key.batch, 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
+  // images of up to 1024 tokens: half the threads (two tokens each), cheaper barriers
+  k_select<<<p->key.batch, p->max_np <= 1024 ? 512 : 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
                                                   pos_out, c->status);
   c->launches += 1;

@@ -400,7 +400,7 @@ __device__ __noinline__ void select_image(
     kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
 }
 
-// One CTA (1024 threads) per image.
+// One CTA (512 or 1024 threads) per image.
 __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ desc,
                                                  const float* __restrict__ s_raw,
                                                  const int* __restrict__ pos, int window, float coef,
@@ -413,7 +413,7 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
   __shared__ SelectShared sh;
   const ImgDesc d = desc[blockIdx.x];
   select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-               status, sm_raw, sh, threadIdx.x, 1024, 0);
+               status, sm_raw, sh, threadIdx.x, (int)blockDim.x, 0);
 }
 
 }  // namespace ficoco

@@ -12,6 +12,7 @@
 namespace ficoco {
 
 constexpr int RCOLS = 64;   // columns summed together in the by-column mode
+constexpr int RINF = 12;    // 16-byte loads a thread has in flight in the by-column mode
 
 // s_i = cA * v_i - (1 - cA) * mean_h attn[h, i] for one row chunk of one image, with
 //   by_column == 0:  v_i = (1/Np) sum_j A[i, j]   (Eq. 1 as printed: row i of the map)
@@ -90,22 +91,22 @@ __global__ void __launch_bounds__(256) k_score_rel(const float* __restrict__ rel
     }
     }
   } else if (vec && (w.r0 & 3) == 0) {
-    // 16 groups of four columns x 16 row phases per pass, eight rows in flight per thread
+    // 16 groups of four columns x 16 row phases per pass, RINF rows in flight per thread
     const int tx = tid & 15, ty = tid >> 4;
     for (int c0 = 0; c0 < w.nrows; c0 += RCOLS) {
       const int c = c0 + 4 * tx;
       float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
       if (c < w.nrows) {     // w.r0 + c + 3 < np because both are multiples of four
         const float* col = A + w.r0 + c;
-        for (int j0 = ty; j0 < np; j0 += 128) {
-          float4 a[8];
+        for (int j0 = ty; j0 < np; j0 += 16 * RINF) {
+          float4 a[RINF];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
+          for (int q = 0; q < RINF; ++q) {
             const int j = j0 + 16 * q;
             a[q] = j < np ? __ldg(reinterpret_cast<const float4*>(col + (size_t)j * np)) : make_float4(0.f, 0.f, 0.f, 0.f);
           }
 #pragma unroll
-          for (int q = 0; q < 8; ++q) { s4.x += a[q].x; s4.y += a[q].y; s4.z += a[q].z; s4.w += a[q].w; }
+          for (int q = 0; q < RINF; ++q) { s4.x += a[q].x; s4.y += a[q].y; s4.z += a[q].z; s4.w += a[q].w; }
         }
       }
       red4[ty][tx] = s4;
