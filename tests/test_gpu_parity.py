@@ -355,6 +355,15 @@ def test_full_c2_schedule(ctx):
             synth.regenerate_attention(batch, 2000, step + 1, 1.5)
 
 
+@pytest.mark.parametrize("by_column", [True, False], ids=["by-column", "by-row"])
+def test_full_c2_shape_relation_mode(ctx, by_column):
+    """The shape bench.py times for the relation mode: 32 images, 576 x 576 maps."""
+    batch = synth.workload(2)
+    rels = _relations(batch, 94, stochastic=by_column, times_n=True)
+    gaps.repair_v_relation(batch, rels, by_column)
+    parity.run_and_compare_v_relation(ctx, batch, rels, by_column, fo.Params(), DEV, what="c2-relation")
+
+
 def test_full_c3_first_step(ctx):
     batch = synth.workload(3)
     gaps.repair_v(batch)
