@@ -577,6 +577,19 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     want_split = best.want_split;
   }
 
+  // output rows per merge CTA: fewer than the usual 16 when that would leave most SMs with less
+  // than two CTAs (few or very wide rows), as far as the work table goes
+  int out_rows_cta = OUT_ROWS_PER_CTA;
+  {
+    auto n_out_ctas = [&](int r) {
+      long long n = 0;
+      for (int b = 0; b < B; ++b) n += (cls + key.keep[b] + tail + r - 1) / r;
+      return n;
+    };
+    while (out_rows_cta > 2 && n_out_ctas(out_rows_cta) < 2LL * c->num_sms &&
+           n_out_ctas(out_rows_cta / 2) <= c->cap_out)
+      out_rows_cta /= 2;
+  }
   for (int b = 0; b < B; ++b) {
     ImgDesc& d = p->h_desc[b];
     d.row0 = (int)row0; d.patch0 = (int)patch0; d.out_row0 = (int)out0;
@@ -629,8 +642,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     }
     // output rows
     const int orows = d.n_cls + d.n_tgt + d.n_tail;
-    for (int r0 = 0; r0 < orows; r0 += OUT_ROWS_PER_CTA) {
-      WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < OUT_ROWS_PER_CTA) ? orows - r0 : OUT_ROWS_PER_CTA; w.aux = 0;
+    for (int r0 = 0; r0 < orows; r0 += out_rows_cta) {
+      WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < out_rows_cta) ? orows - r0 : out_rows_cta; w.aux = 0;
       outw.push_back(w);
     }
     row0 += key.ntok[b]; patch0 += d.np; out0 += orows; src0 += d.n_src; tgt0 += d.n_tgt;

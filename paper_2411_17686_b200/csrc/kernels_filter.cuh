@@ -200,7 +200,13 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
   float* dst = t + ((size_t)b * M + k) * N;
   for (int i = threadIdx.x; i < N; i += 256) {
     float s = 0.f;
-    for (int h = 0; h < H; ++h) s += __ldg(src + (size_t)h * M * N + i);
+    for (int h0 = 0; h0 < H; h0 += 8) {      // eight heads in flight, added in head order
+      float a[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) a[q] = h0 + q < H ? __ldg(src + (size_t)(h0 + q) * M * N + i) : 0.f;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) s += a[q];
+    }
     dst[i] = s * inv_h;
   }
 }
