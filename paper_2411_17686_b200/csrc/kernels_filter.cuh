@@ -21,11 +21,20 @@ __global__ void __launch_bounds__(256) k_rownorm(const T* __restrict__ tokens, i
   for (int r = warp; r < w.nrows; r += 8) {
     const T* row = tokens + (size_t)(d.row0 + d.n_cls + w.r0 + r) * D;
     float ss = 0.f;
-    for (int v = lane; v < nvec; v += 32) {
-      float f[E];
-      unpack(ldg16(row + (size_t)v * E), f, (const T*)nullptr);
+    for (int v0 = lane; v0 < nvec; v0 += 32 * 8) {     // eight 16-byte loads in flight per lane
+      uint4 u[8];
 #pragma unroll
-      for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
+      for (int k = 0; k < 8; ++k) {
+        const int v = v0 + 32 * k;
+        u[k] = v < nvec ? ldg16(row + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        float f[E];
+        unpack(u[k], f, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
+      }
     }
     ss = warp_sum(ss);
     if (lane == 0) rn[d.patch0 + w.r0 + r] = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
@@ -167,12 +176,24 @@ __global__ void __launch_bounds__(256) k_score(const T* __restrict__ tokens, int
   for (int r = warp; r < w.nrows; r += 8) {
     const T* row = tokens + (size_t)(d.row0 + d.n_cls + w.r0 + r) * D;
     float dot = 0.f;
-    for (int v = lane; v < nvec; v += 32) {
-      float f[E];
-      unpack(ldg16(row + (size_t)v * E), f, (const T*)nullptr);
-      const float* m = msum + (size_t)v * E;
+    for (int v0 = lane; v0 < nvec; v0 += 32 * 8) {     // eight 16-byte loads in flight per lane
+      uint4 u[8];
 #pragma unroll
-      for (int e = 0; e < E; ++e) dot = fmaf(f[e], m[e], dot);
+      for (int k = 0; k < 8; ++k) {
+        const int v = v0 + 32 * k;
+        u[k] = v < nvec ? ldg16(row + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int v = v0 + 32 * k;
+        if (v < nvec) {
+          float f[E];
+          unpack(u[k], f, (const T*)nullptr);
+          const float* m = msum + (size_t)v * E;
+#pragma unroll
+          for (int e = 0; e < E; ++e) dot = fmaf(f[e], m[e], dot);
+        }
+      }
     }
     dot = warp_sum(dot);
     if (lane == 0) vrow[r] = dot * rn[d.patch0 + w.r0 + r] * inv_np;
