@@ -31,7 +31,7 @@ WORKLOAD = "c2 step 1: 32 images x (1 CLS + 24x24 patches) x 1024 bf16, 576 -> 2
 N_INSTANCES = 8       # distinct input/output buffer sets cycled through: 8 x 58 MB > 3 x L2
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (bytes); an entry is removed when its kernel changes after the capture.
-NCU_TRAFFIC = {"filter_fused": 39074560 + 6400, "correlate_umma": 37964800 + 1792, "merge_compact": 37891072 + 61440}
+NCU_TRAFFIC = {"filter_fused": 39075072, "correlate_umma": 37965056, "merge_compact": 37890560 + 66816}
 
 
 def algorithmic_bytes() -> dict:
