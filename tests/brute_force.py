@@ -14,7 +14,7 @@ def _dot(a, b):
 
 
 def reduce_v(P, cls_attn_heads, pos, gh, gw, keep, lam=0.35, eps=0.998, coef=2.0, window=2,
-             penalty=True):
+             penalty=True, max_targets=None):
     """P: list of patch rows (lists of floats); cls_attn_heads: list over heads of lists.
     Returns dict with scores, S (set), T (sorted list), J, alpha, merged rows (floats)."""
     n = len(P)
@@ -42,10 +42,10 @@ def reduce_v(P, cls_attn_heads, pos, gh, gw, keep, lam=0.35, eps=0.998, coef=2.0
     ranked = sorted(range(n), key=lambda i: (-s[i], i))
     S = ranked[:n_src]
     T = sorted(set(range(n)) - set(S))
-    return _correlate_compress(P, S, T, lambda i, j: A[i][j], eps, s_raw, s)
+    return _correlate_compress(P, S, T, lambda i, j: A[i][j], eps, s_raw, s, max_targets)
 
 
-def reduce_l(P, t2v_heads, keep, beta=0.6, gamma=0.6, eps=0.998):
+def reduce_l(P, t2v_heads, keep, beta=0.6, gamma=0.6, eps=0.998, max_targets=None):
     """P: vision rows; t2v_heads[h][k][i]: attention of text token k to vision token i."""
     n = len(P)
     H = len(t2v_heads)
@@ -67,24 +67,33 @@ def reduce_l(P, t2v_heads, keep, beta=0.6, gamma=0.6, eps=0.998):
         bridge = math.fsum(t[k][i] * t[k][j] for k in range(M)) / M
         return gamma * A[i][j] + (1.0 - gamma) * bridge
 
-    return _correlate_compress(P, S, T, corr, eps, list(s), s)
+    return _correlate_compress(P, S, T, corr, eps, list(s), s, max_targets)
 
 
-def _correlate_compress(P, S, T, corr, eps, s_raw, s):
+def _correlate_compress(P, S, T, corr, eps, s_raw, s, max_targets=None):
+    """max_targets None: the token-wise quantile threshold; k >= 0: the fixed-K ablation, every
+    discarded token goes to its k most correlated preserved tokens (ties: lower token first)."""
     D = len(P[0])
     C = {(i, j): corr(i, j) for i in S for j in T}
     J = {}
     alpha = {}
+    taus = {}
     for i in S:
-        if not T:
+        if not T or max_targets == 0:
             J[i] = []
             continue
-        row = sorted(C[(i, j)] for j in T)
-        q = eps * (len(row) - 1)
-        lo = int(math.floor(q))
-        hi = min(lo + 1, len(row) - 1)
-        tau = row[lo] + (q - lo) * (row[hi] - row[lo])
-        Ji = [j for j in T if C[(i, j)] >= tau]
+        if max_targets is None:
+            row = sorted(C[(i, j)] for j in T)
+            q = eps * (len(row) - 1)
+            lo = int(math.floor(q))
+            hi = min(lo + 1, len(row) - 1)
+            tau = row[lo] + (q - lo) * (row[hi] - row[lo])
+            Ji = [j for j in T if C[(i, j)] >= tau]
+        else:
+            best = sorted(T, key=lambda j: (-C[(i, j)], j))[:min(max_targets, len(T))]
+            tau = C[(i, best[-1])]              # the smallest correlation that is still taken
+            Ji = sorted(best)
+        taus[i] = tau
         den = math.fsum(max(C[(i, j)], 0.0) for j in Ji)
         if den <= 1e-12:
             J[i] = []
@@ -104,7 +113,7 @@ def _correlate_compress(P, S, T, corr, eps, s_raw, s):
         merged[j] = row
         wsum[j] = w
     return {"s_raw": s_raw, "s": s, "S": S, "T": T, "J": J, "alpha": alpha, "merged": merged,
-            "wsum": wsum, "C": C}
+            "wsum": wsum, "C": C, "tau": taus}
 
 
 def group_means(P, S, T, J):

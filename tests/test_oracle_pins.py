@@ -44,6 +44,59 @@ def test_hand_worked_example():
         assert r.kept_idx.tolist() == g["T"]
 
 
+def _golden():
+    return json.load(open(os.path.join(HERE, "golden", "hand_example.json")))
+
+
+def check_fixed_k_hand_cases():
+    """Fixed K on the hand-worked example: K = 1 is its eps = 1 case, K = 2 = N^T its eps = 0 case,
+    and tau_i is the smallest correlation still taken."""
+    g = _golden()
+    P = np.array(g["patches"], dtype=np.float32)
+    attn = np.array(g["cls_attention"], dtype=np.float32)
+    for case in g["fixed_k_cases"]:
+        p = fo.Params(lam=g["lambda"], local_penalty=False, max_targets=case["max_targets"])
+        r = fo.ficoco_v_reduce(P, attn, None, (2, 2), g["keep"], has_cls=False, p=p)
+        order = np.argsort(r.S)
+        for k, si in enumerate(order):
+            assert r.J[si].tolist() == case["J"][k]
+            np.testing.assert_allclose(r.alpha[si], case["alpha"][k], atol=1e-12)
+            np.testing.assert_allclose(r.tau[si], case["tau"][k], atol=1e-12)
+        np.testing.assert_allclose(r.out.astype(np.float64), case["merged"], rtol=1e-6)
+
+
+def check_tie_hand_cases():
+    """Equal scores: across the selection boundary the lower token index is discarded; inside a
+    local-penalty window the lower token index is the one multiplied."""
+    t = _golden()["tie_cases"]
+    P = np.array(t["patches"], dtype=np.float32)
+    attn = np.array(t["cls_attention"], dtype=np.float32)
+    for c in t["selection"]:
+        r = fo.ficoco_v_reduce(P, attn, None, (2, 2), c["keep"], False, fo.Params(lam=t["lambda"], local_penalty=False))
+        np.testing.assert_allclose(r.score, t["score"], atol=1e-8)
+        assert r.score[0] == r.score[1] and r.score[2] == r.score[3]
+        assert sorted(r.S.tolist()) == c["S"] and r.T.tolist() == c["T"]
+        assert r.kept_idx.tolist() == c["T"]
+    w = t["window"]
+    r = fo.ficoco_v_reduce(P, attn, None, tuple(w["grid"]), w["keep"], False,
+                           fo.Params(lam=t["lambda"], window=w["window"], penalty_coef=w["coef"]))
+    np.testing.assert_allclose(r.score, w["score_after_penalty"], atol=1e-8)
+    assert sorted(r.S.tolist()) == w["S"] and r.T.tolist() == w["T"]
+    wo = t["window_only"]
+    out = fo.local_penalty(np.array(wo["scores"]), np.array(wo["pos"]), tuple(wo["grid"]), wo["window"], wo["coef"])
+    assert out.tolist() == wo["expected"]
+    # the selection helper on its own, ties inside and across the boundary
+    S, T = fo.filter_topk(np.array([0.3, 0.5, 0.5, 0.1, 0.5]), 2)
+    assert S.tolist() == [1, 2] and T.tolist() == [0, 3, 4]
+    S, T = fo.filter_topk(np.array([0.5, 0.5, 0.5]), 1)
+    assert S.tolist() == [0] and T.tolist() == [1, 2]
+
+
+def test_fixed_k_and_tie_hand_cases():
+    check_fixed_k_hand_cases()
+    check_tie_hand_cases()
+
+
 # ---------------------------------------------------------------------------
 # independent scalar-loop transcription on tiny inputs
 # ---------------------------------------------------------------------------
@@ -60,6 +113,8 @@ def _compare_with_brute(r, b, P64):
             assert abs(a - b["alpha"][(i, Tl[jj])]) < 1e-12
         for jj, j in enumerate(Tl):
             assert abs(r.C[k, jj] - b["C"][(i, j)]) < 1e-12
+        if i in b["tau"]:
+            assert abs(r.tau[k] - b["tau"][i]) < 1e-12
     return Tl
 
 
@@ -98,6 +153,112 @@ def test_l_matches_brute_force(seed, eps):
     # text rows pass through untouched after the preserved vision rows
     assert np.array_equal(r.out[len(Tl):], lb.tokens[0][14:])
     assert r.kept_idx.tolist() == Tl + list(range(14, 19))
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+@pytest.mark.parametrize("kfix", [0, 1, 2, 3, 8, 11])
+def test_fixed_k_matches_brute_force_v(seed, kfix):
+    """Fixed-K ablation (every discarded token to its K most correlated targets) against the
+    scalar transcription, K from 0 (pruning) to beyond N^T = 8."""
+    batch = tiny_v(seed)
+    tok, attn = batch.tokens[0], batch.attn[0]
+    r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 8, True, fo.Params(max_targets=kfix))
+    P = tok[1:].astype(np.float64)
+    b = bf.reduce_v(P.tolist(), attn.astype(np.float64).tolist(), list(range(16)), 4, 4, 8, max_targets=kfix)
+    Tl = _compare_with_brute(r, b, P)
+    assert all(len(j) == min(kfix, 8) for j in r.J) or kfix == 0
+    for jj, j in enumerate(Tl):
+        np.testing.assert_allclose(r.out[1 + jj].astype(np.float64), b["merged"][j], rtol=2e-7, atol=1e-7)
+
+
+@pytest.mark.parametrize("kfix", [1, 2, 3, 9])
+def test_fixed_k_matches_brute_force_l(kfix):
+    lb = synth.make_l_batch(14, 1, 14, 5, 8, 3, 6, "fp32", scale=1.0)
+    r = fo.ficoco_l_reduce(lb.tokens[0], lb.attn_t2v[0], 14, 6, fo.Params(max_targets=kfix))
+    P = lb.tokens[0][:14].astype(np.float64)
+    b = bf.reduce_l(P.tolist(), lb.attn_t2v[0].astype(np.float64).tolist(), 6, max_targets=kfix)
+    Tl = _compare_with_brute(r, b, P)
+    for jj, j in enumerate(Tl):
+        np.testing.assert_allclose(r.out[jj].astype(np.float64), b["merged"][j], rtol=2e-7, atol=1e-7)
+
+
+def test_fixed_k_ties_go_to_the_lower_column():
+    C = np.array([[0.5, 0.9, 0.9, 0.1], [0.2, 0.2, 0.2, 0.2]])
+    J, A, tau = fo.targets_and_weights(C, fo.Params(max_targets=1))
+    assert J[0].tolist() == [1] and J[1].tolist() == [0] and tau.tolist() == [0.9, 0.2]
+    J, A, tau = fo.targets_and_weights(C, fo.Params(max_targets=3))
+    assert J[0].tolist() == [0, 1, 2] and J[1].tolist() == [0, 1, 2] and tau.tolist() == [0.5, 0.2]
+    np.testing.assert_allclose(A[0], np.array([0.5, 0.9, 0.9]) / 2.3, atol=1e-15)
+
+
+def test_planted_mistakes_in_fixed_k_and_tie_rules_are_caught(monkeypatch):
+    """The fixed-K branch and the two tie rules, each flipped in the checker, must break a pin."""
+    real_tw, real_topk, real_pen = fo.targets_and_weights, fo.filter_topk, fo.local_penalty
+
+    def fails(check):
+        try:
+            check()
+        except AssertionError:
+            return True
+        return False
+
+    def brute_k():
+        batch = tiny_v(2)
+        tok, attn = batch.tokens[0], batch.attn[0]
+        P = tok[1:].astype(np.float64)
+        for kfix in (1, 2, 3):
+            r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 8, True, fo.Params(max_targets=kfix))
+            b = bf.reduce_v(P.tolist(), attn.astype(np.float64).tolist(), list(range(16)), 4, 4, 8, max_targets=kfix)
+            Tl = _compare_with_brute(r, b, P)
+            for jj, j in enumerate(Tl):
+                np.testing.assert_allclose(r.out[1 + jj].astype(np.float64), b["merged"][j], rtol=2e-7, atol=1e-7)
+
+    assert not fails(brute_k) and not fails(check_fixed_k_hand_cases) and not fails(check_tie_hand_cases)
+
+    def tw_variant(kind):
+        def wrong(C, p):
+            if p.max_targets is None or p.max_targets == 0:
+                return real_tw(C, p)
+            J, A, tau = [], [], np.full(C.shape[0], np.nan)
+            for i in range(C.shape[0]):
+                row = C[i]
+                k = min(p.max_targets, C.shape[1])
+                if kind == "one_more":
+                    order = np.argsort(-row, kind="stable")[:k + 1]
+                elif kind == "ascending":
+                    order = np.argsort(row, kind="stable")[:k]
+                else:
+                    order = np.argsort(-row, kind="stable")[:k]
+                tau[i] = row[order[0]] if kind == "tau_first" else row[order[-1]]
+                j = np.sort(order)
+                cpos = np.maximum(row[j], 0.0)
+                J.append(j.astype(np.int64)); A.append(cpos / max(cpos.sum(), 1e-300))
+            return J, A, tau
+        return wrong
+
+    for kind in ("one_more", "ascending", "tau_first"):
+        with monkeypatch.context() as m:
+            m.setattr(fo, "targets_and_weights", tw_variant(kind))
+            assert fails(brute_k), f"fixed-K mistake '{kind}' passes the scalar transcription"
+            assert fails(check_fixed_k_hand_cases), f"fixed-K mistake '{kind}' passes the hand example"
+
+    def topk_high(s, n_src):     # ties to the higher index
+        order = np.argsort(-s[::-1], kind="stable")
+        S = (s.shape[0] - 1 - order)[:n_src]
+        mask = np.ones(s.shape[0], dtype=bool)
+        mask[S] = False
+        return S.astype(np.int64), np.nonzero(mask)[0].astype(np.int64)
+
+    def penalty_high(s, pos, grid, window, coef):   # ties inside a window to the higher index
+        n = s.shape[0]
+        return real_pen(s[::-1].copy(), np.asarray(pos)[::-1].copy(), grid, window, coef)[::-1].copy()
+
+    with monkeypatch.context() as m:
+        m.setattr(fo, "filter_topk", topk_high)
+        assert fails(check_tie_hand_cases), "selection tie rule flipped, no pin noticed"
+    with monkeypatch.context() as m:
+        m.setattr(fo, "local_penalty", penalty_high)
+        assert fails(check_tie_hand_cases), "window tie rule flipped, no pin noticed"
 
 
 def test_planted_mistakes_are_caught(monkeypatch):
@@ -346,6 +507,12 @@ def test_untouched_rows_keep_their_bits_and_bf16_rounding():
     ref = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(mine, ref)
     assert np.array_equal(fo.widen(mine), synth.bf16_bits_to_f32(mine).astype(np.float64))
+    # widening against torch's own reinterpretation of the bits as bfloat16, all finite patterns
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    finite = (bits & 0x7F80) != 0x7F80
+    tw = torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy()
+    assert np.array_equal(fo.widen(bits[finite]), tw[finite])
+    assert np.array_equal(np.signbit(fo.widen(bits[finite])), np.signbit(tw[finite]))
 
 
 def test_ficoco_l_special_cases():
