@@ -29,6 +29,8 @@ UNIT = "images/s"
 B, GH, GW, D, H, KEEP = 32, 24, 24, 1024, 16, 288
 WORKLOAD = "c2 step 1: 32 images x (1 CLS + 24x24 patches) x 1024 bf16, 576 -> 288 patch tokens"
 N_INSTANCES = 8       # distinct input/output buffer sets cycled through: 8 x 58 MB > 3 x L2
+MIN_TIMED_MS = 50.0   # device time the timed repetitions add up to, at least
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # vendor figures, reported beside the measured peaks
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (bytes); an entry is removed when its kernel changes after the capture.
 NCU_TRAFFIC = {"filter_fused": 39075072, "correlate_umma": 37965056, "merge_compact": 37890560 + 66816}
@@ -277,6 +279,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             pout=torch.empty((B * KEEP,), dtype=torch.int32, device=dev)))
     ctx = binding.Context(max_tokens=B * n, max_dim=D, max_batch=B, device=local_rank)
     prm = binding.ficoco_default_params()
+    prm.flags |= binding.FICOCO_BACK_TO_BACK     # the timed stream carries nothing but reduce steps
     stream = torch.cuda.Stream(device=dev)
 
     def step(i: int):
@@ -296,35 +299,72 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     torch.cuda.synchronize()
     launches_per_step = ctx.ficoco_last_launch_count()
 
-    # optional CUDA graph over one cycle of the instances (launch overhead off the GPU timeline)
-    graph = None
-    if args.graph and args.steps % N_INSTANCES == 0:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=stream):
-            for i in range(N_INSTANCES):
+    # The timed steps are always replayed from CUDA graphs (the host's launch cost stays off the GPU
+    # timeline whatever --steps is): one graph of a full cycle over the buffer sets, one of the
+    # steps % N_INSTANCES remaining steps, together exactly `steps` steps per repetition.
+    def capture(n_steps: int):
+        if n_steps == 0:
+            return None
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(n_steps):
                 step(i)
-        graph.replay()
+        return g
+
+    graph = rem_graph = None
+    if args.graph:
+        graph = capture(N_INSTANCES) if args.steps >= N_INSTANCES else None
+        rem_graph = capture(args.steps % N_INSTANCES)
+        with torch.cuda.stream(stream):
+            for g in (graph, rem_graph):
+                if g is not None:
+                    g.replay()
         torch.cuda.synchronize()
+
+    def run_steps():
+        if not args.graph:
+            for i in range(args.steps):
+                step(i)
+            return
+        for _ in range(args.steps // N_INSTANCES):
+            graph.replay()
+        if rem_graph is not None:
+            rem_graph.replay()
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # The `steps`-step region is repeated until at least MIN_TIMED_MS of device time has been timed
+    # (at least 3, at most 400 repetitions); every repetition is bracketed by its own pair of events
+    # and the reported time per step is the median over the repetitions.
+    reps = []
     barrier()
     with torch.cuda.stream(stream):
-        e0.record(stream)
-        if graph is not None:
-            for _ in range(args.steps // N_INSTANCES):
-                graph.replay()
-        else:
-            for i in range(args.steps):
-                step(i)
-        e1.record(stream)
+        probe0, probe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        probe0.record(stream)
+        run_steps()
+        probe1.record(stream)
+    torch.cuda.synchronize()
+    est_ms = max(probe0.elapsed_time(probe1), 1e-3)
+    n_rep = int(min(400, max(3, np.ceil(MIN_TIMED_MS / est_ms))))
+    if world > 1:                       # every rank runs the same number of repetitions
+        t = torch.tensor([n_rep], dtype=torch.int64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        n_rep = int(t.item())
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_rep)]
     barrier()
-    ms = e0.elapsed_time(e1)
+    with torch.cuda.stream(stream):
+        for a, b in evs:
+            a.record(stream)
+            run_steps()
+            b.record(stream)
+    barrier()
+    reps = [a.elapsed_time(b) for a, b in evs]
     clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms, world, dev)
+    ms = max_over_ranks(float(np.median(reps)), world, dev)
+    ms_min = max_over_ranks(float(np.min(reps)), world, dev)
+    ms_max = max_over_ranks(float(np.max(reps)), world, dev)
     ms_per_step = ms / args.steps
     value = aggregate_images_per_s(ms_per_step, world)
 
@@ -403,7 +443,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": B, "tokens_per_image": n, "dim": D, "heads": H,
                    "keep": KEEP, "l2": f"inputs larger than L2: {N_INSTANCES} buffer sets cycled",
-                   "cuda_graph": graph is not None},
+                   "cuda_graph": bool(args.graph), "repetitions": n_rep,
+                   "ms_per_step_min": ms_min / args.steps, "ms_per_step_max": ms_max / args.steps,
+                   "timed_ms": float(np.sum(reps)),
+                   "stream": "reduce steps only, FICOCO_BACK_TO_BACK set"},
         "tokens_per_s": value * n,
         "clocks": clocks,
         "equivalent_token": eq_info,
@@ -414,7 +457,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "roofline": roof,
         "step_roofline": {"bound": "hbm" if ab["total"] / (pk["hbm_gbs"] * 1e3) >= t_roof_us - 1e-9 else "tensor",
                           "t_roof_us": t_roof_us, "t_measured_us": ms_per_step * 1e3,
-                          "frac": t_roof_us / (ms_per_step * 1e3), "algorithmic_bytes": ab["total"],
+                          "frac": t_roof_us / (ms_per_step * 1e3),
+                          "frac_of_nominal": max(ab["total"] / (NOMINAL["hbm_gbs"] * 1e3),
+                                                 2.0 * B * (GH * GW - KEEP) * KEEP * D / (NOMINAL["bf16_tflops"] * 1e6))
+                          / (ms_per_step * 1e3),
+                          "algorithmic_bytes": ab["total"],
                           "peak": f"{pk['source']} {pk['hbm_gbs']} GB/s, {pk['bf16_tflops']} TFLOP/s bf16"},
         "kernels": kern,
     }
@@ -476,13 +523,13 @@ def cpu_baseline(batch, budget_s: float = 12.0) -> dict:
 
 
 def run_reference(args, rank: int):
-    """Reference arm: the float64 checker on the host cores, each step a bounded sample
-    (4 images) of the workload."""
+    """Reference arm: the float64 checker on the host cores, each step one whole batch of the
+    workload (all 32 images, about a quarter of a second)."""
     if rank != 0:
         return None
     from oracle import ficoco_oracle as fo
     batch = make_instances(0)
-    sample = 4
+    sample = B
     cores = os.cpu_count() or 1
     try:
         from threadpoolctl import threadpool_info
@@ -506,11 +553,42 @@ def run_reference(args, rank: int):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample_per_step": f"{sample} of {B} images"},
+        "config": {"workload": WORKLOAD, "batch_per_gpu": B, "tokens_per_image": 1 + GH * GW, "dim": D, "heads": H,
+                   "keep": KEEP, "sample_per_step": f"all {B} images of a batch"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{sample} images per step, {args.steps} steps"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
+
+
+def spawn_ranks(n: int, argv) -> int:
+    """`bench.py --gpus N` started as a plain process: start N ranks of this file, one per GPU,
+    the way the multi-GPU launch line does (torch.distributed.run on 127.0.0.1), and pass their
+    output through."""
+    port = 29500 + os.getpid() % 2000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def run_dry(args, rank: int, world: int):
+    """The N > 1 plumbing without a GPU: a gloo group, one shard seed per rank, a made-up step time
+    per rank (rank r: 10 + 5 r ms for `steps` steps), the max over ranks and the aggregate."""
+    import torch.distributed as dist
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("gloo")
+    ms = max_over_ranks(10.0 + 5.0 * rank, world)
+    seeds = [shard_seed(r) for r in range(world)]
+    line = None
+    if rank == 0:
+        line = {"metric": METRIC, "dry_run": True, "n_gpus": world, "steps": args.steps, "unit": UNIT,
+                "ms_per_step": ms / args.steps, "value": aggregate_images_per_s(ms / args.steps, world),
+                "scaling": "weak", "shard_seeds": seeds}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return line
 
 
 def main():
@@ -523,7 +601,11 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-extras", dest="extras", action="store_false",
                     help="skip the schedule / other-workload timings that follow the headline measurement")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="exercise the multi-rank plumbing on CPU (gloo, no kernels): ranks, shards, max-over-ranks")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -536,6 +618,11 @@ def main():
         return
     args.steps = args.steps if args.steps is not None else 2000
     args.warmup = args.warmup if args.warmup is not None else 10
+    if args.dry_run:
+        line = run_dry(args, rank, world)
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return
     if world > 1:
         import torch
         import torch.distributed as dist

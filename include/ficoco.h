@@ -35,6 +35,11 @@
  *   - Every function returns FICOCO_OK (0) or a negative ficoco_error; nothing is launched
  *     when argument validation fails.  Problems only the device can see (a `pos` entry
  *     outside the grid) set bits in a status word read by ficoco_status.
+ *   - No output buffer may overlap an input buffer of the same call (Eq. 2 reads the tokens
+ *     as they were before the update); such a call returns FICOCO_ERR_INVALID_ARG.
+ *   - Device-side waits (between the thread blocks of one kernel) are bounded by elapsed time.
+ *     Should one run out, the step stops writing, bit 2 of the status word is raised, and every
+ *     later step of the context does nothing until ficoco_status has read and cleared it.
  *   - Token rows must be 16-byte aligned: dim % 8 == 0 for bf16, dim % 4 == 0 for fp32.
  *     A token row of all zeros has no direction; its cosine is taken as 0.
  *   - At most 8192 vision tokens per image; the top list needed for tau_i,
@@ -69,10 +74,19 @@ enum ficoco_error {
 enum ficoco_flags {
   FICOCO_HAS_CLS = 1u,           /* row 0 of every image is a CLS token: never scored, always kept */
   FICOCO_LOCAL_PENALTY = 2u,     /* apply the local penalty (FiCoCo-V default) */
-  FICOCO_AVERAGE_COMPRESSION = 4u /* ablation "average compression" (Sec. "Ablation Study", Compress:
+  FICOCO_AVERAGE_COMPRESSION = 4u, /* ablation "average compression" (Sec. "Ablation Study", Compress:
                                     the features are averaged directly): every alpha_ij of Eq. 2
                                     is 1, so a preserved token becomes the plain mean of itself
                                     and the discarded tokens sent to it; J_i is unchanged */
+  FICOCO_BACK_TO_BACK = 8u       /* scheduling hint, no effect on results: the caller states that the
+                                    work enqueued on the stream right before this call is the
+                                    previous reduce step of this library (any context) and nothing
+                                    else.  The step's first kernel may then start reading tokens
+                                    and attention while that previous step is still finishing,
+                                    provided its inputs do not overlap that step's outputs (the
+                                    library checks the address ranges).  Without the flag every
+                                    step starts in plain stream order, which is what a stream
+                                    that also carries other kernels needs. */
 };
 
 /* Hyper-parameters; defaults are the paper's (Sec. "Implementation Details"):
@@ -206,9 +220,16 @@ int ficoco_l_reduce_host(ficoco_ctx* ctx, const ficoco_l_args* host_args,
 
 /* Synchronise `cuda_stream`, read and clear the device status word into *device_status
  * (0 = clean; bit 0 (1): a pos entry outside grid_h*grid_w was ignored by the local penalty;
- * bit 2 (4): a bounded wait inside the tensor-core correlate kernel ran out, the step's
- * outputs are then invalid). */
+ * bit 2 (4): a bounded device-side wait ran out: the outputs of that step and of every step
+ * enqueued after it are invalid).  Returns FICOCO_OK when the word could be read, whatever it
+ * holds. */
 int ficoco_status(ficoco_ctx* ctx, void* cuda_stream, int* device_status);
+
+/* Testing hook for the bounded waits.  wait_ns > 0 sets the time after which a device-side wait
+ * of this context gives up (default 20 ms); extra_arrivals > 0 makes the fused filter kernel wait
+ * for that many arrivals more than will ever come, so that the wait runs out by itself (nothing
+ * spins past the bound, nothing faults); 0 restores normal operation.  Affects later calls. */
+int ficoco_debug_waits(ficoco_ctx* ctx, long long wait_ns, int extra_arrivals);
 
 /*
  * Inspection of the intermediate results of the most recent reduce call on this context

@@ -29,6 +29,11 @@ Readings taken where the paper is silent:
   * all preserved tokens are updated at once from the pre-update X;
   * "average compression" (ablation tables; "directly averaging the features") keeps J_i as
     it is and sets every alpha_ij to 1, whatever the sign of C_ij;
+  * "convergent correlation" (ablation tables; Sec. "Correlation-based Information Recycling":
+    all discarded tokens merge into one additional token) says nothing about weights: the
+    additional token is the plain mean of the discarded tokens, it is appended after the
+    preserved vision tokens (before the text rows of FiCoCo-L), preserved tokens stay as they
+    are, and its kept index is -1; with nothing discarded there is no additional token;
   * for FiCoCo-L the supplied text->vision block t (head mean, M x N) is used for both
     the task term (1/M) sum_k t[k,i] and the text-bridged term (1/M) sum_k t[k,i] t[k,j]
     (main-text equations, which carry the 1/M that Algorithm 2 omits).
@@ -60,6 +65,7 @@ class Params:
     local_penalty: bool = True
     max_targets: Optional[int] = None  # None: token-adaptive K (paper); 0: pruning; k>0: fixed K
     average_compression: bool = False  # ablation "average compression": every alpha_ij = 1
+    convergent: bool = False           # ablation "convergent correlation": one additional token
 
 
 # ----------------------------------------------------------------------------
@@ -325,12 +331,19 @@ def ficoco_v_reduce(tokens: np.ndarray, attn: np.ndarray, pos: Optional[np.ndarr
     S, T = filter_topk(s, n_src)
     # Stage 2: Correlate
     C = correlation_v(R, S, T)
+    rn = 1.0 / np.sqrt(np.sum(P * P, axis=1))
+    if p.convergent:
+        extra = convergent_token(P, S) if n_src > 0 else None
+        out = _assemble_convergent(tokens, c, T, extra, 0)
+        kept = np.concatenate([np.arange(c), T + c, [-1] if n_src > 0 else []]).astype(np.int32)
+        none = [np.zeros(0, dtype=np.int64) for _ in range(n_src)]
+        return StepResult(out, kept, pos[T].astype(np.int32), s_raw, s, S, T, C, np.full(n_src, np.nan), none,
+                          [np.zeros(0) for _ in range(n_src)], np.zeros(T.shape[0]), rn, v, a)
     # Stage 3: Compress
     J, A, tau = targets_and_weights(C, p)
     merged, wsum = compress(P, S, T, J, A)
     out = _assemble(tokens, c, T, merged, wsum, tail_rows=0)
     kept = np.concatenate([np.arange(c), T + c]).astype(np.int32)
-    rn = 1.0 / np.sqrt(np.sum(P * P, axis=1))
     return StepResult(out, kept, pos[T].astype(np.int32), s_raw, s, S, T, C, tau, J, A, wsum, rn, v, a)
 
 
@@ -353,13 +366,39 @@ def ficoco_l_reduce(tokens: np.ndarray, attn_t2v: np.ndarray, n_vision: int, kee
     s_raw = score_l(v, t, p.beta)      # no local penalty in FiCoCo-L
     S, T = filter_topk(s_raw, n_src)
     C = correlation_l(R, t, S, T, p.gamma)
+    rn = 1.0 / np.sqrt(np.sum(P * P, axis=1))
+    if p.convergent:
+        extra = convergent_token(P, S) if n_src > 0 else None
+        out = _assemble_convergent(tokens, 0, T, extra, m)
+        kept = np.concatenate([T, [-1] if n_src > 0 else [], np.arange(n, n + m)]).astype(np.int32)
+        none = [np.zeros(0, dtype=np.int64) for _ in range(n_src)]
+        return StepResult(out, kept, None, s_raw, s_raw.copy(), S, T, C, np.full(n_src, np.nan), none,
+                          [np.zeros(0) for _ in range(n_src)], np.zeros(T.shape[0]), rn, v, t.sum(axis=0) / m)
     J, A, tau = targets_and_weights(C, p)
     merged, wsum = compress(P, S, T, J, A)
     out = _assemble(tokens, 0, T, merged, wsum, tail_rows=m)
     kept = np.concatenate([T, np.arange(n, n + m)]).astype(np.int32)
-    rn = 1.0 / np.sqrt(np.sum(P * P, axis=1))
     return StepResult(out, kept, None, s_raw, s_raw.copy(), S, T, C, tau, J, A, wsum, rn, v,
                       t.sum(axis=0) / m)
+
+
+def convergent_token(P: np.ndarray, S: np.ndarray) -> np.ndarray:
+    """Ablation "convergent correlation": the one additional token all discarded tokens merge
+    into, taken as their plain mean (float64; the paper gives no weights)."""
+    return P[np.sort(S)].sum(axis=0) / S.shape[0]
+
+
+def _assemble_convergent(tokens: np.ndarray, c: int, T: np.ndarray, extra: Optional[np.ndarray],
+                         tail_rows: int) -> np.ndarray:
+    """Output of the convergent variant: CLS rows, preserved rows bit for bit, the additional
+    token (rounded once to the storage format) when there is one, trailing rows."""
+    n_in = tokens.shape[0]
+    parts = [tokens[:c], tokens[c + T]]
+    if extra is not None:
+        parts.append(round_like(extra[None, :], tokens))
+    if tail_rows:
+        parts.append(tokens[n_in - tail_rows:])
+    return np.concatenate(parts, axis=0)
 
 
 def _assemble(tokens: np.ndarray, c: int, T: np.ndarray, merged: np.ndarray, wsum: np.ndarray,

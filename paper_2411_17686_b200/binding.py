@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libficoco.so")
 
 FICOCO_FP32, FICOCO_BF16 = 0, 1
-FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY, FICOCO_AVERAGE_COMPRESSION = 1, 2, 4
+FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY, FICOCO_AVERAGE_COMPRESSION, FICOCO_BACK_TO_BACK = 1, 2, 4, 8
 KCAP = 16
 
 INSPECT = {
@@ -32,7 +32,7 @@ EXPORTS = [
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
     "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
-    "ficoco_equivalent_token", "ficoco_v_reduce_relation",
+    "ficoco_equivalent_token", "ficoco_v_reduce_relation", "ficoco_debug_waits",
 ]
 
 
@@ -93,6 +93,7 @@ def load_library() -> C.CDLL:
     lib.ficoco_v_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params)]
     lib.ficoco_l_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params)]
     lib.ficoco_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
+    lib.ficoco_debug_waits.argtypes = [C.c_void_p, C.c_longlong, C.c_int]
     lib.ficoco_inspect.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.ficoco_last_launch_count.argtypes = [C.c_void_p]
     lib.ficoco_profile.argtypes = [C.c_void_p, C.c_int]
@@ -111,12 +112,14 @@ def ficoco_default_params() -> ficoco_params:
 
 
 def make_params(lam=0.35, beta=0.6, gamma=0.6, eps=0.998, penalty_coef=2.0, window=2,
-                max_targets=-1, has_cls=True, local_penalty=True, average_compression=False) -> ficoco_params:
+                max_targets=-1, has_cls=True, local_penalty=True, average_compression=False,
+                back_to_back=False) -> ficoco_params:
     p = ficoco_params()
     p.lambda_, p.beta, p.gamma, p.eps, p.penalty_coef = lam, beta, gamma, eps, penalty_coef
     p.window, p.max_targets = window, -1 if max_targets is None else max_targets
     p.flags = ((FICOCO_HAS_CLS if has_cls else 0) | (FICOCO_LOCAL_PENALTY if local_penalty else 0) |
-               (FICOCO_AVERAGE_COMPRESSION if average_compression else 0))
+               (FICOCO_AVERAGE_COMPRESSION if average_compression else 0) |
+               (FICOCO_BACK_TO_BACK if back_to_back else 0))
     return p
 
 
@@ -328,6 +331,9 @@ class Context:
         if n.value:
             _check(self.h, self.lib.ficoco_inspect(self.h, code, buf.ctypes.data, n.value, None))
         return buf.reshape(-1, width) if width > 1 else buf
+
+    def ficoco_debug_waits(self, wait_ns: int = 0, extra_arrivals: int = 0) -> None:
+        _check(self.h, self.lib.ficoco_debug_waits(self.h, wait_ns, extra_arrivals))
 
     def ficoco_last_launch_count(self) -> int:
         return int(self.lib.ficoco_last_launch_count(self.h))

@@ -1,5 +1,6 @@
 // mbarrier, cp.async and bulk-copy (TMA) primitives shared by the kernels.  Every wait is
-// bounded: it gives up after SPIN_LIMIT polls and the caller raises STATUS_TIMEOUT.
+// bounded by elapsed time on the GPU's global timer: it gives up after `limit_ns` nanoseconds
+// (WAIT_NS_DEFAULT unless the kernel is given another limit) and the caller raises STATUS_TIMEOUT.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -7,7 +8,30 @@
 namespace ficoco {
 
 constexpr unsigned STATUS_TIMEOUT = 4u;
-constexpr int SPIN_LIMIT = 1 << 22;
+constexpr unsigned long long WAIT_NS_DEFAULT = 20ull * 1000 * 1000;   // 20 ms: far beyond any wait of a healthy step
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Optional phase timestamps (compile with -DFICOCO_PHASE_TIMERS): thread 0 of a CTA notes the SM
+// clock at named points of a kernel; phase 0 also notes the global timer, so that the CTAs of a
+// grid can be laid on one time line.  Compiled out by default.
+#ifdef FICOCO_PHASE_TIMERS
+constexpr int PH_KERNELS = 4, PH_CTAS = 1024, PH_SLOTS = 16;
+__device__ unsigned long long g_phase_ts[PH_KERNELS][PH_CTAS][PH_SLOTS];
+#define FICOCO_PHASE(k, p)                                                             \
+  do {                                                                                 \
+    if (threadIdx.x == 0 && blockIdx.x < ficoco::PH_CTAS) {                            \
+      ficoco::g_phase_ts[k][blockIdx.x][p] = (unsigned long long)clock64();            \
+      if ((p) == 0) ficoco::g_phase_ts[k][blockIdx.x][ficoco::PH_SLOTS - 1] = ficoco::global_ns(); \
+    }                                                                                  \
+  } while (0)
+#else
+#define FICOCO_PHASE(k, p) do { } while (0)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -18,10 +42,13 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait on a phase parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait on a phase parity; false = gave up after limit_ns.  The clock is read only once
+// a try has failed, so a wait that succeeds at once costs one instruction.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity,
+                                          unsigned long long limit_ns = WAIT_NS_DEFAULT) {
   const uint32_t a = smem_u32(bar);
-  for (int it = 0; it < SPIN_LIMIT; ++it) {
+  unsigned long long t0 = 0;
+  for (;;) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -29,8 +56,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         "selp.b32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(a), "r"(parity) : "memory");
     if (ok) return true;
+    const unsigned long long t = global_ns();
+    if (t0 == 0) t0 = t;
+    else if (t - t0 > limit_ns) return false;
   }
-  return false;
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");

@@ -67,6 +67,7 @@ struct Plan {
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
   bool need_finalize = false;   // some image merges nothing: its per-token counts are zeroed by a kernel
   bool umma = false;
+  bool csr_in_tail = false;     // the tensor-core correlate kernel also builds the per-target segments
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
   size_t um_smem = 0;
   std::vector<ImgDesc> h_desc;
@@ -166,7 +167,14 @@ struct ficoco_ctx {
   float* tmean = nullptr;
   unsigned* status = nullptr;
   int* tile_cnt = nullptr;  // per source tile: column splits of the correlate kernel that are done
-  int* img_cnt = nullptr;   // 2 * max_batch per-image piece counters of the fused filter kernel
+  int* csr_cnt = nullptr;   // per image: source tiles whose targets and weights are final
+  int* seg_begin = nullptr; // per preserved token (+1 per image): start of its entries in csr_src / csr_w
+  int* csr_src = nullptr;   // (target, source, alpha) entries ordered by target, then token index
+  float* csr_w = nullptr;
+  int* img_cnt = nullptr;   // two sets of 3 * max_batch per-image counters of the fused filter kernel
+  unsigned long long epoch = 0;          // fused filter launches so far (its parity picks the counter set)
+  unsigned long long wait_ns = WAIT_NS_DEFAULT;   // bound of every device-side wait
+  int dbg_extra_arrivals = 0;            // testing hook: arrivals the fused filter waits for that never come
   int num_sms = 0;
   bool coop_ok = false;
   bool coop_pdl_ok = false;  // a cooperative grid may also be a programmatic dependent
@@ -298,7 +306,22 @@ extern "C" void ficoco_default_params(ficoco_params* p) {
   p->reserved = 0;
 }
 
+#ifdef FICOCO_PHASE_TIMERS
+// Phase timestamps of the most recent launch of every instrumented kernel (profiling builds only).
+extern "C" int ficoco_phase_read(void* host_dst, size_t bytes) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return FICOCO_ERR_CUDA;
+  const size_t n = sizeof(unsigned long long) * PH_KERNELS * PH_CTAS * PH_SLOTS;
+  return cudaMemcpyFromSymbol(host_dst, g_phase_ts, bytes < n ? bytes : n) == cudaSuccess ? FICOCO_OK : FICOCO_ERR_CUDA;
+}
+#endif
+
 extern "C" int ficoco_last_cuda_error(const ficoco_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+extern "C" int ficoco_debug_waits(ficoco_ctx* c, long long wait_ns, int extra_arrivals) {
+  if (!c || wait_ns < 0 || extra_arrivals < 0) return FICOCO_ERR_INVALID_ARG;
+  c->wait_ns = wait_ns > 0 ? (unsigned long long)wait_ns : WAIT_NS_DEFAULT;
+  c->dbg_extra_arrivals = extra_arrivals;
+  return FICOCO_OK;
+}
 extern "C" int ficoco_last_launch_count(const ficoco_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens, int max_dim,
@@ -357,8 +380,9 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
-  const size_t o_icnt = carve(2 * B * 4);
+  const size_t o_icnt = carve(6 * B * 4);
   const size_t o_tcnt = carve((size_t)c->cap_corr * 4);
+  const size_t o_ccnt = carve(B * 4), o_seg = carve((T + B) * 4), o_cs = carve(T * KCAP * 4), o_cwt = carve(T * KCAP * 4);
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
@@ -383,10 +407,13 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
   c->img_cnt = (int*)(b + o_icnt);
   c->tile_cnt = (int*)(b + o_tcnt);
+  c->csr_cnt = (int*)(b + o_ccnt); c->seg_begin = (int*)(b + o_seg);
+  c->csr_src = (int*)(b + o_cs); c->csr_w = (float*)(b + o_cwt);
   c->plan_slots = b + o_pl;
 
   // kernels that may need more than 48 KB of dynamic shared memory
   cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaFuncSetAttribute(k_build_csr, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
   {
     const int um_smem_max = 221 * 1024;
     cudaFuncSetAttribute(k_correlate_umma<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
@@ -686,7 +713,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     size_t sel_need = 0;
     for (int b = 0; b < B; ++b) {
       const ImgDesc& d = p->h_desc[b];
-      const size_t need = select_work_bytes(d.np, key.mode == 0 ? d.gh * d.gw : 0);
+      const size_t need = d.np <= SEL_SMALL_MAX ? select_small_bytes(d.np, key.mode == 0 ? d.gh * d.gw : 0)
+                                                : select_work_bytes(d.np, key.mode == 0 ? d.gh * d.gw : 0);
       if (need > sel_need) sel_need = need;
     }
     if (ns < 2 || sel_need > (size_t)ns * stage) p->fused = false;
@@ -725,6 +753,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     if (p->um_smem < epi) p->um_smem = epi;
     if (p->um_smem > 220 * 1024) return FICOCO_ERR_UNSUPPORTED;
   }
+  p->csr_in_tail = p->umma && csr_work_bytes(p->max_tgt) + 1024 <= p->um_smem;
 
   char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
   p->d_desc = (ImgDesc*)slot_dev;
@@ -823,7 +852,8 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
                             (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
-                            p->f_nstage, p->f_max_piece);
+                            p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), c->wait_ns,
+                            c->dbg_extra_arrivals);
 }
 
 template <class T, int VPL>
@@ -839,7 +869,7 @@ template <class T>
 int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn, int attn_rows,
              float cA, const int* pos, int window, float coef, int penalty, const float* tmean, int M,
              float gamma, T* out_tokens, int* kept_idx, int* pos_out, float* scores_out,
-             cudaStream_t st, const float* rel = nullptr) {
+             cudaStream_t st, bool back_to_back, const float* rel = nullptr) {
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
@@ -851,7 +881,14 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
                                    span_of(kept_idx, (size_t)p->tot_out_rows * sizeof(int)),
                                    span_of(pos_out, (size_t)p->tot_tgt * sizeof(int)),
                                    span_of(scores_out, (size_t)p->tot_patch * sizeof(float))};
-  const bool overlap_prev = inputs_clear_of_last_outputs(c->device, st, in_spans, 3);
+  const Span rel_span = span_of(rel, rel ? (size_t)p->h_desc.back().rel0 * 4 + (size_t)p->h_desc.back().np * p->h_desc.back().np * 4 : 0);
+  for (int o = 0; o < N_SPANS; ++o) {
+    for (int i = 0; i < 3; ++i)
+      if (spans_overlap(out_spans[o], in_spans[i])) return FICOCO_ERR_INVALID_ARG;
+    if (spans_overlap(out_spans[o], rel_span)) return FICOCO_ERR_INVALID_ARG;
+  }
+  // the early start is taken only when the caller vouches for what sits in front of this step
+  const bool overlap_prev = back_to_back && inputs_clear_of_last_outputs(c->device, st, in_spans, 3);
   record_last_outputs(c->device, st, out_spans, N_SPANS);
   if (p->fused) {
     prof_tick(c, st, "filter_fused");
@@ -894,7 +931,11 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
   c->launches += 1;
   }
-  const size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
+  size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
+  if (p->max_np <= SEL_SMALL_MAX) {
+    const size_t small = select_small_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
+    if (small > sel_smem) sel_smem = small;
+  }
   prof_tick(c, st, "select");
   // images of up to 1024 tokens: half the threads (two tokens each), cheaper barriers
   k_select<<<p->key.batch, p->max_np <= 1024 ? 512 : 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
@@ -902,6 +943,10 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
                                                   pos_out, c->status);
   c->launches += 1;
   }
+  CsrArgs csr = {};
+  csr.S_idx = c->S_idx; csr.tmp_src = c->part_idx; csr.tmp_w = c->part_val; csr.seg_begin = c->seg_begin;
+  csr.csr_src = c->csr_src; csr.csr_w = c->csr_w; csr.img_tiles = c->csr_cnt;
+  bool csr_done = false;
   if (p->n_corr > 0) {
     if (rel) {
       prof_tick(c, st, "correlate_relation");
@@ -918,13 +963,14 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #undef FICOCO_REL_GO
     } else if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
+      csr_done = p->csr_in_tail;
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
   launch_dependent(k_correlate_umma<NS, LC>, p->n_corr, UTHREADS, p->um_smem, st, tk, D,               \
       (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
       (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
       p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-      c->e_w, c->e_c, tmean, M, p->max_np, gamma)
+      c->e_w, c->e_c, tmean, M, p->max_np, gamma, c->wait_ns, csr, p->csr_in_tail ? 1 : 0)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 6) FICOCO_UMMA_LAUNCH(6, LC);                                                  \
@@ -952,11 +998,17 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
         p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c);
     c->launches += 1;
   }
+  if (p->n_corr > 0 && !csr_done) {
+    prof_tick(c, st, "build_segments");
+    k_build_csr<<<p->key.batch, 256, csr_work_bytes(p->max_tgt), st>>>(p->d_desc, c->e_tgt, c->e_w, csr, c->status);
+    c->launches += 1;
+  }
   prof_tick(c, st, "merge_compact");
   const int after_correlate = p->n_corr > 0 ? 1 : 0;   // else the grid before may be the filter itself
-  launch_dependent(k_merge_scan<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
-                   (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
-                   (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate);
+  launch_dependent(k_merge_csr<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+                   (const WorkItem*)p->d_out, (const int*)c->T_idx, (const int*)c->seg_begin,
+                   (const int*)c->csr_src, (const float*)c->csr_w, out_tokens, after_correlate,
+                   (const unsigned*)c->status);
   c->launches += 1;
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);
@@ -1013,14 +1065,15 @@ int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* pr
   c->last_plan = p;
   c->launches = 0;
   const int penalty = (prm->flags & FICOCO_LOCAL_PENALTY) ? 1 : 0;
+  const bool b2b = (prm->flags & FICOCO_BACK_TO_BACK) != 0;
   if (a->dtype == FICOCO_BF16)
     return run_step<__nv_bfloat16>(c, p, (const __nv_bfloat16*)a->tokens, a->dim, a->attn, a->heads,
                                    (float)prm->lambda_, a->pos, prm->window, (float)prm->penalty_coef,
                                    penalty, nullptr, 0, 1.0f, (__nv_bfloat16*)a->out_tokens, a->kept_idx,
-                                   a->pos_out, a->scores_out, st, rel);
+                                   a->pos_out, a->scores_out, st, b2b, rel);
   return run_step<float>(c, p, (const float*)a->tokens, a->dim, a->attn, a->heads, (float)prm->lambda_,
                          a->pos, prm->window, (float)prm->penalty_coef, penalty, nullptr, 0, 1.0f,
-                         (float*)a->out_tokens, a->kept_idx, a->pos_out, a->scores_out, st, rel);
+                         (float*)a->out_tokens, a->kept_idx, a->pos_out, a->scores_out, st, b2b, rel);
 }
 }  // namespace
 
@@ -1069,10 +1122,10 @@ extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const fico
     return run_step<__nv_bfloat16>(c, p, (const __nv_bfloat16*)a->tokens, a->dim, c->tmean, a->n_text,
                                    (float)prm->beta, nullptr, 1, 1.0f, 0, c->tmean, a->n_text,
                                    (float)prm->gamma, (__nv_bfloat16*)a->out_tokens, a->kept_idx, nullptr,
-                                   a->scores_out, st);
+                                   a->scores_out, st, false);
   return run_step<float>(c, p, (const float*)a->tokens, a->dim, c->tmean, a->n_text, (float)prm->beta,
                          nullptr, 1, 1.0f, 0, c->tmean, a->n_text, (float)prm->gamma,
-                         (float*)a->out_tokens, a->kept_idx, nullptr, a->scores_out, st);
+                         (float*)a->out_tokens, a->kept_idx, nullptr, a->scores_out, st, false);
 }
 
 extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_status) {
@@ -1085,8 +1138,9 @@ extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_statu
   CUDA_TRY(c, cudaStreamSynchronize(st));
   if (v & STATUS_TIMEOUT) {
     // a kernel gave up half-way: its per-image counters may be left non-zero
-    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 2 * (size_t)c->max_batch * sizeof(int), st));
+    CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 6 * (size_t)c->max_batch * sizeof(int), st));
     CUDA_TRY(c, cudaMemsetAsync(c->tile_cnt, 0, (size_t)c->cap_corr * sizeof(int), st));
+    CUDA_TRY(c, cudaMemsetAsync(c->csr_cnt, 0, (size_t)c->max_batch * sizeof(int), st));
     CUDA_TRY(c, cudaStreamSynchronize(st));
   }
   *device_status = (int)v;

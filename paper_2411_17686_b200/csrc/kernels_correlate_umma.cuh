@@ -169,14 +169,17 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
     int stage_bytes, int a_bytes, int tmem_cols, int* __restrict__ img_done, int* __restrict__ corr_cnt,
     float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
-    const float* __restrict__ tmean, int M, int NV, float gamma) {
+    const float* __restrict__ tmean, int M, int NV, float gamma, unsigned long long wait_ns, CsrArgs csr,
+    int csr_in_tail) {
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
   __shared__ int rowS[UM * UM_SUB], rowT[UN_MAX];
   __shared__ float rnT[UN_MAX];
-  __shared__ int failed, acc_committed, is_last;
+  __shared__ int failed, acc_committed, is_last, dead;
+  __shared__ int csr_scan_tmp[33];
 
+  FICOCO_PHASE(1, 0);
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int L = d.list_len;
@@ -204,8 +207,21 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   // may run while the filter grid is still finishing; the index lists and norms it wrote are
   // read below.  The dependent (merge) grid is released only after this wait, so by the time
   // any of its blocks starts, the filter grid is complete as well.
+  FICOCO_PHASE(1, 1);
   grid_dep_wait();
   grid_dep_launch();
+  FICOCO_PHASE(1, 2);
+  // A filter grid that gave up left no valid index lists: do nothing but give the TMEM back.
+  if (tid == 0) dead = (*reinterpret_cast<const volatile unsigned*>(status) & STATUS_TIMEOUT) ? 1 : 0;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (dead) {
+    if (warp == 4)
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base_s), "r"((uint32_t)tmem_cols)
+                   : "memory");
+    return;
+  }
   if (tid < UM * UM_SUB) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
   for (int c = tid; c < UN_MAX; c += UTHREADS) {
     const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
@@ -216,6 +232,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  FICOCO_PHASE(1, 3);
 
   if (warp != 4) {
     // ---------------- producers (all eight epilogue warps): gather rows, 16 bytes per copy -------
@@ -250,7 +267,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     for (int kb = 0; kb < nkb + LAG; ++kb) {
       if (kb < nkb) {
         const int s = kb % NSTAGE;
-        if (kb >= NSTAGE && ok) ok = mbar_wait(&empty_bar[s], ((kb / NSTAGE) - 1) & 1);
+        if (kb >= NSTAGE && ok) ok = mbar_wait(&empty_bar[s], ((kb / NSTAGE) - 1) & 1, wait_ns);
         if (ok) {
           const uint32_t a0 = ring + (uint32_t)s * stage_bytes + dsw;
           const uint32_t b0 = a0 + (uint32_t)a_bytes;
@@ -273,8 +290,10 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       }
     }
     cp_async_wait<0>();
+    FICOCO_PHASE(1, 4);
     if (!ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
-    bool acc_ok = ok && mbar_wait(&acc_bar, 0);
+    bool acc_ok = ok && mbar_wait(&acc_bar, 0, wait_ns);
+    FICOCO_PHASE(1, 5);
     if (!acc_ok) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
     acc_ok = __all_sync(0xFFFFFFFFu, acc_ok);          // tcgen05.ld below is warp-collective
     tc_fence_after();
@@ -387,7 +406,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       bool ok = true;
       for (int kb = 0; kb < nkb && ok; ++kb) {
         const int s = kb % NSTAGE;
-        ok = mbar_wait(&full_bar[s], (kb / NSTAGE) & 1);
+        ok = mbar_wait(&full_bar[s], (kb / NSTAGE) & 1, wait_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t a0 = ring + (uint32_t)s * stage_bytes;
@@ -409,22 +428,28 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     __syncwarp();
   }
 
+  FICOCO_PHASE(1, 6);
   tc_fence_before();
   __syncthreads();
+  FICOCO_PHASE(1, 7);
   if (warp == 4) {
     if (failed) {
       // MMAs may still be in flight: give them a bounded time to drain before freeing TMEM
       if (lane == 0) {
         if (!acc_committed) umma_commit(&acc_bar);
-        mbar_wait(&acc_bar, 0);
+        mbar_wait(&acc_bar, 0, wait_ns);
       }
       __syncwarp();
     }
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                  : "memory");
   }
+  // the operand ring is idle by now: the CTA that completes its image sorts the image's entries there
+  csr.work = csr_in_tail ? um_raw + (ring - smem_u32(um_raw)) : nullptr;
+  csr.scan_tmp = csr_scan_tmp;
   correlate_tail<LCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c,
-                       &is_last);
+                       &is_last, csr);
+  FICOCO_PHASE(1, 8);
 }
 
 }  // namespace ficoco

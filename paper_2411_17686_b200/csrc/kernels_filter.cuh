@@ -427,6 +427,274 @@ __device__ __noinline__ void select_image(
     kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
 }
 
+// ---------------------------------------------------------------------------------------
+// The same step for images of up to SEL_SMALL_MAX tokens by exactly 512 threads, two tokens per
+// thread held in registers, built for a short critical path (seven or eight barriers, no
+// contended atomics):
+//   1. scores and grid positions are loaded once; a grid-cell -> token map in shared memory lets
+//      one thread per window pick the window's maximum (lower token index on equal scores) and
+//      multiply it in place;
+//   2. keys are made dense: key - min key, shifted so that the largest has its top bit set, so the
+//      first radix digit already spreads the tokens over its 256 bins (raw fp32 keys of one
+//      image share sign and exponent and would all hit one bin); every warp reads the histogram
+//      and finds the digit by itself, so a pass costs one barrier; passes that could only see
+//      zero bits are skipped;
+//   3. membership flags become ascending positions with two ballots per warp and one 32-entry
+//      table of per-warp counts.
+// Only the outputs of tokens w_lo <= i < w_hi are written (plus the CLS / trailing entries of
+// kept_idx when w_lo == 0), so the CTAs that scored an image can each run the selection and
+// write their own slice.  select_small_prepare() zeroes the work area; a barrier (or any
+// inter-CTA wait that ends in one) must separate it from select_small().
+// ---------------------------------------------------------------------------------------
+constexpr int SEL_SMALL_MAX = 1024;
+constexpr int SEL_SMALL_THREADS = 512;
+
+struct SelectSmallShared {
+  uint32_t wmin[16], wmax[16];
+  int cnt[32];
+};
+
+__host__ __device__ inline size_t select_small_bytes(int np, int cells) {
+  return (size_t)np * 8 + 16 + 4 * 256 * sizeof(int) + (size_t)cells * 2 + 16;
+}
+
+struct SelectSmallWork {
+  float* sc;        // [np] scores (penalised in place)
+  uint32_t* nk;     // [np] dense keys
+  int* hist;        // [4][256]
+  short* cell;      // [gh * gw] token of every grid cell, -1 = no alive token
+};
+__device__ __forceinline__ SelectSmallWork select_small_layout(unsigned char* work, int np) {
+  SelectSmallWork w;
+  w.sc = reinterpret_cast<float*>(work);
+  w.nk = reinterpret_cast<uint32_t*>(work + (size_t)np * 4);
+  w.hist = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(work + (size_t)np * 8) + 15) & ~(uintptr_t)15);
+  w.cell = reinterpret_cast<short*>(w.hist + 4 * 256);
+  return w;
+}
+
+__device__ __forceinline__ void select_small_prepare(const ImgDesc& d, int penalty, unsigned char* work, int tid) {
+  const SelectSmallWork w = select_small_layout(work, d.np);
+  w.hist[tid] = 0;
+  w.hist[tid + SEL_SMALL_THREADS] = 0;
+  if (penalty) {
+    const int cells = d.gh * d.gw;
+    #pragma unroll 1
+    for (int c = tid; c < cells; c += SEL_SMALL_THREADS) w.cell[c] = -1;
+  }
+}
+
+__device__ __noinline__ void select_small(
+    const ImgDesc& d, const float* s_raw, const int* __restrict__ pos, int window, float coef,
+    int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
+    int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
+    unsigned* __restrict__ status, unsigned char* work, SelectSmallShared& sh, int tid, int bar,
+    int w_lo, int w_hi) {
+  constexpr int NT = SEL_SMALL_THREADS;
+  const int np = d.np, lane = tid & 31, warp = tid >> 5;
+  const SelectSmallWork wk = select_small_layout(work, np);
+  const int cells = d.gh * d.gw;
+  float s[2];
+  int pp[2];
+  bool on[2];
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + NT * q;
+    on[q] = i < np;
+    s[q] = on[q] ? __ldcg(s_raw + d.patch0 + i) : 0.f;
+    pp[q] = on[q] ? (pos ? pos[d.patch0 + i] : i) : -1;
+  }
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + NT * q;
+    if (!on[q]) continue;
+    wk.sc[i] = s[q];
+    if (penalty) {
+      if (pp[q] >= 0 && pp[q] < cells) wk.cell[pp[q]] = (short)i;
+      else atomicOr(status, STATUS_POS_RANGE);
+    }
+  }
+  cta_sync(bar, NT);
+
+  // ---- local penalty: one thread per window ------------------------------------------------
+  if (penalty) {
+    const int nwc = (d.gw + window - 1) / window, nwr = (d.gh + window - 1) / window;
+    #pragma unroll 1
+    for (int wdx = tid; wdx < nwc * nwr; wdx += NT) {
+      const int r0 = (wdx / nwc) * window, c0 = (wdx % nwc) * window;
+      const int r1 = min(d.gh, r0 + window), c1 = min(d.gw, c0 + window);
+      int best = -1;
+      float bs = 0.f;
+      #pragma unroll 1
+      for (int r = r0; r < r1; ++r)
+        #pragma unroll 1
+        for (int c = c0; c < c1; ++c) {
+          const int t = wk.cell[r * d.gw + c];
+          if (t < 0) continue;
+          const float v = wk.sc[t];
+          if (best < 0 || v > bs || (v == bs && t < best)) { best = t; bs = v; }
+        }
+      if (best >= 0) wk.sc[best] = bs * coef;      // windows are disjoint: nobody else touches this token
+    }
+    cta_sync(bar, NT);
+  }
+
+  // ---- keys, their range, dense keys -----------------------------------------------------------
+  uint32_t key[2];
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + NT * q;
+    if (on[q]) {
+      s[q] = wk.sc[i] + 0.0f;                      // -0 and +0 are one score
+      key[q] = order_key(s[q]);
+      kmin = min(kmin, key[q]);
+      kmax = max(kmax, key[q]);
+      if (i >= w_lo && i < w_hi) {
+        s_pen[d.patch0 + i] = s[q];
+        if (scores_out) scores_out[d.patch0 + i] = s[q];
+      }
+    } else {
+      key[q] = 0u;
+    }
+  }
+  kmin = __reduce_min_sync(0xFFFFFFFFu, kmin);
+  kmax = __reduce_max_sync(0xFFFFFFFFu, kmax);
+  if (lane == 0) { sh.wmin[warp] = kmin; sh.wmax[warp] = kmax; }
+  cta_sync(bar, NT);
+  {
+    const uint32_t a = sh.wmin[lane & 15], b = sh.wmax[lane & 15];
+    kmin = __reduce_min_sync(0xFFFFFFFFu, a);
+    kmax = __reduce_max_sync(0xFFFFFFFFu, b);
+  }
+  const int k = d.n_src;
+  const uint32_t range = kmax - kmin;
+  const int sh_l = range ? __clz(range) : 0;
+  uint32_t nk[2];
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    nk[q] = range ? (key[q] - kmin) << sh_l : 0u;
+    if (on[q]) wk.nk[tid + NT * q] = nk[q];
+  }
+
+  // ---- radix select on the dense keys: the n_src-th largest -------------------------------------
+  uint32_t thr = 0;      // threshold (dense key)
+  int need_eq = 0;       // how many of the keys equal to thr are selected (lowest indices)
+  int c_eq = 0;          // how many keys equal thr
+  if (k > 0 && k < np) {
+    const int npass = range ? (32 - sh_l + 7) / 8 : 1;   // the low sh_l bits of every dense key are zero
+    uint32_t prefix = 0, mask = 0;
+    int remaining = k;
+    #pragma unroll 1
+    for (int pass = 0; pass < npass; ++pass) {
+      const int shift = 24 - 8 * pass;
+      int* h = wk.hist + 256 * pass;
+#pragma unroll
+      for (int q = 0; q < 2; ++q)
+        if (on[q] && (nk[q] & mask) == prefix) atomicAdd(&h[(nk[q] >> shift) & 255], 1);
+      cta_sync(bar, NT);
+      // every warp: lane l owns bins 255-8l .. 248-8l (descending); find where the running count
+      // from the top reaches `remaining`
+      int c[8], tot = 0;
+      {
+        const int4 lo = *reinterpret_cast<const int4*>(h + 248 - 8 * lane);
+        const int4 hi = *reinterpret_cast<const int4*>(h + 252 - 8 * lane);
+        c[0] = hi.w; c[1] = hi.z; c[2] = hi.y; c[3] = hi.x;
+        c[4] = lo.w; c[5] = lo.z; c[6] = lo.y; c[7] = lo.x;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) tot += c[j];
+      int inc = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += n;
+      }
+      const int before = inc - tot;
+      const bool mine = before < remaining && inc >= remaining;
+      int digit = 0, rem_new = 0, ceq_new = 0;
+      if (mine) {
+        int cum = before;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (cum < remaining && cum + c[j] >= remaining) {
+            digit = 255 - 8 * lane - j;
+            rem_new = remaining - cum;
+            ceq_new = c[j];
+          }
+          cum += c[j];
+        }
+      }
+      const int src = __ffs(__ballot_sync(0xFFFFFFFFu, mine)) - 1;   // exactly one lane (0 < remaining <= total)
+      digit = __shfl_sync(0xFFFFFFFFu, digit, src);
+      remaining = __shfl_sync(0xFFFFFFFFu, rem_new, src);
+      c_eq = __shfl_sync(0xFFFFFFFFu, ceq_new, src);
+      prefix |= (uint32_t)digit << shift;
+      mask |= 0xFFu << shift;
+    }
+    thr = prefix;
+    need_eq = remaining;
+  }
+
+  // ---- membership ---------------------------------------------------------------------------------
+  bool sel[2];
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    const int i = tid + NT * q;
+    if (!on[q]) sel[q] = false;
+    else if (k <= 0) sel[q] = false;
+    else if (k >= np) sel[q] = true;
+    else if (nk[q] != thr) sel[q] = nk[q] > thr;
+    else if (need_eq >= c_eq) sel[q] = true;
+    else {
+      // equal scores straddle the boundary: the lowest indices among them are taken
+      int before = 0;
+      #pragma unroll 1
+      for (int j = 0; j < i; ++j) before += wk.nk[j] == thr ? 1 : 0;
+      sel[q] = before < need_eq;
+    }
+  }
+
+  // ---- ascending positions ------------------------------------------------------------------------
+  const unsigned b0 = __ballot_sync(0xFFFFFFFFu, sel[0]), b1 = __ballot_sync(0xFFFFFFFFu, sel[1]);
+  if (lane == 0) { sh.cnt[warp] = __popc(b0); sh.cnt[16 + warp] = __popc(b1); }
+  cta_sync(bar, NT);
+  {
+    const int mycnt = sh.cnt[lane];
+    int inc = mycnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    const int excl = inc - mycnt;                 // selected tokens in the 32-token groups before group `lane`
+    const unsigned lt = (1u << lane) - 1u;
+    const int rank0 = __shfl_sync(0xFFFFFFFFu, excl, warp) + __popc(b0 & lt);
+    const int rank1 = __shfl_sync(0xFFFFFFFFu, excl, 16 + warp) + __popc(b1 & lt);
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      const int i = tid + NT * q;
+      if (!on[q] || i < w_lo || i >= w_hi) continue;
+      const int rank = q ? rank1 : rank0;          // selected tokens with a lower index
+      if (sel[q]) {
+        S_idx[d.src0 + rank] = i;
+      } else {
+        const int tp = i - rank;
+        T_idx[d.tgt0 + tp] = i;
+        kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
+        if (pos_out) pos_out[d.tgt0 + tp] = pp[q];
+      }
+    }
+  }
+  if (w_lo == 0) {
+    #pragma unroll 1
+    for (int i = tid; i < d.n_cls; i += NT) kept_idx[d.out_row0 + i] = i;
+    #pragma unroll 1
+    for (int i = tid; i < d.n_tail; i += NT)
+      kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
+  }
+}
+
 // One CTA (512 or 1024 threads) per image.
 __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ desc,
                                                  const float* __restrict__ s_raw,
@@ -438,7 +706,15 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
                                                  unsigned* __restrict__ status) {
   extern __shared__ unsigned char sm_raw[];
   __shared__ SelectShared sh;
+  __shared__ SelectSmallShared shs;
   const ImgDesc d = desc[blockIdx.x];
+  if (d.np <= SEL_SMALL_MAX && blockDim.x == SEL_SMALL_THREADS) {
+    select_small_prepare(d, penalty, sm_raw, threadIdx.x);
+    __syncthreads();
+    select_small(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
+                 status, sm_raw, shs, threadIdx.x, 0, 0, d.np);
+    return;
+  }
   select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
                status, sm_raw, sh, threadIdx.x, (int)blockDim.x, 0);
 }

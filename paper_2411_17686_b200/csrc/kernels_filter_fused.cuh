@@ -9,9 +9,13 @@
 //   pass 2  (rows read again, now L2-resident, with plain 16-byte loads, three rows in flight
 //           per warp) once all pieces of the image are in:
 //           v_i = rn_i (x_i . sum of partials) / Np,  s_i = cA v_i - (1 - cA) a_i;
-//           the CTA that finishes the last piece of an image runs the local penalty and the
-//           radix select for that image and resets the image's counters.
-// The only inter-CTA waits are the bounded polls of the per-image counter between the passes.
+//   select  images of up to 1024 tokens: every CTA that scored a piece waits until all of the
+//           image's scores are in, runs the (short) selection on the whole image and writes the
+//           outputs of its own tokens; larger images: the CTA that finishes the last piece runs
+//           the selection alone.  The last CTA to leave an image resets its counters.
+// The inter-CTA waits are polls of per-image counters, bounded by elapsed time (wait_ns).  The
+// counters exist twice; a launch uses the set of its parity and zeroes the other one, so a step
+// that gave up half-way cannot leave counts behind for the step after the next.
 #pragma once
 #include "async_ops.cuh"
 #include "common.cuh"
@@ -26,12 +30,27 @@ constexpr int F_NCONS = 512;      // consumer threads
 constexpr int F_THREADS = 544;    // + one producer warp
 constexpr int F_MAXSTAGE = 16;
 constexpr int F_MAXWON = 32;      // pieces per CTA (and therefore selections it can win)
-constexpr int F_POLL_LIMIT = 1 << 20;
+static_assert(F_NCONS == SEL_SMALL_THREADS, "the short selection is written for the consumer threads");
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
   asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+
+// Poll until *p >= need.  Gives up after limit_ns, or at once when another CTA has already
+// raised STATUS_TIMEOUT (its pieces will never arrive).  One thread calls this.
+__device__ __forceinline__ bool poll_count(const int* p, int need, unsigned long long limit_ns,
+                                           const unsigned* status) {
+  unsigned long long t0 = 0;
+  for (;;) {
+    if (ld_acquire(p) >= need) return true;
+    const unsigned long long t = global_ns();
+    if (t0 == 0) t0 = t;
+    else if (t - t0 > limit_ns) return false;
+    if (*reinterpret_cast<const volatile unsigned*>(status) & STATUS_TIMEOUT) return false;
+    __nanosleep(32);
+  }
 }
 
 // The mean direction m (one float per column) is kept in shared memory so that a warp reads it
@@ -85,15 +104,17 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     const int* __restrict__ pos, int window, float coef, int penalty, float* __restrict__ s_pen,
     float* __restrict__ scores_out, int* __restrict__ S_idx, int* __restrict__ T_idx,
     int* __restrict__ kept_idx, int* __restrict__ pos_out, unsigned* __restrict__ status,
-    int nstage, int max_piece) {
+    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals) {
   constexpr int E = VecTraits<T>::E;
   constexpr int F_P2B = VPL <= 4 ? 2 : 1;   // rows a warp scores together in pass 2 (and has in flight from L2)
   extern __shared__ __align__(128) unsigned char fs_raw[];
   __shared__ uint64_t full_bar[F_MAXSTAGE], empty_bar[F_MAXSTAGE];
   __shared__ SelectShared sel_sh;
+  __shared__ SelectSmallShared sel_small_sh;
   // All CTAs of this grid are co-resident, so the next grid may be staged right away: its blocks
   // take over SMs as blocks of this grid exit and park until this grid has completed.
   grid_dep_launch();
+  FICOCO_PHASE(0, 0);
   __shared__ int won[F_MAXWON];
   __shared__ int nwon, failed;
 
@@ -105,6 +126,14 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   float* fold = reinterpret_cast<float*>(fs_raw + (size_t)nstage * stage_bytes);   // [FFOLD][D], msum aliases fold[0]
   float* a_s = fold + (size_t)FFOLD * D;                                            // [max_piece]
   const int p_begin = cta_first[blockIdx.x], p_end = cta_first[blockIdx.x + 1];
+  // counters of this launch: [0, B) pieces through pass 1, [B, 2B) pieces scored, [2B, 3B) pieces
+  // whose CTA has left the selection.  The other set belongs to the launch before and the one after.
+  {
+    int* other = cnt + (parity ? 0 : 3 * B);
+    if (blockIdx.x == 0)
+      for (int i = tid; i < 3 * B; i += F_THREADS) other[i] = 0;
+    cnt += parity ? 3 * B : 0;
+  }
 
   if (tid == 0) {
     for (int s = 0; s < nstage; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], FWARPS); }
@@ -126,7 +155,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
             reinterpret_cast<const unsigned char*>(tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D);
         for (int g = 0; g * FROWS < w.nrows && ok; ++g, ++seq) {
           const int s = seq % nstage;
-          if (seq >= nstage) ok = mbar_wait(&empty_bar[s], ((seq / nstage) - 1) & 1);
+          if (seq >= nstage) ok = mbar_wait(&empty_bar[s], ((seq / nstage) - 1) & 1, wait_ns);
           if (!ok) break;
           const int rows = min(FROWS, w.nrows - g * FROWS);
           mbar_expect_tx(&full_bar[s], (uint32_t)(rows * row_bytes));
@@ -140,6 +169,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   }
 
   // --------------------------------- consumers ----------------------------------------------
+  FICOCO_PHASE(0, 1);
   int seq = 0;
   bool ok = true;
   // pass 1: norms and column sums
@@ -153,7 +183,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       for (int e = 0; e < E; ++e) acc[k][e] = 0.f;
     for (int g = 0; g * FROWS < w.nrows; ++g, ++seq) {
       const int s = seq % nstage;
-      if (ok) ok = mbar_wait(&full_bar[s], (seq / nstage) & 1);
+      if (ok) ok = mbar_wait(&full_bar[s], (seq / nstage) & 1, wait_ns);
       const int r = g * FROWS + warp;
       if (r < w.nrows) {
         const unsigned char* rp = ring + (size_t)s * stage_bytes + (size_t)warp * row_bytes;
@@ -233,6 +263,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     if (tid == 0) red_release_add(&cnt[w.img], 1);   // pairs with the ld.acquire poll of pass 2
   }
   if (!ok && lane == 0) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+  FICOCO_PHASE(0, 2);
 
   // pass 2: scores.  The last `nstage` row groups of pass 1 are still in the ring and are read
   // from there (only when every wait of pass 1 succeeded); the older ones are L2-resident and
@@ -244,14 +275,11 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     const ImgDesc d = desc[w.img];
     const int seq_piece = seq2;                     // number of this piece's first group
     seq2 += (w.nrows + FROWS - 1) / FROWS;
-    if (tid == 0) {
-      bool in = false;
-      for (int it = 0; it < F_POLL_LIMIT && !in; ++it) {
-        in = ld_acquire(&cnt[w.img]) >= d.n_chunks;
-        if (!in) __nanosleep(64);
-      }
-      if (!in) { atomicOr(status, STATUS_TIMEOUT); failed = 1; }
+    if (tid == 0 && !poll_count(&cnt[w.img], d.n_chunks + dbg_extra_arrivals, wait_ns, status)) {
+      atomicOr(status, STATUS_TIMEOUT);
+      failed = 1;
     }
+    if (pi == p_begin) FICOCO_PHASE(0, 3);
     const float inv_h = 1.0f / (float)H;
     for (int r = tid; r < w.nrows; r += F_NCONS) {     // attention term, does not depend on the wait
       const float* a = attn + d.attn0 + w.r0 + r;
@@ -274,6 +302,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       msum[msum_slot<E>(c, nvec)] = t;
     }
     cta_sync(1, F_NCONS);
+    if (pi == p_begin) FICOCO_PHASE(0, 4);
     const float inv_np = 1.0f / (float)d.np;
     const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D;
     // This warp owns line `warp` of every 16-row group of the piece.  Groups numbered below
@@ -338,26 +367,56 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     if (tid == 0) {
       // release this piece's scores, and (for the CTA that arrives last) acquire everyone else's
       const int old = atom_acq_rel_add(&cnt[B + w.img], 1);
-      if (old == d.n_chunks - 1 && nwon < F_MAXWON) won[nwon++] = w.img;
+      if (d.np > SEL_SMALL_MAX && old == d.n_chunks - 1 && nwon < F_MAXWON) won[nwon++] = w.img;
     }
   }
   cta_sync(1, F_NCONS);
 
-  // selections this CTA won (the ring is idle now and serves as work area)
+  FICOCO_PHASE(0, 5);
   if (failed) return;
   // Up to here the kernel wrote only scratch that no grid but a filter or correlate grid reads,
   // and those of the step before were complete before this grid could start.  The index lists
   // and outputs written below are read by the merge grid of the step before: wait for it.
   grid_dep_wait();
-  const int nw = nwon;
-  for (int k = 0; k < nw; ++k) {
-    const int img = won[k];
-    const ImgDesc d = desc[img];
-    select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-                 status, ring, sel_sh, tid, F_NCONS, 1);
-    cta_sync(1, F_NCONS);
-    if (tid == 0) { cnt[img] = 0; cnt[B + img] = 0; }
+  FICOCO_PHASE(0, 6);
+  // selections (the ring is idle now and serves as work area), image by image over this CTA's pieces
+  int pi = p_begin;
+  #pragma unroll 1
+  while (pi < p_end) {
+    const WorkItem w0 = pieces[pi];
+    const ImgDesc d = desc[w0.img];
+    int pj = pi, hi = w0.r0;
+    while (pj < p_end && pieces[pj].img == w0.img) { hi = pieces[pj].r0 + pieces[pj].nrows; ++pj; }
+    if (d.np <= SEL_SMALL_MAX) {
+      select_small_prepare(d, penalty, ring, tid);
+      if (tid == 0 && !poll_count(&cnt[B + w0.img], d.n_chunks, wait_ns, status)) {
+        atomicOr(status, STATUS_TIMEOUT);
+        failed = 1;
+      }
+      cta_sync(1, F_NCONS);
+      if (failed) return;
+      FICOCO_PHASE(0, 7);
+      select_small(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
+                   status, ring, sel_small_sh, tid, 1, w0.r0, hi);
+      cta_sync(1, F_NCONS);
+      if (tid == 0) {
+        // the last pieces to leave reset the image's counters (everybody is past its polls by then)
+        const int old = atomicAdd(&cnt[2 * B + w0.img], pj - pi);
+        if (old + (pj - pi) == d.n_chunks) { cnt[w0.img] = 0; cnt[B + w0.img] = 0; cnt[2 * B + w0.img] = 0; }
+      }
+    } else {
+      bool mine = false;
+      for (int k = 0; k < nwon; ++k) mine = mine || won[k] == w0.img;
+      if (mine) {
+        select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
+                     status, ring, sel_sh, tid, F_NCONS, 1);
+        cta_sync(1, F_NCONS);
+        if (tid == 0) { cnt[w0.img] = 0; cnt[B + w0.img] = 0; }
+      }
+    }
+    pi = pj;
   }
+  FICOCO_PHASE(0, 8);
 }
 
 }  // namespace ficoco

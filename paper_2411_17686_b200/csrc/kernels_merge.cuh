@@ -8,7 +8,7 @@ constexpr int MHUB = 4;        // source rows a lane has in flight for a hub row
 constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the per-row arrays)
 constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
 constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
-constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
+constexpr int MLIST = 1024;    // (source, alpha) entries a CTA copies to shared memory (more are read in place)
 constexpr int MHEAVY = 2;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
 
@@ -46,147 +46,81 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
   }
 }
 
-// Compress + compact.  No per-target lists are built in global memory.  A CTA owns up to 32
-// consecutive output rows of one image (warp w: rows w, w + 8, w + 16, w + 24).
-//   1. every warp resolves the input row of its output rows (L1 prefetches of the rows were tried:
-//      they never produced L1 hits and cost 1.7 us per step, so there are none);
-//   2. meanwhile the CTA scans the image's (source -> target) entries twice (count, then fill)
-//      to file those that hit its rows into per-row lists in shared memory (token index,
-//      alpha), and orders every list by token index so that the
-//      fp32 sums have one fixed order and no atomics touch floats;
-//   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
-//      rows with few sources by their own warp; hub rows are cut into blocks of 32 vectors that
-//      are dealt to the warps, every lane summing the sources of its vector in list order.
-// If the CTA's rows receive more than MLIST sources in total, a slow in-order rescan is used.
+// Compress + compact.  A CTA owns up to 32 consecutive output rows of one image (warp w: rows
+// w, w + 8, w + 16, w + 24).
+//   1. every row resolves its input row (CLS / preserved token / trailing text row) and, for a
+//      preserved token, the bounds of its segment in the per-target entry lists that the
+//      correlate step left (ordered by token index, so the fp32 sums have one fixed order and no
+//      atomics touch floats); the segments of consecutive rows are contiguous, so the CTA's
+//      entries are one run, copied to shared memory (read in place when there are more than MLIST);
+//   2. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
+//      rows without sources are copied in one batch, rows with few sources are merged by their
+//      own warp; hub rows are cut into blocks of 32 vectors that are dealt to the warps, every
+//      lane summing the sources of its vector in list order.
 template <class T>
-__global__ void __launch_bounds__(256) k_merge_scan(
+__global__ void __launch_bounds__(256) k_merge_csr(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
-    const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
-    const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out,
-    int index_before_wait) {
+    const WorkItem* __restrict__ work, const int* __restrict__ T_idx,
+    const int* __restrict__ seg_begin, const int* __restrict__ csr_src, const float* __restrict__ csr_w,
+    T* __restrict__ out, int index_before_wait, const unsigned* __restrict__ status) {
   constexpr int E = VecTraits<T>::E;
-  __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
-  __shared__ int lsrc[MLIST];
-  __shared__ float lw[MLIST];
-  __shared__ int tsrc[MLIST];
-  __shared__ float tw[MLIST];
+  __shared__ int cnt[MROWS], beg[MROWS + 1], srow_s[MROWS];
+  __shared__ int lsrc_s[MLIST];
+  __shared__ float lw_s[MLIST];
   __shared__ int heavy_rows[MROWS];
-  __shared__ int n_heavy;
+  __shared__ int n_heavy, dead;
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = D / E;
-  const int L = d.list_len;
   const int tp_lo = max(w.r0 - d.n_cls, 0);
   const int tp_hi = min(w.r0 + w.nrows - d.n_cls, d.n_tgt);
-  const int n_ent = d.n_src * L;
+  const int n_tp = (d.list_len > 0 && tp_hi > tp_lo) ? tp_hi - tp_lo : 0;   // target rows that may have sources
   const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
 
-  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
+  FICOCO_PHASE(2, 0);
+  if (tid < MROWS) cnt[tid] = 0;
   if (tid == 0) n_heavy = 0;
   // When the grid before this one is a correlate grid, the filter grid (which wrote T_idx) had
   // completed before this grid could start, so the row lookup may overlap that
   // grid's tail; otherwise wait first.
   if (!index_before_wait) grid_dep_wait();
-  // input row of every output row (CLS / preserved token / trailing text row)
-  #pragma unroll 1
-  for (int r = warp; r < w.nrows; r += 8) {
-    const int orow = w.r0 + r;
+  if (tid < w.nrows) {
+    const int orow = w.r0 + tid;
     int srow;
     if (orow < d.n_cls) srow = orow;
     else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
     else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
-    if (lane == 0) srow_s[r] = srow;
+    srow_s[tid] = srow;
   }
   if (index_before_wait) grid_dep_wait();
   grid_dep_launch();   // correlate is complete: the next step's filter may stream its rows under our tail
+  FICOCO_PHASE(2, 1);
+  // a step whose filter or correlate grid gave up has no valid index lists: write nothing
+  if (tid == 0) dead = (*reinterpret_cast<const volatile unsigned*>(status) & 4u) ? 1 : 0;
+  if (tid <= n_tp && n_tp > 0) beg[tid] = __ldcg(seg_begin + d.tgt0 + w.img + tp_lo + tid);
   __syncthreads();
-  // file the entries that hit this CTA's rows.  Up to 1024 entries per image every thread looks
-  // at no more than four, keeps its matches in registers and needs one pass; larger images
-  // take a counting pass and a filling pass.
-  const bool one_pass = n_ent <= 4 * 256;
-  int st_row[4], st_slot[4], st_src[4];
-  float st_w[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) st_row[i] = -1;
-  if (tp_hi > tp_lo) {
-    if (one_pass) {
-      int t4[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        // target, source and weight are fetched together: a source fetched only for the matches
-        // would add a second round trip to L2
-        const int e = tid + 256 * i;
-        const bool on = e < n_ent;
-        t4[i] = on ? e_tgt[d.ent0 + e] : -1;
-        st_src[i] = on ? S_idx[d.src0 + e / L] : 0;
-        st_w[i] = on ? e_w[d.ent0 + e] : 0.f;
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int t = t4[i];
-        if (t >= tp_lo && t < tp_hi) {
-          st_row[i] = t - tp_lo;
-          st_slot[i] = atomicAdd(&cnt[t - tp_lo], 1);
-        }
-      }
-    } else {
-      for (int e = tid; e < n_ent; e += 256) {
-        const int t = e_tgt[d.ent0 + e];
-        if (t >= tp_lo && t < tp_hi) atomicAdd(&cnt[t - tp_lo], 1);
-      }
-    }
-  }
-  __syncthreads();
-  if (warp == 0) {
-    // exclusive scan of the 32 counts
-    const int c = cnt[lane];
-    int inc = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-      if (lane >= o) inc += n;
-    }
-    beg[lane] = inc - c;
-    if (lane == 31) beg[MROWS] = inc;
-    if (c > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = lane;
-  }
-  __syncthreads();
-  const int total = beg[MROWS];
+  if (dead) return;
+  const int e0 = n_tp ? beg[0] : 0;
+  const int total = n_tp ? beg[n_tp] - e0 : 0;
   const bool fits = total <= MLIST;
-  if (fits && total > 0) {
-    if (one_pass) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (st_row[i] >= 0) {
-          const int slot = beg[st_row[i]] + st_slot[i];
-          tsrc[slot] = st_src[i];
-          tw[slot] = st_w[i];
-        }
-    } else {
-      for (int e = tid; e < n_ent; e += 256) {
-        const int t = e_tgt[d.ent0 + e];
-        if (t >= tp_lo && t < tp_hi) {
-          const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
-          const int si = S_idx[d.src0 + e / L];
-          tsrc[slot] = si;
-          tw[slot] = e_w[d.ent0 + e];
-        }
-      }
-    }
-    __syncthreads();
-    // order every list by token index (rank of each entry inside its row)
+  const int* lsrc = csr_src + d.ent0 + e0;
+  const float* lw = csr_w + d.ent0 + e0;
+  if (fits) {
     for (int i = tid; i < total; i += 256) {
-      int r = 0;
-      while (i >= beg[r + 1]) ++r;
-      const int my = tsrc[i];
-      int rank = 0;
-      for (int k = beg[r]; k < beg[r + 1]; ++k) rank += tsrc[k] < my ? 1 : 0;
-      lsrc[beg[r] + rank] = my;
-      lw[beg[r] + rank] = tw[i];
+      lsrc_s[i] = __ldcg(lsrc + i);
+      lw_s[i] = __ldcg(lw + i);
     }
+    lsrc = lsrc_s;
+    lw = lw_s;
+  }
+  if (tid < n_tp) {
+    const int c = beg[tid + 1] - beg[tid];
+    cnt[tid] = c;
+    if (c > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = tid;
   }
   __syncthreads();
+  FICOCO_PHASE(2, 2);
 
   // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
   #pragma unroll 1
@@ -220,6 +154,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     }
   }
 
+  FICOCO_PHASE(2, 3);
   // ---- rows with a few sources: one warp per row --------------------------------------------------
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
@@ -231,8 +166,8 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
     if (n == 0) {
       continue;
-    } else if (fits && n <= MHEAVY) {
-      const int b0 = beg[li];
+    } else if (n <= MHEAVY) {
+      const int b0 = beg[li] - e0;
       float wsum = 0.f;
       for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
       const float inv_den = 1.0f / (1.0f + wsum);   // one division per row, then multiplies
@@ -255,33 +190,10 @@ __global__ void __launch_bounds__(256) k_merge_scan(
           }
         }
       }
-    } else if (!fits) {
-      // too many sources for shared memory: walk the entries in order (ascending source)
-      const int tp = orow - d.n_cls;
-      float wsum = 0.f;
-      for (int e = 0; e < n_ent; ++e)
-        if (e_tgt[d.ent0 + e] == tp) wsum += e_w[d.ent0 + e];
-      const float den = 1.0f + wsum;
-      for (int v = lane; v < nvec; v += 32) {
-        float acc[E];
-        unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
-        for (int e = 0; e < n_ent; ++e) {
-          if (e_tgt[d.ent0 + e] != tp) continue;
-          const T* x0 = pbase + (size_t)S_idx[d.src0 + e / L] * D;
-          float f[E];
-          unpack(ldg16(x0 + (size_t)v * E), f, (const T*)nullptr);
-          const float a0 = e_w[d.ent0 + e];
-#pragma unroll
-          for (int q = 0; q < E; ++q) acc[q] = fmaf(a0, f[q], acc[q]);
-        }
-#pragma unroll
-        for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
-        reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
-      }
     }
   }
-  if (!fits) return;
 
+  FICOCO_PHASE(2, 4);
   // ---- hub rows: (row, block of 32 vectors) items dealt to the warps; each lane sums all the
   // sources of its one vector in list order, MHUB source rows in flight ---------------------
   const int nh = n_heavy;
@@ -292,7 +204,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     const int v = (it % nblk) * 32 + lane;
     if (v >= nvec) continue;
     const int tp = tp_lo + li;
-    const int b0 = beg[li], n = cnt[li];
+    const int b0 = beg[li] - e0, n = cnt[li];
     const T* src = tokens + (size_t)(d.row0 + srow_s[tp + d.n_cls - w.r0]) * D;
     T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
     float wsum = 0.f;
@@ -322,6 +234,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
     reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
   }
+  FICOCO_PHASE(2, 5);
 }
 
 }  // namespace ficoco

@@ -235,8 +235,9 @@ __global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
       }
     }
   }
+  CsrArgs no_csr = {};
   correlate_tail<LC>(d, w, (int)blockIdx.x - w.aux, tile_done, part_val, part_idx, corr_cnt, tau_out,
-                     e_tgt, e_w, e_c, &is_last);
+                     e_tgt, e_w, e_c, &is_last, no_csr);
 }
 
 }  // namespace ficoco

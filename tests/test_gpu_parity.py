@@ -1,6 +1,8 @@
 """GPU parity: the CUDA library (through its C ABI) against the float64 checker, element by
 element, on seeded inputs whose discrete decisions were made unambiguous beforehand."""
 import copy
+import json
+import os
 
 import numpy as np
 import pytest
@@ -199,6 +201,7 @@ def test_back_to_back_steps_without_sync(ctx):
     batch = synth.make_v_batch(91, nb, g, g, 512, heads, g * g // 2, "bf16", True, 1.5)
     pk = packing.pack_v(batch, DEV)
     prm = parity.params_to_abi(fo.Params(), True)
+    prm.flags |= binding.FICOCO_BACK_TO_BACK       # nothing but reduce steps goes onto the stream below
     gen = torch.Generator().manual_seed(5)
     k1, k2 = g * g // 2, g * g // 4
     attn2 = torch.softmax(1.5 * torch.randn(nb, heads, k1, generator=gen), -1).reshape(-1).to(DEV)
@@ -290,6 +293,110 @@ def test_canaries_around_outputs(ctx):
     assert bool((kidx[pad:pad + rows] >= 0).all())
 
 
+def test_hand_built_ties_follow_the_lower_index(ctx):
+    """The two hand-built tie inputs of tests/golden (bit-identical scores across the selection
+    boundary, and inside one local-penalty window), with no margin repair: the library takes the
+    same decisions as the checker, which the golden file pins by hand."""
+    g = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "hand_example.json")))["tie_cases"]
+    P = np.array(g["patches"], dtype=np.float32)
+    attn = np.array(g["cls_attention"], dtype=np.float32)
+    # the same tokens in a wider batch: copies of the image, plus a bf16 variant with more columns
+    for dtype in ("fp32", "bf16"):
+        tok = P if dtype == "fp32" else synth.f32_to_bf16_bits(np.pad(P, ((0, 0), (0, 4))))
+        for case in g["selection"] + [g["window"]]:
+            penalty = "window" in case
+            batch = synth.VBatch(dtype, False, tok.shape[1], 1, [tok.copy() for _ in range(3)],
+                                 [attn.copy() for _ in range(3)], [np.arange(4, dtype=np.int32)] * 3,
+                                 [(2, 2)] * 3, [case["keep"]] * 3, "ties")
+            p = fo.Params(lam=g["lambda"], local_penalty=penalty)
+            res, results = parity.run_and_compare_v(ctx, batch, p, DEV, what="ties")
+            kidx = binding.to_numpy(res.kept_idx).reshape(3, -1)
+            assert all(kidx[b].tolist() == case["T"] for b in range(3))
+            assert all(sorted(r.S.tolist()) == case["S"] for r in results)
+    # a larger image with many equal scores: identical tokens and attention in groups of four
+    rng = synth.rng_for(95)
+    base = rng.standard_normal((40, 64)).astype(np.float32)
+    tok = np.repeat(base, 4, axis=0)                      # 160 tokens, every score appears four times
+    a = np.repeat(rng.random((2, 40)).astype(np.float32), 4, axis=1)
+    a /= a.sum(axis=1, keepdims=True)
+    for keep, penalty in ((77, False), (82, False), (61, True)):
+        batch = synth.VBatch("fp32", False, 64, 2, [tok], [a], [np.arange(160, dtype=np.int32)], [(10, 16)],
+                             [keep], "ties-wide")
+        res, results = parity.run_and_compare_v(ctx, batch, fo.Params(local_penalty=penalty, max_targets=0), DEV,
+                                                what="ties-wide")
+        # groups straddling the boundary exist (160 - keep is not a multiple of four), and the
+        # checker's scores really tie bit for bit inside a group
+        sraw = results[0].score_raw.reshape(40, 4)
+        assert np.all(sraw == sraw[:, :1]) and (160 - keep) % 4 != 0
+
+
+def test_bounded_wait_runs_out_and_the_context_recovers():
+    """A wait between thread blocks that can never be satisfied (the testing hook makes the fused
+    filter expect one arrival more than there are pieces) must end by itself: the kernels return,
+    bit 2 of the status word is raised, later steps stay off until the status has been read, and
+    after that an ordinary call gives exactly the bytes of a clean run."""
+    c = binding.Context(max_tokens=8192, max_dim=512, max_batch=8, device=0)
+    batch = synth.make_v_batch(96, 6, 16, 16, 256, 4, 128, "bf16", True, 1.2)
+    pk = packing.pack_v(batch, DEV)
+
+    def run():
+        r = c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **pk.call_kwargs())
+        torch.cuda.synchronize()
+        return r
+
+    clean = run()
+    assert c.ficoco_status() == 0
+    ref = [binding.to_numpy(t) for t in (clean.out_tokens, clean.kept_idx, clean.pos_out)]
+    c.ficoco_debug_waits(wait_ns=200_000, extra_arrivals=1)
+    run()
+    c.ficoco_debug_waits(0, 0)
+    sentinel = torch.full_like(clean.out_tokens, 3.0)
+    r2 = c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, out_tokens=sentinel,
+                           **pk.call_kwargs())
+    torch.cuda.synchronize()
+    assert bool((sentinel == 3.0).all()), "a step enqueued after the timeout wrote outputs before the status was read"
+    assert c.ficoco_status() & 4
+    assert c.ficoco_status() == 0
+    for rep in range(2):
+        again = run()
+        assert c.ficoco_status() == 0
+        for a, b in zip(ref, (again.out_tokens, again.kept_idx, again.pos_out)):
+            assert np.array_equal(a, binding.to_numpy(b))
+    c.close()
+
+
+def test_step_behind_a_foreign_producer_kernel(ctx):
+    """Tokens and attention written by other kernels of the same stream right before the step
+    (here: device copies) are read in stream order: by default no kernel of the step starts
+    early.  With FICOCO_BACK_TO_BACK set on steps that do follow each other directly the results
+    are the same bytes."""
+    batch = synth.make_v_batch(97, 16, 24, 24, 512, 4, 288, "bf16", True, 1.5)
+    pk = packing.pack_v(batch, DEV)
+    prm = parity.params_to_abi(fo.Params(), True)
+    ref = ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm, **pk.call_kwargs())
+    torch.cuda.synchronize()
+    want = [binding.to_numpy(t) for t in (ref.out_tokens, ref.kept_idx, ref.pos_out)]
+    tok2, attn2 = torch.zeros_like(pk.tokens), torch.zeros_like(pk.attn)
+    for rep in range(6):
+        tok2.zero_(); attn2.zero_()
+        ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm, **pk.call_kwargs())
+        tok2.copy_(pk.tokens); attn2.copy_(pk.attn)          # the producers
+        got = ctx.ficoco_v_reduce(tok2, attn2, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm,
+                                  n_tokens=pk.n_tokens, pos=pk.pos)
+        torch.cuda.synchronize()
+        for a, b in zip(want, (got.out_tokens, got.kept_idx, got.pos_out)):
+            assert np.array_equal(a, binding.to_numpy(b)), f"repetition {rep}"
+    b2b = parity.params_to_abi(fo.Params(), True)
+    b2b.flags |= binding.FICOCO_BACK_TO_BACK
+    outs = [ctx.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=b2b, **pk.call_kwargs())
+            for _ in range(4)]
+    torch.cuda.synchronize()
+    assert ctx.ficoco_status() == 0
+    for o in outs:
+        for a, b in zip(want, (o.out_tokens, o.kept_idx, o.pos_out)):
+            assert np.array_equal(a, binding.to_numpy(b))
+
+
 def test_error_codes_and_status(ctx):
     batch = synth.make_v_batch(84, 2, 6, 6, 64, 2, 20, "bf16", True, 1.0)
     pk = packing.pack_v(batch, DEV)
@@ -324,6 +431,13 @@ def test_error_codes_and_status(ctx):
     with pytest.raises(binding.FicocoError) as e:
         ctx.ficoco_v_reduce(odd, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, n_tokens=37)
     assert e.value.code == -2
+    # outputs may not overlap inputs (Eq. 2 reads the pre-update tokens)
+    with pytest.raises(binding.FicocoError) as e:
+        call(out_tokens=pk.tokens)
+    assert e.value.code == -1
+    with pytest.raises(binding.FicocoError) as e:
+        call(pos_out=pk.pos)
+    assert e.value.code == -1
     # a position outside the grid is reported through the status word, not a fault
     bad = pk.pos.clone()
     bad[5] = 36 + 1000

@@ -43,3 +43,24 @@ def test_two_ranks_shard_without_exchange_and_take_the_slowest_time():
     assert ms0 == ms1 == 15.0                                     # the slowest rank's time on both
     import bench
     assert v0 == v1 == 2 * bench.B / 15e-3                        # aggregate over both ranks
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself; the dry run
+    takes the same path on CPU (gloo): rank 0 prints one line for n_gpus = 2 with the slowest
+    rank's time and the aggregate over both shards."""
+    import json
+    import subprocess
+    env = dict(os.environ)
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        env.pop(k, None)
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "5", "--dry-run"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    import bench
+    assert line["n_gpus"] == 2 and line["dry_run"] and line["shard_seeds"] == [bench.shard_seed(0), bench.shard_seed(1)]
+    assert abs(line["ms_per_step"] - 15.0 / 5) < 1e-12
+    assert abs(line["value"] - 2 * bench.B / (3.0e-3)) < 1e-6

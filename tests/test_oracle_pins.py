@@ -455,6 +455,48 @@ def test_average_compression_is_the_group_mean():
             assert not np.array_equal(r.out, base.out)
 
 
+def test_convergent_correlation_is_one_mean_token():
+    """Ablation 'convergent correlation' (all discarded tokens merge into one additional token):
+    same S and T as the default method, preserved rows untouched bit for bit, one appended row
+    equal to the plain mean of the discarded rows (scalar loops), kept index -1 for it, the mass
+    identity N^S * extra = sum_{i in S} x_i, a single discarded token reproduced exactly, nothing
+    appended when nothing is discarded, and for FiCoCo-L the row sits before the text rows."""
+    import math
+    batch = tiny_v(41)
+    tok, attn = batch.tokens[0], batch.attn[0]
+    P = tok[1:].astype(np.float64)
+    base = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 9, True, fo.Params())
+    r = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 9, True, fo.Params(convergent=True))
+    assert r.S.tolist() == base.S.tolist() and r.T.tolist() == base.T.tolist()
+    assert r.out.shape[0] == 1 + 9 + 1 and r.kept_idx.tolist() == base.kept_idx.tolist() + [-1]
+    assert np.array_equal(r.out[:10], tok[base.kept_idx])
+    Sl = r.S.tolist()
+    mean = [math.fsum(P[i][d] for i in Sl) / len(Sl) for d in range(P.shape[1])]
+    np.testing.assert_allclose(r.out[10].astype(np.float64), mean, rtol=2e-7, atol=1e-7)
+    np.testing.assert_allclose(len(Sl) * fo.convergent_token(P, r.S), P[Sl].sum(axis=0), atol=1e-12)
+    assert r.pos_out.tolist() == base.pos_out.tolist()
+    one = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 15, True, fo.Params(convergent=True))
+    assert one.out.shape[0] == 17 and np.array_equal(one.out[16], tok[1 + int(one.S[0])])
+    none = fo.ficoco_v_reduce(tok, attn, None, (4, 4), 16, True, fo.Params(convergent=True))
+    assert np.array_equal(none.out, tok) and none.kept_idx.tolist() == list(range(17))
+    # bf16 storage: the mean is rounded once
+    bb = synth.make_v_batch(42, 1, 4, 4, 8, 2, 6, "bf16", True, 1.0)
+    rb = fo.ficoco_v_reduce(bb.tokens[0], bb.attn[0], None, (4, 4), 6, True, fo.Params(convergent=True))
+    Pb = fo.widen(bb.tokens[0])[1:]
+    exact = Pb[rb.S].sum(axis=0) / 10
+    got = fo.widen(rb.out[-1])
+    assert np.all(np.abs(got - exact) <= np.abs(exact) * 2.0 ** -8 + 1e-30)
+    # FiCoCo-L: preserved vision rows, the additional token, then the text rows
+    lb = synth.make_l_batch(43, 1, 14, 5, 8, 3, 6, "fp32", scale=1.0)
+    ld = fo.ficoco_l_reduce(lb.tokens[0], lb.attn_t2v[0], 14, 6, fo.Params())
+    lc = fo.ficoco_l_reduce(lb.tokens[0], lb.attn_t2v[0], 14, 6, fo.Params(convergent=True))
+    assert lc.T.tolist() == ld.T.tolist() and lc.out.shape[0] == 6 + 1 + 5
+    assert lc.kept_idx.tolist() == ld.T.tolist() + [-1] + list(range(14, 19))
+    assert np.array_equal(lc.out[:6], lb.tokens[0][ld.T]) and np.array_equal(lc.out[7:], lb.tokens[0][14:])
+    Pl = lb.tokens[0][:14].astype(np.float64)
+    np.testing.assert_allclose(lc.out[6].astype(np.float64), Pl[lc.S].mean(axis=0), rtol=2e-7, atol=1e-7)
+
+
 def test_relation_argument():
     """The relation argument replaces A^v everywhere and nothing else: (i) given the cosine
     similarity computed by torch it reproduces the default step; (ii) for a symmetric map the two
