@@ -56,6 +56,7 @@ struct Plan {
   WorkItem* d_corr = nullptr;
   WorkItem* d_out = nullptr;
   int n_rows = 0, n_corr = 0, n_out = 0;
+  int out_rows_cta = 0;         // output rows per merge CTA
   // totals and maxima used to size launches and inspection copies
   int tot_patch = 0, tot_src = 0, tot_tgt = 0, tot_out_rows = 0;
   int max_np = 0, max_tgt = 0, max_src = 0, max_rc = 0, max_nwin_cells = 0, max_list = 0;
@@ -67,7 +68,6 @@ struct Plan {
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
   bool need_finalize = false;   // some image merges nothing: its per-token counts are zeroed by a kernel
   bool umma = false;
-  bool csr_in_tail = false;     // the tensor-core correlate kernel also builds the per-target segments
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
   size_t um_smem = 0;
   std::vector<ImgDesc> h_desc;
@@ -167,10 +167,10 @@ struct ficoco_ctx {
   float* tmean = nullptr;
   unsigned* status = nullptr;
   int* tile_cnt = nullptr;  // per source tile: column splits of the correlate kernel that are done
-  int* csr_cnt = nullptr;   // per image: source tiles whose targets and weights are final
-  int* seg_begin = nullptr; // per preserved token (+1 per image): start of its entries in csr_src / csr_w
-  int* csr_src = nullptr;   // (target, source, alpha) entries ordered by target, then token index
-  float* csr_w = nullptr;
+  TgtRec* rec = nullptr;    // per preserved token: the discarded tokens merged into it (first REC_INLINE inline)
+  int* pool_cnt = nullptr;  // per image: entries in the overflow pool
+  PoolEnt* pool = nullptr;  // entries past the inline ones
+  int merge_ctas_per_sm = 1;    // resident CTAs of the merge kernel per SM
   int* img_cnt = nullptr;   // two sets of 3 * max_batch per-image counters of the fused filter kernel
   unsigned long long epoch = 0;          // fused filter launches so far (its parity picks the counter set)
   unsigned long long wait_ns = WAIT_NS_DEFAULT;   // bound of every device-side wait
@@ -382,7 +382,8 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
   const size_t o_icnt = carve(6 * B * 4);
   const size_t o_tcnt = carve((size_t)c->cap_corr * 4);
-  const size_t o_ccnt = carve(B * 4), o_seg = carve((T + B) * 4), o_cs = carve(T * KCAP * 4), o_cwt = carve(T * KCAP * 4);
+  const size_t o_rec = carve(T * sizeof(TgtRec)), o_pcnt = carve(B * 4), o_pool = carve(T * KCAP * sizeof(PoolEnt));
+
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
   const size_t o_pv = carve((size_t)c->cap_part * 4), o_pi = carve((size_t)c->cap_part * 4);
@@ -407,13 +408,12 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
   c->img_cnt = (int*)(b + o_icnt);
   c->tile_cnt = (int*)(b + o_tcnt);
-  c->csr_cnt = (int*)(b + o_ccnt); c->seg_begin = (int*)(b + o_seg);
-  c->csr_src = (int*)(b + o_cs); c->csr_w = (float*)(b + o_cwt);
+  c->rec = (TgtRec*)(b + o_rec); c->pool_cnt = (int*)(b + o_pcnt); c->pool = (PoolEnt*)(b + o_pool);
+
   c->plan_slots = b + o_pl;
 
   // kernels that may need more than 48 KB of dynamic shared memory
   cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  cudaFuncSetAttribute(k_build_csr, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024);
   {
     const int um_smem_max = 221 * 1024;
     cudaFuncSetAttribute(k_correlate_umma<2, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
@@ -437,6 +437,11 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
     FICOCO_FUSED_ATTR(__nv_bfloat16, 1); FICOCO_FUSED_ATTR(__nv_bfloat16, 2); FICOCO_FUSED_ATTR(__nv_bfloat16, 4);
     FICOCO_FUSED_ATTR(__nv_bfloat16, 5); FICOCO_FUSED_ATTR(__nv_bfloat16, 8);
 #undef FICOCO_FUSED_ATTR
+  }
+  {
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_rec<__nv_bfloat16>, 256, 0) == cudaSuccess && nb > 0)
+      c->merge_ctas_per_sm = nb;
   }
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -616,6 +621,15 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     while (out_rows_cta > 2 && n_out_ctas(out_rows_cta) < 2LL * c->num_sms &&
            n_out_ctas(out_rows_cta / 2) <= c->cap_out)
       out_rows_cta /= 2;
+    // a grid a little larger than what the GPU holds at once would run its last CTAs alone: grow
+    // the CTAs (up to MROWS rows) until the grid fits, if that takes at most half as many rows again
+    const long long slots = (long long)c->num_sms * c->merge_ctas_per_sm;
+    if (out_rows_cta == OUT_ROWS_PER_CTA && n_out_ctas(out_rows_cta) > slots) {
+      int r = out_rows_cta;
+      while (r < MROWS && r < OUT_ROWS_PER_CTA * 3 / 2 && n_out_ctas(r) > slots) ++r;
+      if (n_out_ctas(r) <= slots) out_rows_cta = r;
+    }
+    p->out_rows_cta = out_rows_cta;
   }
   for (int b = 0; b < B; ++b) {
     ImgDesc& d = p->h_desc[b];
@@ -670,7 +684,8 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     // output rows
     const int orows = d.n_cls + d.n_tgt + d.n_tail;
     for (int r0 = 0; r0 < orows; r0 += out_rows_cta) {
-      WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < out_rows_cta) ? orows - r0 : out_rows_cta; w.aux = 0;
+      WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < out_rows_cta) ? orows - r0 : out_rows_cta;
+      w.aux = r0 / out_rows_cta;
       outw.push_back(w);
     }
     row0 += key.ntok[b]; patch0 += d.np; out0 += orows; src0 += d.n_src; tgt0 += d.n_tgt;
@@ -753,7 +768,6 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     if (p->um_smem < epi) p->um_smem = epi;
     if (p->um_smem > 220 * 1024) return FICOCO_ERR_UNSUPPORTED;
   }
-  p->csr_in_tail = p->umma && csr_work_bytes(p->max_tgt) + 1024 <= p->um_smem;
 
   char* slot_dev = c->plan_slots + (size_t)slot * c->slot_bytes;
   p->d_desc = (ImgDesc*)slot_dev;
@@ -853,7 +867,7 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
                             p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), c->wait_ns,
-                            c->dbg_extra_arrivals);
+                            c->dbg_extra_arrivals, MergeLists{c->rec, c->pool_cnt, c->pool});
 }
 
 template <class T, int VPL>
@@ -873,6 +887,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
+  const MergeLists ml{c->rec, c->pool_cnt, c->pool};
   const size_t in_rows = (size_t)p->tot_patch + (size_t)p->key.batch * (p->key.has_cls + (p->key.mode == 1 ? p->key.n_text : 0));
   const Span in_spans[3] = {span_of(tok, in_rows * D * sizeof(T)),
                             span_of(attn, (size_t)attn_rows * p->tot_patch * sizeof(float)),
@@ -940,13 +955,9 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   // images of up to 1024 tokens: half the threads (two tokens each), cheaper barriers
   k_select<<<p->key.batch, p->max_np <= 1024 ? 512 : 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
-                                                  pos_out, c->status);
+                                                  pos_out, c->status, ml);
   c->launches += 1;
   }
-  CsrArgs csr = {};
-  csr.S_idx = c->S_idx; csr.tmp_src = c->part_idx; csr.tmp_w = c->part_val; csr.seg_begin = c->seg_begin;
-  csr.csr_src = c->csr_src; csr.csr_w = c->csr_w; csr.img_tiles = c->csr_cnt;
-  bool csr_done = false;
   if (p->n_corr > 0) {
     if (rel) {
       prof_tick(c, st, "correlate_relation");
@@ -956,21 +967,20 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #define FICOCO_REL_GO(LC)                                                                              \
   k_correlate_rel<LC><<<p->n_corr, 256, (size_t)rel_cols * sizeof(int), st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
                                                  c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-                                                 c->e_w, c->e_c)
+                                                 c->e_w, c->e_c, ml)
       if (p->max_list <= 2) FICOCO_REL_GO(2);
       else if (p->max_list <= 4) FICOCO_REL_GO(4);
       else FICOCO_REL_GO(16);
 #undef FICOCO_REL_GO
     } else if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
-      csr_done = p->csr_in_tail;
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
 #define FICOCO_UMMA_LAUNCH(NS, LC)                                                                     \
   launch_dependent(k_correlate_umma<NS, LC>, p->n_corr, UTHREADS, p->um_smem, st, tk, D,               \
       (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
       (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
       p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-      c->e_w, c->e_c, tmean, M, p->max_np, gamma, c->wait_ns, csr, p->csr_in_tail ? 1 : 0)
+      c->e_w, c->e_c, tmean, M, p->max_np, gamma, c->wait_ns, ml)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 6) FICOCO_UMMA_LAUNCH(6, LC);                                                  \
@@ -988,27 +998,23 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
                                                      c->T_idx, tmean, M, gamma, c->part_val, c->part_idx,
                                                      c->tile_cnt, c->corr_cnt, c->tau,
-                                                     c->e_tgt, c->e_w, c->e_c);
+                                                     c->e_tgt, c->e_w, c->e_c, ml);
     }
     c->launches += 1;
   }
   if (p->max_src > 0 && p->need_finalize) {
     prof_tick(c, st, "finalize");
     k_finalize_src<<<dim3(p->key.batch, (p->max_src + 255) / 256), 256, 0, st>>>(
-        p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c);
-    c->launches += 1;
-  }
-  if (p->n_corr > 0 && !csr_done) {
-    prof_tick(c, st, "build_segments");
-    k_build_csr<<<p->key.batch, 256, csr_work_bytes(p->max_tgt), st>>>(p->d_desc, c->e_tgt, c->e_w, csr, c->status);
+        p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c, c->S_idx, ml);
     c->launches += 1;
   }
   prof_tick(c, st, "merge_compact");
   const int after_correlate = p->n_corr > 0 ? 1 : 0;   // else the grid before may be the filter itself
-  launch_dependent(k_merge_csr<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
-                   (const WorkItem*)p->d_out, (const int*)c->T_idx, (const int*)c->seg_begin,
-                   (const int*)c->csr_src, (const float*)c->csr_w, out_tokens, after_correlate,
-                   (const unsigned*)c->status);
+  launch_dependent(k_merge_rec<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+                   (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
+                   (const int*)c->e_tgt, (const float*)c->e_w, (const TgtRec*)c->rec, (const int*)c->pool_cnt,
+                   (const PoolEnt*)c->pool, out_tokens, after_correlate, (const unsigned*)c->status,
+                   p->out_rows_cta);
   c->launches += 1;
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);
@@ -1140,7 +1146,6 @@ extern "C" int ficoco_status(ficoco_ctx* c, void* cuda_stream, int* device_statu
     // a kernel gave up half-way: its per-image counters may be left non-zero
     CUDA_TRY(c, cudaMemsetAsync(c->img_cnt, 0, 6 * (size_t)c->max_batch * sizeof(int), st));
     CUDA_TRY(c, cudaMemsetAsync(c->tile_cnt, 0, (size_t)c->cap_corr * sizeof(int), st));
-    CUDA_TRY(c, cudaMemsetAsync(c->csr_cnt, 0, (size_t)c->max_batch * sizeof(int), st));
     CUDA_TRY(c, cudaStreamSynchronize(st));
   }
   *device_status = (int)v;

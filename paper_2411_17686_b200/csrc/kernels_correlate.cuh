@@ -11,26 +11,13 @@ constexpr int CBM = 64;   // source rows per CTA
 constexpr int CBN = 64;   // target columns per tile
 constexpr int CKC = 16;   // reduction chunk
 
-// Per-target segments for the merge kernel, see csr_build_image().
-struct CsrArgs {
-  const int* S_idx;
-  int* tmp_src;        // scratch, at least n_src * L entries per image at d.part0
-  float* tmp_w;
-  int* seg_begin;      // [sum_b (n_tgt_b + 1)]: image b's segment starts at d.tgt0 + b
-  int* csr_src;        // per image at d.ent0: token index of every (target, source) entry
-  float* csr_w;        // alpha of that entry
-  int* img_tiles;      // per image: source tiles finalized so far
-  unsigned char* work; // shared memory of csr_work_bytes(n_tgt) bytes, or nullptr: a later kernel builds the segments
-  int* scan_tmp;       // 33 ints of shared memory
-};
-
 template <int LC>
 __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
     const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
     int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem,
-    const CsrArgs& csr);
+    const int* __restrict__ S_idx, const MergeLists& ml);
 
 // ---------------------------------------------------------------------------------------
 // fp32 SIMT correlate (the path for fp32 tokens, where 1e-5 relative accuracy rules out
@@ -48,7 +35,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     const float* __restrict__ tmean, int M, float gamma,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ img_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c) {
+    float* __restrict__ e_w, float* __restrict__ e_c, MergeLists ml) {
   __shared__ int is_last;
   __shared__ __align__(16) float As[CKC][CBM + 4];
   __shared__ __align__(16) float Bs[CKC][CBN + 4];
@@ -208,9 +195,8 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     part_val[o] = lv[r][k];
     part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
   }
-  CsrArgs no_csr = {};
   correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last,
-                       no_csr);
+                       S_idx, ml);
 }
 
 }  // namespace ficoco
@@ -222,15 +208,16 @@ namespace ficoco {
 //   tau_i = v[L-1] + frac * (v[L-2] - v[L-1])  (v descending: the two order statistics around
 //   eps*(n-1)), J_i = { entries >= tau_i }, alpha_ij = C+_ij / sum_{J_i} C+  (Eq. 2).
 // Results go to compact per-image arrays with L slots per token: e_tgt (position in T, or -1),
-// e_w (alpha), e_c (the L largest C, descending).
+// e_w (alpha), e_c (the L largest C, descending), and every (target, token, alpha) entry is
+// filed under its target for the merge kernel (record of the preserved token, overflow pool).
 // grid = (images, ceil(max N^S / 256)).
 // ---------------------------------------------------------------------------------------
 // LC: compile-time bound on the list length L of the image (lists live in registers).
 template <int LC>
 __device__ __forceinline__ void finalize_source(
-    const ImgDesc& d, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
+    const ImgDesc& d, int img, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c) {
+    float* __restrict__ e_w, float* __restrict__ e_c, const int* __restrict__ S_idx, const MergeLists& ml) {
   const int L = d.list_len;
   const size_t o = (size_t)(d.src0 + s);
   if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; return; }
@@ -285,12 +272,26 @@ __device__ __forceinline__ void finalize_source(
   corr_cnt[o] = nj;
   tau_out[o] = tau;
   const size_t eb = (size_t)d.ent0 + (size_t)s * L;
+  const int tok = nj > 0 ? S_idx[d.src0 + s] : 0;
 #pragma unroll
   for (int k = 0; k < LC; ++k) {
     if (k < L) {
+      const float wk = k < nj ? (d.avg ? 1.0f : fmaxf(v[k], 0.f) / den) : 0.f;
       e_tgt[eb + k] = k < nj ? ix[k] : -1;
-      e_w[eb + k] = k < nj ? (d.avg ? 1.0f : fmaxf(v[k], 0.f) / den) : 0.f;
+      e_w[eb + k] = wk;
       e_c[eb + k] = v[k];
+      if (k < nj) {
+        TgtRec* r = ml.rec + d.tgt0 + ix[k];
+        const int slot = atomicAdd(&r->cnt, 1);
+        if (slot < REC_INLINE) {
+          r->e[slot] = make_int2(tok, __float_as_int(wk));
+        } else {
+          const int q = atomicAdd(ml.pool_cnt + img, 1);
+          PoolEnt pe;
+          pe.tgt = ix[k]; pe.src = tok; pe.w = wk; pe.pad = 0;
+          ml.pool[(size_t)d.ent0 + q] = pe;
+        }
+      }
     }
   }
 }
@@ -298,93 +299,26 @@ __device__ __forceinline__ void finalize_source(
 __global__ void __launch_bounds__(256) k_finalize_src(
     const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
-    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
+    const int* __restrict__ S_idx, MergeLists ml) {
   const ImgDesc d = desc[blockIdx.x];
   const int s = blockIdx.y * 256 + threadIdx.x;
   if (s >= d.n_src) return;
-  finalize_source<KCAP>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
-}
-
-// ---------------------------------------------------------------------------------------
-// Per-target segments ("CSR by target") of one image for the merge kernel: the (target, source,
-// alpha) entries that the correlate step leaves per discarded token are counted per preserved
-// token, placed by a prefix sum and ordered by token index inside every segment, so that the merge
-// kernel finds the sources of an output row as one contiguous, ordered run and the fp32 sums of
-// Eq. 2 have one fixed order.  One CTA (`nthr` threads on barrier `bar`) per image.
-//   seg_begin[t] .. seg_begin[t + 1]  : entries of preserved token t (position in T) in csr_src / csr_w
-// `work`: shared memory, csr_work_bytes(n_tgt) bytes.
-// ---------------------------------------------------------------------------------------
-__host__ __device__ inline size_t csr_work_bytes(int n_tgt) { return (size_t)(2 * n_tgt + 2) * sizeof(int); }
-
-__device__ __noinline__ void csr_build_image(const ImgDesc& d, int img, const int* __restrict__ e_tgt,
-                                             const float* __restrict__ e_w, const CsrArgs& a, int tid, int nthr,
-                                             int bar) {
-  const int nt = d.n_tgt, L = d.list_len, n_ent = d.n_src * L;
-  int* begv = reinterpret_cast<int*>(a.work);     // [nt + 1] counts, then segment begins
-  int* cur = begv + nt + 1;                        // [nt] fill cursors
-  int* sb = a.seg_begin + d.tgt0 + img;
-  #pragma unroll 1
-  for (int t = tid; t <= nt; t += nthr) begv[t] = 0;
-  cta_sync(bar, nthr);
-  #pragma unroll 1
-  for (int e = tid; e < n_ent; e += nthr) {
-    const int t = __ldcg(e_tgt + d.ent0 + e);
-    if (t >= 0) atomicAdd(&begv[t], 1);
-  }
-  cta_sync(bar, nthr);
-  int carry = 0;
-  #pragma unroll 1
-  for (int base = 0; base < nt; base += nthr) {
-    const int t = base + tid;
-    const int v = t < nt ? begv[t] : 0;
-    int tot;
-    const int ex = block_exclusive_scan(v, a.scan_tmp, &tot, bar, nthr);
-    if (t < nt) { begv[t] = carry + ex; cur[t] = carry + ex; sb[t] = carry + ex; }
-    carry += tot;
-  }
-  if (tid == 0) { begv[nt] = carry; sb[nt] = carry; }
-  cta_sync(bar, nthr);
-  // fill, in whatever order the atomics hand out the slots
-  #pragma unroll 1
-  for (int e = tid; e < n_ent; e += nthr) {
-    const int t = __ldcg(e_tgt + d.ent0 + e);
-    if (t >= 0) {
-      const int slot = atomicAdd(&cur[t], 1);
-      a.tmp_src[d.part0 + slot] = a.S_idx[d.src0 + e / L];
-      a.tmp_w[d.part0 + slot] = __ldcg(e_w + d.ent0 + e);
-    }
-  }
-  cta_sync(bar, nthr);
-  // order every segment by token index: the rank of an entry inside its segment is its place
-  #pragma unroll 1
-  for (int i = tid; i < carry; i += nthr) {
-    int lo = 0, hi = nt - 1;                       // the last t with begv[t] <= i and a non-empty segment
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (begv[mid] <= i) lo = mid; else hi = mid - 1;
-    }
-    const int b = begv[lo], e2 = begv[lo + 1];
-    const int my = __ldcg(a.tmp_src + d.part0 + i);
-    int rank = 0;
-    for (int k = b; k < e2; ++k) rank += __ldcg(a.tmp_src + d.part0 + k) < my ? 1 : 0;
-    a.csr_src[d.ent0 + b + rank] = my;
-    a.csr_w[d.ent0 + b + rank] = __ldcg(a.tmp_w + d.part0 + i);
-  }
+  finalize_source<KCAP>(d, (int)blockIdx.x, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, S_idx, ml);
 }
 
 // Tail of a correlate CTA: once its partial lists are written it bumps the counter of its
 // source tile (`tile` = index of the tile's first work item); the CTA that completes the tile
 // (the last of its d.nsplit column splits) turns the partial lists of the tile's discarded
-// tokens into tau_i, J_i and alpha_ij, and resets the counter.  The CTA that completes the
-// image's last tile then builds the image's per-target segments (when csr.work is given).
-// Nobody waits: there is no spinning.  Call from all threads of the CTA.
+// tokens into tau_i, J_i and alpha_ij, and resets the counter.  Nobody waits: there is no
+// spinning.  Call from all threads of the CTA.
 template <int LC>
 __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
     const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
     int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem,
-    const CsrArgs& csr) {
+    const int* __restrict__ S_idx, const MergeLists& ml) {
   __syncthreads();
   if (threadIdx.x == 0) {
     // publishes this CTA's partial lists and, for the split that arrives last, observes the others'
@@ -394,34 +328,9 @@ __device__ __forceinline__ void correlate_tail(
     *is_last_smem = last;
   }
   __syncthreads();
-  if (!*is_last_smem) return;
-  for (int s = w.r0 + (int)threadIdx.x; s < w.r0 + w.nrows; s += blockDim.x)
-    finalize_source<LC>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
-  if (csr.work == nullptr) return;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int n_tiles = d.corr_items / d.nsplit;
-    const int old = atom_acq_rel_add(&csr.img_tiles[w.img], 1);
-    const int last = old == n_tiles - 1;
-    if (last) csr.img_tiles[w.img] = 0;
-    *is_last_smem = last;
-  }
-  __syncthreads();
-  if (*is_last_smem) csr_build_image(d, w.img, e_tgt, e_w, csr, (int)threadIdx.x, (int)blockDim.x, 0);
-}
-
-// Segments built by a kernel of their own (one CTA per image) where the correlate kernel has no
-// shared memory to spare for them.
-__global__ void __launch_bounds__(256) k_build_csr(const ImgDesc* __restrict__ desc, const int* __restrict__ e_tgt,
-                                                   const float* __restrict__ e_w, CsrArgs a,
-                                                   const unsigned* __restrict__ status) {
-  extern __shared__ unsigned char csr_smem[];
-  __shared__ int scan_tmp[33];
-  const ImgDesc d = desc[blockIdx.x];
-  if (d.list_len == 0 || (*status & STATUS_TIMEOUT)) return;
-  a.work = csr_smem;
-  a.scan_tmp = scan_tmp;
-  csr_build_image(d, (int)blockIdx.x, e_tgt, e_w, a, (int)threadIdx.x, 256, 0);
+  if (*is_last_smem)
+    for (int s = w.r0 + (int)threadIdx.x; s < w.r0 + w.nrows; s += blockDim.x)
+      finalize_source<LC>(d, w.img, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, S_idx, ml);
 }
 
 }  // namespace ficoco

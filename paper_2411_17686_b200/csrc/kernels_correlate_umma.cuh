@@ -169,15 +169,13 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
     int stage_bytes, int a_bytes, int tmem_cols, int* __restrict__ img_done, int* __restrict__ corr_cnt,
     float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
-    const float* __restrict__ tmean, int M, int NV, float gamma, unsigned long long wait_ns, CsrArgs csr,
-    int csr_in_tail) {
+    const float* __restrict__ tmean, int M, int NV, float gamma, unsigned long long wait_ns, MergeLists ml) {
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
   __shared__ int rowS[UM * UM_SUB], rowT[UN_MAX];
   __shared__ float rnT[UN_MAX];
   __shared__ int failed, acc_committed, is_last, dead;
-  __shared__ int csr_scan_tmp[33];
 
   FICOCO_PHASE(1, 0);
   const WorkItem w = work[blockIdx.x];
@@ -444,11 +442,8 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tmem_cols)
                  : "memory");
   }
-  // the operand ring is idle by now: the CTA that completes its image sorts the image's entries there
-  csr.work = csr_in_tail ? um_raw + (ring - smem_u32(um_raw)) : nullptr;
-  csr.scan_tmp = csr_scan_tmp;
   correlate_tail<LCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c,
-                       &is_last, csr);
+                       &is_last, S_idx, ml);
   FICOCO_PHASE(1, 8);
 }
 
