@@ -39,24 +39,6 @@ struct ImgDesc {
   long long rel0;  // offset (floats) of this image's [Np, Np] relation block (relation mode)
 };
 
-// What the correlate step leaves for the merge kernel, per preserved token: how many discarded
-// tokens are merged into it and the first REC_INLINE of them (token index, alpha); entries past
-// that go to a per-image overflow pool.  Entries arrive in no particular order (the slot comes
-// from an atomic counter); the merge kernel orders them by token index before it sums.
-constexpr int REC_INLINE = 7;
-struct __align__(16) TgtRec {
-  int cnt;                 // all entries of this token, inline and pooled
-  int pad;
-  int2 e[REC_INLINE];      // (token index inside the image, alpha as bits)
-};
-static_assert(sizeof(TgtRec) == 64, "one record is four 16-byte vectors");
-struct __align__(16) PoolEnt { int tgt; int src; float w; int pad; };   // tgt: position in T
-struct MergeLists {
-  TgtRec* rec;       // [sum_b n_tgt_b], image b at d.tgt0
-  int* pool_cnt;     // [batch] entries in the image's pool
-  PoolEnt* pool;     // image b at d.ent0, at most n_src * L entries
-};
-
 struct WorkItem {
   int img;
   int r0;      // first row (patch / source slot / output row) inside the image

@@ -167,9 +167,6 @@ struct ficoco_ctx {
   float* tmean = nullptr;
   unsigned* status = nullptr;
   int* tile_cnt = nullptr;  // per source tile: column splits of the correlate kernel that are done
-  TgtRec* rec = nullptr;    // per preserved token: the discarded tokens merged into it (first REC_INLINE inline)
-  int* pool_cnt = nullptr;  // per image: entries in the overflow pool
-  PoolEnt* pool = nullptr;  // entries past the inline ones
   int merge_ctas_per_sm = 1;    // resident CTAs of the merge kernel per SM
   int* img_cnt = nullptr;   // two sets of 3 * max_batch per-image counters of the fused filter kernel
   unsigned long long epoch = 0;          // fused filter launches so far (its parity picks the counter set)
@@ -382,7 +379,6 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
   const size_t o_icnt = carve(6 * B * 4);
   const size_t o_tcnt = carve((size_t)c->cap_corr * 4);
-  const size_t o_rec = carve(T * sizeof(TgtRec)), o_pcnt = carve(B * 4), o_pool = carve(T * KCAP * sizeof(PoolEnt));
 
   const size_t o_sraw = carve(T * 4), o_spen = carve(T * 4);
   const size_t o_S = carve(T * 4), o_T = carve(T * 4);
@@ -408,7 +404,6 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->tmean = (float*)(b + o_tm); c->status = (unsigned*)(b + o_st);
   c->img_cnt = (int*)(b + o_icnt);
   c->tile_cnt = (int*)(b + o_tcnt);
-  c->rec = (TgtRec*)(b + o_rec); c->pool_cnt = (int*)(b + o_pcnt); c->pool = (PoolEnt*)(b + o_pool);
 
   c->plan_slots = b + o_pl;
 
@@ -440,7 +435,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   }
   {
     int nb = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_rec<__nv_bfloat16>, 256, 0) == cudaSuccess && nb > 0)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_scan<__nv_bfloat16>, 256, 0) == cudaSuccess && nb > 0)
       c->merge_ctas_per_sm = nb;
   }
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -621,14 +616,6 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     while (out_rows_cta > 2 && n_out_ctas(out_rows_cta) < 2LL * c->num_sms &&
            n_out_ctas(out_rows_cta / 2) <= c->cap_out)
       out_rows_cta /= 2;
-    // a grid a little larger than what the GPU holds at once would run its last CTAs alone: grow
-    // the CTAs (up to MROWS rows) until the grid fits, if that takes at most half as many rows again
-    const long long slots = (long long)c->num_sms * c->merge_ctas_per_sm;
-    if (out_rows_cta == OUT_ROWS_PER_CTA && n_out_ctas(out_rows_cta) > slots) {
-      int r = out_rows_cta;
-      while (r < MROWS && r < OUT_ROWS_PER_CTA * 3 / 2 && n_out_ctas(r) > slots) ++r;
-      if (n_out_ctas(r) <= slots) out_rows_cta = r;
-    }
     p->out_rows_cta = out_rows_cta;
   }
   for (int b = 0; b < B; ++b) {
@@ -867,7 +854,7 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
                             p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), c->wait_ns,
-                            c->dbg_extra_arrivals, MergeLists{c->rec, c->pool_cnt, c->pool});
+                            c->dbg_extra_arrivals);
 }
 
 template <class T, int VPL>
@@ -887,7 +874,6 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   constexpr int E = VecTraits<T>::E;
   const int nvec = D / E;
   const int vpl = (nvec + 31) / 32;
-  const MergeLists ml{c->rec, c->pool_cnt, c->pool};
   const size_t in_rows = (size_t)p->tot_patch + (size_t)p->key.batch * (p->key.has_cls + (p->key.mode == 1 ? p->key.n_text : 0));
   const Span in_spans[3] = {span_of(tok, in_rows * D * sizeof(T)),
                             span_of(attn, (size_t)attn_rows * p->tot_patch * sizeof(float)),
@@ -955,7 +941,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   // images of up to 1024 tokens: half the threads (two tokens each), cheaper barriers
   k_select<<<p->key.batch, p->max_np <= 1024 ? 512 : 1024, sel_smem, st>>>(p->d_desc, c->s_raw, pos, window, coef, penalty,
                                                   c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx,
-                                                  pos_out, c->status, ml);
+                                                  pos_out, c->status);
   c->launches += 1;
   }
   if (p->n_corr > 0) {
@@ -967,7 +953,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #define FICOCO_REL_GO(LC)                                                                              \
   k_correlate_rel<LC><<<p->n_corr, 256, (size_t)rel_cols * sizeof(int), st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
                                                  c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-                                                 c->e_w, c->e_c, ml)
+                                                 c->e_w, c->e_c)
       if (p->max_list <= 2) FICOCO_REL_GO(2);
       else if (p->max_list <= 4) FICOCO_REL_GO(4);
       else FICOCO_REL_GO(16);
@@ -980,7 +966,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
       (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
       p->um_stage_bytes, p->um_a_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-      c->e_w, c->e_c, tmean, M, p->max_np, gamma, c->wait_ns, ml)
+      c->e_w, c->e_c, tmean, M, p->max_np, gamma, c->wait_ns)
 #define FICOCO_UMMA_STAGES(LC)                                                                         \
   do {                                                                                                 \
     if (p->um_nstage == 6) FICOCO_UMMA_LAUNCH(6, LC);                                                  \
@@ -998,23 +984,22 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
                                                      c->T_idx, tmean, M, gamma, c->part_val, c->part_idx,
                                                      c->tile_cnt, c->corr_cnt, c->tau,
-                                                     c->e_tgt, c->e_w, c->e_c, ml);
+                                                     c->e_tgt, c->e_w, c->e_c);
     }
     c->launches += 1;
   }
   if (p->max_src > 0 && p->need_finalize) {
     prof_tick(c, st, "finalize");
     k_finalize_src<<<dim3(p->key.batch, (p->max_src + 255) / 256), 256, 0, st>>>(
-        p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c, c->S_idx, ml);
+        p->d_desc, c->part_val, c->part_idx, c->corr_cnt, c->tau, c->e_tgt, c->e_w, c->e_c);
     c->launches += 1;
   }
   prof_tick(c, st, "merge_compact");
   const int after_correlate = p->n_corr > 0 ? 1 : 0;   // else the grid before may be the filter itself
-  launch_dependent(k_merge_rec<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+  launch_dependent(k_merge_scan<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
                    (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
-                   (const int*)c->e_tgt, (const float*)c->e_w, (const TgtRec*)c->rec, (const int*)c->pool_cnt,
-                   (const PoolEnt*)c->pool, out_tokens, after_correlate, (const unsigned*)c->status,
-                   p->out_rows_cta);
+                   (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
+                   (const unsigned*)c->status);
   c->launches += 1;
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);

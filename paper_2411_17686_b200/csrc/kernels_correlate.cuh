@@ -16,8 +16,7 @@ __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
     const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
-    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem,
-    const int* __restrict__ S_idx, const MergeLists& ml);
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem);
 
 // ---------------------------------------------------------------------------------------
 // fp32 SIMT correlate (the path for fp32 tokens, where 1e-5 relative accuracy rules out
@@ -35,7 +34,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     const float* __restrict__ tmean, int M, float gamma,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ img_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c, MergeLists ml) {
+    float* __restrict__ e_w, float* __restrict__ e_c) {
   __shared__ int is_last;
   __shared__ __align__(16) float As[CKC][CBM + 4];
   __shared__ __align__(16) float Bs[CKC][CBN + 4];
@@ -195,8 +194,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     part_val[o] = lv[r][k];
     part_idx[o] = li[r][k] == INT_MAX ? -1 : li[r][k];
   }
-  correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last,
-                       S_idx, ml);
+  correlate_tail<KCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
@@ -208,16 +206,15 @@ namespace ficoco {
 //   tau_i = v[L-1] + frac * (v[L-2] - v[L-1])  (v descending: the two order statistics around
 //   eps*(n-1)), J_i = { entries >= tau_i }, alpha_ij = C+_ij / sum_{J_i} C+  (Eq. 2).
 // Results go to compact per-image arrays with L slots per token: e_tgt (position in T, or -1),
-// e_w (alpha), e_c (the L largest C, descending), and every (target, token, alpha) entry is
-// filed under its target for the merge kernel (record of the preserved token, overflow pool).
+// e_w (alpha), e_c (the L largest C, descending).
 // grid = (images, ceil(max N^S / 256)).
 // ---------------------------------------------------------------------------------------
 // LC: compile-time bound on the list length L of the image (lists live in registers).
 template <int LC>
 __device__ __forceinline__ void finalize_source(
-    const ImgDesc& d, int img, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
+    const ImgDesc& d, int s, const float* __restrict__ part_val, const int* __restrict__ part_idx,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c, const int* __restrict__ S_idx, const MergeLists& ml) {
+    float* __restrict__ e_w, float* __restrict__ e_c) {
   const int L = d.list_len;
   const size_t o = (size_t)(d.src0 + s);
   if (L == 0) { corr_cnt[o] = 0; tau_out[o] = 0.f; return; }
@@ -272,26 +269,12 @@ __device__ __forceinline__ void finalize_source(
   corr_cnt[o] = nj;
   tau_out[o] = tau;
   const size_t eb = (size_t)d.ent0 + (size_t)s * L;
-  const int tok = nj > 0 ? S_idx[d.src0 + s] : 0;
 #pragma unroll
   for (int k = 0; k < LC; ++k) {
     if (k < L) {
-      const float wk = k < nj ? (d.avg ? 1.0f : fmaxf(v[k], 0.f) / den) : 0.f;
       e_tgt[eb + k] = k < nj ? ix[k] : -1;
-      e_w[eb + k] = wk;
+      e_w[eb + k] = k < nj ? (d.avg ? 1.0f : fmaxf(v[k], 0.f) / den) : 0.f;
       e_c[eb + k] = v[k];
-      if (k < nj) {
-        TgtRec* r = ml.rec + d.tgt0 + ix[k];
-        const int slot = atomicAdd(&r->cnt, 1);
-        if (slot < REC_INLINE) {
-          r->e[slot] = make_int2(tok, __float_as_int(wk));
-        } else {
-          const int q = atomicAdd(ml.pool_cnt + img, 1);
-          PoolEnt pe;
-          pe.tgt = ix[k]; pe.src = tok; pe.w = wk; pe.pad = 0;
-          ml.pool[(size_t)d.ent0 + q] = pe;
-        }
-      }
     }
   }
 }
@@ -299,12 +282,11 @@ __device__ __forceinline__ void finalize_source(
 __global__ void __launch_bounds__(256) k_finalize_src(
     const ImgDesc* __restrict__ desc, const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
-    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
-    const int* __restrict__ S_idx, MergeLists ml) {
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c) {
   const ImgDesc d = desc[blockIdx.x];
   const int s = blockIdx.y * 256 + threadIdx.x;
   if (s >= d.n_src) return;
-  finalize_source<KCAP>(d, (int)blockIdx.x, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, S_idx, ml);
+  finalize_source<KCAP>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
 // Tail of a correlate CTA: once its partial lists are written it bumps the counter of its
@@ -317,8 +299,7 @@ __device__ __forceinline__ void correlate_tail(
     const ImgDesc& d, const WorkItem& w, int tile, int* __restrict__ tile_done,
     const float* __restrict__ part_val,
     const int* __restrict__ part_idx, int* __restrict__ corr_cnt, float* __restrict__ tau_out,
-    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem,
-    const int* __restrict__ S_idx, const MergeLists& ml) {
+    int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c, int* is_last_smem) {
   __syncthreads();
   if (threadIdx.x == 0) {
     // publishes this CTA's partial lists and, for the split that arrives last, observes the others'
@@ -330,7 +311,7 @@ __device__ __forceinline__ void correlate_tail(
   __syncthreads();
   if (*is_last_smem)
     for (int s = w.r0 + (int)threadIdx.x; s < w.r0 + w.nrows; s += blockDim.x)
-      finalize_source<LC>(d, w.img, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c, S_idx, ml);
+      finalize_source<LC>(d, s, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c);
 }
 
 }  // namespace ficoco

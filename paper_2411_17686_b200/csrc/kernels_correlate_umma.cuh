@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
     float* __restrict__ part_val, int* __restrict__ part_idx, unsigned* __restrict__ status,
     int stage_bytes, int a_bytes, int tmem_cols, int* __restrict__ img_done, int* __restrict__ corr_cnt,
     float* __restrict__ tau_out, int* __restrict__ e_tgt, float* __restrict__ e_w, float* __restrict__ e_c,
-    const float* __restrict__ tmean, int M, int NV, float gamma, unsigned long long wait_ns, MergeLists ml) {
+    const float* __restrict__ tmean, int M, int NV, float gamma, unsigned long long wait_ns) {
   extern __shared__ unsigned char um_raw[];
   __shared__ uint64_t full_bar[NSTAGE], empty_bar[NSTAGE], acc_bar;
   __shared__ uint32_t tmem_base_s;
@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
                  : "memory");
   }
   correlate_tail<LCAP>(d, w, (int)blockIdx.x - w.aux, img_done, part_val, part_idx, corr_cnt, tau_out, e_tgt, e_w, e_c,
-                       &is_last, S_idx, ml);
+                       &is_last);
   FICOCO_PHASE(1, 8);
 }
 

@@ -260,10 +260,8 @@ __device__ __noinline__ void select_image(
     const ImgDesc& d, const float* s_raw, const int* __restrict__ pos, int window, float coef,
     int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
     int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
-    unsigned* __restrict__ status, unsigned char* work, SelectShared& sh, int tid, int nthr, int bar,
-    const MergeLists& ml, int img) {
+    unsigned* __restrict__ status, unsigned char* work, SelectShared& sh, int tid, int nthr, int bar) {
   const int np = d.np;
-  if (tid == 0) ml.pool_cnt[img] = 0;            // the merge lists of this image start empty
   uint32_t* keys = reinterpret_cast<uint32_t*>(work);
   float* sc = reinterpret_cast<float*>(work + (size_t)np * 4);
   int* pp = reinterpret_cast<int*>(work + (size_t)np * 8);
@@ -415,7 +413,6 @@ __device__ __noinline__ void select_image(
       } else {
         const int tp = i - sel_rank;
         T_idx[d.tgt0 + tp] = i;
-        ml.rec[d.tgt0 + tp].cnt = 0;
         kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
         if (pos_out) pos_out[d.tgt0 + tp] = pp[i];
       }
@@ -492,7 +489,7 @@ __device__ __noinline__ void select_small(
     int penalty, float* __restrict__ s_pen, float* __restrict__ scores_out, int* __restrict__ S_idx,
     int* __restrict__ T_idx, int* __restrict__ kept_idx, int* __restrict__ pos_out,
     unsigned* __restrict__ status, unsigned char* work, SelectSmallShared& sh, int tid, int bar,
-    int w_lo, int w_hi, const MergeLists& ml, int img) {
+    int w_lo, int w_hi) {
   constexpr int NT = SEL_SMALL_THREADS;
   const int np = d.np, lane = tid & 31, warp = tid >> 5;
   const SelectSmallWork wk = select_small_layout(work, np);
@@ -684,14 +681,12 @@ __device__ __noinline__ void select_small(
       } else {
         const int tp = i - rank;
         T_idx[d.tgt0 + tp] = i;
-        ml.rec[d.tgt0 + tp].cnt = 0;               // the merge list of this preserved token starts empty
         kept_idx[d.out_row0 + d.n_cls + tp] = d.n_cls + i;
         if (pos_out) pos_out[d.tgt0 + tp] = pp[q];
       }
     }
   }
   if (w_lo == 0) {
-    if (tid == 0) ml.pool_cnt[img] = 0;
     #pragma unroll 1
     for (int i = tid; i < d.n_cls; i += NT) kept_idx[d.out_row0 + i] = i;
     #pragma unroll 1
@@ -708,7 +703,7 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
                                                  float* __restrict__ scores_out,
                                                  int* __restrict__ S_idx, int* __restrict__ T_idx,
                                                  int* __restrict__ kept_idx, int* __restrict__ pos_out,
-                                                 unsigned* __restrict__ status, MergeLists ml) {
+                                                 unsigned* __restrict__ status) {
   extern __shared__ unsigned char sm_raw[];
   __shared__ SelectShared sh;
   __shared__ SelectSmallShared shs;
@@ -717,11 +712,11 @@ __global__ void __launch_bounds__(1024) k_select(const ImgDesc* __restrict__ des
     select_small_prepare(d, penalty, sm_raw, threadIdx.x);
     __syncthreads();
     select_small(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-                 status, sm_raw, shs, threadIdx.x, 0, 0, d.np, ml, (int)blockIdx.x);
+                 status, sm_raw, shs, threadIdx.x, 0, 0, d.np);
     return;
   }
   select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-               status, sm_raw, sh, threadIdx.x, (int)blockDim.x, 0, ml, (int)blockIdx.x);
+               status, sm_raw, sh, threadIdx.x, (int)blockDim.x, 0);
 }
 
 }  // namespace ficoco

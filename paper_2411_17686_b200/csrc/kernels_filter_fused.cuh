@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     const int* __restrict__ pos, int window, float coef, int penalty, float* __restrict__ s_pen,
     float* __restrict__ scores_out, int* __restrict__ S_idx, int* __restrict__ T_idx,
     int* __restrict__ kept_idx, int* __restrict__ pos_out, unsigned* __restrict__ status,
-    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals, MergeLists ml) {
+    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals) {
   constexpr int E = VecTraits<T>::E;
   constexpr int F_P2B = VPL <= 4 ? 2 : 1;   // rows a warp scores together in pass 2 (and has in flight from L2)
   extern __shared__ __align__(128) unsigned char fs_raw[];
@@ -397,7 +397,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       if (failed) return;
       FICOCO_PHASE(0, 7);
       select_small(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-                   status, ring, sel_small_sh, tid, 1, w0.r0, hi, ml, w0.img);
+                   status, ring, sel_small_sh, tid, 1, w0.r0, hi);
       cta_sync(1, F_NCONS);
       if (tid == 0) {
         // the last pieces to leave reset the image's counters (everybody is past its polls by then)
@@ -409,7 +409,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       for (int k = 0; k < nwon; ++k) mine = mine || won[k] == w0.img;
       if (mine) {
         select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
-                     status, ring, sel_sh, tid, F_NCONS, 1, ml, w0.img);
+                     status, ring, sel_sh, tid, F_NCONS, 1);
         cta_sync(1, F_NCONS);
         if (tid == 0) { cnt[w0.img] = 0; cnt[B + w0.img] = 0; }
       }

@@ -5,14 +5,13 @@
 
 namespace ficoco {
 
+constexpr int MHUB = 4;        // source rows a lane has in flight for a hub row
 constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the per-row arrays)
 constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
-constexpr int MCOPY = 3;       // rows a warp copies in one batch (covers CTAs of up to 24 rows)
-constexpr int MLIST = 2048;    // entries of hub rows a CTA can order in shared memory
-constexpr int MHUBS = 256;     // hub rows a CTA can keep track of (each has more than REC_INLINE entries)
-constexpr int MMAP = 2048;      // preserved tokens per image up to which the image's hub rows are shared by its CTAs
+constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
+constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
+constexpr int MHEAVY = 2;      // rows with more sources than this are split into 32-vector blocks over the warps
 constexpr int MVB = 4;         // 16-byte vectors a lane accumulates at a time
-constexpr int MHUB = 8;        // source rows a lane has in flight on a hub row
 
 // acc[b][.] += sum over list entries [k0, k1) of alpha * x, for the MVB vectors v0 + 32 b of
 // each row; source rows are fetched four at a time so that 4 * MVB loads are in flight per lane.
@@ -48,175 +47,152 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
   }
 }
 
-// Compress + compact.  A CTA owns up to 32 consecutive output rows of one image (warp w: rows
-// w, w + 8, ...).
-//   1. every row resolves its input row (CLS / preserved token / trailing text row);
-//   2. one pass over the records of the image's preserved tokens (how many discarded tokens are
-//      merged into each and the first REC_INLINE of them): the short lists of the CTA's own rows
-//      are ordered in registers, and every row of the image with more entries (a "hub" row) is
-//      registered with its inline entries; the rest of a hub row's entries come from the image's
-//      overflow pool.  Every list is ordered by token index, so that the fp32 sums of Eq. 2 have
-//      one fixed order and no atomics touch floats;
-//   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once: rows
-//      without sources are copied in one batch, rows with up to REC_INLINE sources are merged by
-//      their own warp (both while the pool entries are in flight);
-//   4. hub rows hold most of the source traffic and sit in few CTAs, so they are shared: every
-//      (hub row, block of 32 vectors) item belongs to the CTA of the image that its number
-//      (position * blocks + block) modulo the image's CTAs names.  A warp takes an item, every
-//      lane summing the sources of its vector in list order, MHUB source rows in flight.  The
-//      lists are built redundantly by the image's CTAs, but nothing is exchanged between CTAs
-//      and nobody waits.
-// When an image has more preserved tokens, hub rows or hub entries than fit (MMAP / MHUBS /
-// MLIST), a CTA merges only the hub rows among its own rows, and if even those do not fit it
-// walks the image's entry arrays in order (slow, degenerate inputs only).
+// Compress + compact.  No per-target lists are built in global memory.  A CTA owns up to 32
+// consecutive output rows of one image (warp w: rows w, w + 8, w + 16, w + 24).
+//   1. every warp resolves the input row of its output rows (L1 prefetches of the rows were tried:
+//      they never produced L1 hits and cost 1.7 us per step, so there are none);
+//   2. meanwhile the CTA scans the image's (source -> target) entries twice (count, then fill)
+//      to file those that hit its rows into per-row lists in shared memory (token index,
+//      alpha), and orders every list by token index so that the
+//      fp32 sums have one fixed order and no atomics touch floats;
+//   3. out_j = (x_j + sum_{i in I_j} alpha_ij x_i) / (1 + sum alpha_ij), rounded once:
+//      rows with few sources by their own warp; hub rows are cut into blocks of 32 vectors that
+//      are dealt to the warps, every lane summing the sources of its vector in list order.
+// If the CTA's rows receive more than MLIST sources in total, a slow in-order rescan is used.
 template <class T>
-__global__ void __launch_bounds__(256, 3) k_merge_rec(
+__global__ void __launch_bounds__(256) k_merge_scan(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
-    const int* __restrict__ e_tgt, const float* __restrict__ e_w, const TgtRec* __restrict__ rec,
-    const int* __restrict__ pool_cnt, const PoolEnt* __restrict__ pool, T* __restrict__ out,
-    int index_before_wait, const unsigned* __restrict__ status, int rows_per_cta) {
+    const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out,
+    int index_before_wait, const unsigned* __restrict__ status) {
   constexpr int E = VecTraits<T>::E;
-  __shared__ int cnt[MROWS], srow_s[MROWS];
-  __shared__ int lsrc_l[MROWS][8];                  // own rows with up to REC_INLINE sources, ordered
-  __shared__ float lw_l[MROWS][8];
-  __shared__ int hsrc[MLIST], tsrc[MLIST];          // hub rows: ordered entries / as they arrived
-  __shared__ float hw[MLIST], tw[MLIST];
-  __shared__ short hmap[MMAP];                      // preserved token (minus scan_lo) -> hub slot, -1 = none
-  __shared__ int hub_t[MHUBS], hub_srow[MHUBS], hoff[MHUBS], hlen[MHUBS], hcur[MHUBS];
-  __shared__ float hub_inv[MHUBS];
-  __shared__ int n_hub_s, hub_total_s, overflow_s, dead;
+  __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
+  __shared__ int lsrc[MLIST];
+  __shared__ float lw[MLIST];
+  __shared__ int tsrc[MLIST];
+  __shared__ float tw[MLIST];
+  __shared__ int heavy_rows[MROWS];
+  __shared__ int n_heavy, dead;
   FICOCO_PHASE(2, 0);
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = D / E;
   const int L = d.list_len;
+  const int tp_lo = max(w.r0 - d.n_cls, 0);
+  const int tp_hi = min(w.r0 + w.nrows - d.n_cls, d.n_tgt);
+  const int n_ent = d.n_src * L;
   const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
-  const int tp_lo = max(w.r0 - d.n_cls, 0);                         // own preserved tokens: [tp_lo, tp_hi)
-  const int tp_hi = max(tp_lo, min(w.r0 + w.nrows - d.n_cls, d.n_tgt));
 
+  if (tid < MROWS) { cnt[tid] = 0; cur[tid] = 0; }
+  if (tid == 0) n_heavy = 0;
   // When the grid before this one is a correlate grid, the filter grid (which wrote T_idx) had
   // completed before this grid could start, so the row lookup may overlap that
   // grid's tail; otherwise wait first.
   if (!index_before_wait) grid_dep_wait();
-  int my_srow = 0;
-  if (tid < w.nrows) {
-    const int orow = w.r0 + tid;
-    if (orow < d.n_cls) my_srow = orow;
-    else if (orow < d.n_cls + d.n_tgt) my_srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
-    else my_srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
+  // input row of every output row (CLS / preserved token / trailing text row)
+  #pragma unroll 1
+  for (int r = warp; r < w.nrows; r += 8) {
+    const int orow = w.r0 + r;
+    int srow;
+    if (orow < d.n_cls) srow = orow;
+    else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
+    else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
+    if (lane == 0) srow_s[r] = srow;
   }
-  // The token rows do not stay in L2 from the kernels before (the step's working set is larger than
-  // what L2 keeps of it), and this grid is resident well before the correlate grid ends: ask L2
-  // for the rows this CTA will copy or merge into, and for its share of the image's discarded rows
-  // (every discarded row is merged somewhere), so that the reads below find them on chip.
-  if (tid < w.nrows) srow_s[tid] = my_srow;
-  __syncthreads();
-  {
-    const int lines = (D * (int)sizeof(T) + 127) / 128;          // 128-byte lines per row
-    #pragma unroll 1
-    for (int r = warp; r < w.nrows; r += 8) {
-      const char* row = reinterpret_cast<const char*>(tokens + (size_t)(d.row0 + srow_s[r]) * D);
-      for (int l = lane; l < lines; l += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + (size_t)l * 128));
-    }
-    if (index_before_wait && L > 0) {                            // S_idx is final: the filter grid has completed
-      const int nct0 = (d.n_cls + d.n_tgt + d.n_tail + rows_per_cta - 1) / rows_per_cta;
-      const int per = (d.n_src + nct0 - 1) / nct0;
-      const int s_end = min(d.n_src, (w.aux + 1) * per);
-      #pragma unroll 1
-      for (int sidx = w.aux * per + warp; sidx < s_end; sidx += 8) {
-        const char* row = reinterpret_cast<const char*>(pbase + (size_t)S_idx[d.src0 + sidx] * D);
-        for (int l = lane; l < lines; l += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + (size_t)l * 128));
-      }
-    }
-  }
-  if (tid < MROWS) cnt[tid] = 0;
-  if (tid == 0) { n_hub_s = 0; hub_total_s = 0; overflow_s = 0; }
-  bool shared_hubs = L > 0 && d.n_tgt <= MMAP;
-  int scan_lo = shared_hubs ? 0 : tp_lo, scan_hi = shared_hubs ? d.n_tgt : tp_hi;
-  for (int i = tid; i < scan_hi - scan_lo; i += 256) hmap[i] = -1;
   if (index_before_wait) grid_dep_wait();
   grid_dep_launch();   // correlate is complete: the next step's filter may stream its rows under our tail
   FICOCO_PHASE(2, 1);
   // a step whose filter or correlate grid gave up has no valid index lists: write nothing
   if (tid == 0) dead = (*reinterpret_cast<const volatile unsigned*>(status) & STATUS_TIMEOUT) ? 1 : 0;
-  const int np_ent = L > 0 ? __ldcg(pool_cnt + w.img) : 0;
   __syncthreads();
   if (dead) return;
-  // ---- one pass over the records: own rows' short lists, hub rows of the scanned range ----------
-  #pragma unroll 1
-  for (int pass = 0; pass < 2; ++pass) {
-    if (L > 0) {
-      #pragma unroll 1
-      for (int t0 = scan_lo + tid; t0 < scan_hi; t0 += 2 * 256) {      // two records in flight per thread
-        uint4 q[2][4];
+  // file the entries that hit this CTA's rows.  Up to 1024 entries per image every thread looks
+  // at no more than four, keeps its matches in registers and needs one pass; larger images
+  // take a counting pass and a filling pass.
+  const bool one_pass = n_ent <= 4 * 256;
+  int st_row[4], st_slot[4], st_src[4];
+  float st_w[4];
 #pragma unroll
-        for (int j = 0; j < 2; ++j)
+  for (int i = 0; i < 4; ++i) st_row[i] = -1;
+  if (tp_hi > tp_lo) {
+    if (one_pass) {
+      int t4[4];
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            q[j][k] = t0 + 256 * j < scan_hi
-                          ? __ldcg(reinterpret_cast<const uint4*>(rec + d.tgt0 + t0 + 256 * j) + k)
-                          : make_uint4(0, 0, 0, 0);
+      for (int i = 0; i < 4; ++i) {
+        // target, source and weight are fetched together: a source fetched only for the matches
+        // would add a second round trip to L2
+        const int e = tid + 256 * i;
+        const bool on = e < n_ent;
+        t4[i] = on ? e_tgt[d.ent0 + e] : -1;
+        st_src[i] = on ? S_idx[d.src0 + e / L] : 0;
+        st_w[i] = on ? e_w[d.ent0 + e] : 0.f;
+      }
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const int t = t0 + 256 * j;
-          if (t >= scan_hi) continue;
-          const int c = (int)q[j][0].x;
-          const int es[REC_INLINE] = {(int)q[j][0].z, (int)q[j][1].x, (int)q[j][1].z, (int)q[j][2].x,
-                                      (int)q[j][2].z, (int)q[j][3].x, (int)q[j][3].z};
-          const uint32_t ew[REC_INLINE] = {q[j][0].w, q[j][1].y, q[j][1].w, q[j][2].y, q[j][2].w, q[j][3].y, q[j][3].w};
-          const bool own = t >= tp_lo && t < tp_hi;
-          const int r = t + d.n_cls - w.r0;                              // own row index
-          if (own) cnt[r] = c;
-          if (c > REC_INLINE) {
-            const int slot = atomicAdd(&n_hub_s, 1);
-            const int off = atomicAdd(&hub_total_s, c);
-            if (slot < MHUBS && off + c <= MLIST) {
-              hub_t[slot] = t; hoff[slot] = off; hlen[slot] = c; hcur[slot] = off + REC_INLINE;
-              hmap[t - scan_lo] = (short)slot;
+      for (int i = 0; i < 4; ++i) {
+        const int t = t4[i];
+        if (t >= tp_lo && t < tp_hi) {
+          st_row[i] = t - tp_lo;
+          st_slot[i] = atomicAdd(&cnt[t - tp_lo], 1);
+        }
+      }
+    } else {
+      for (int e = tid; e < n_ent; e += 256) {
+        const int t = e_tgt[d.ent0 + e];
+        if (t >= tp_lo && t < tp_hi) atomicAdd(&cnt[t - tp_lo], 1);
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    // exclusive scan of the 32 counts
+    const int c = cnt[lane];
+    int inc = c;
 #pragma unroll
-              for (int k = 0; k < REC_INLINE; ++k) { tsrc[off + k] = es[k]; tw[off + k] = __uint_as_float(ew[k]); }
-            } else {
-              overflow_s = 1;
-            }
-          } else if (own) {
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+      if (lane >= o) inc += n;
+    }
+    beg[lane] = inc - c;
+    if (lane == 31) beg[MROWS] = inc;
+    if (c > MHEAVY) heavy_rows[atomicAdd(&n_heavy, 1)] = lane;
+  }
+  __syncthreads();
+  const int total = beg[MROWS];
+  const bool fits = total <= MLIST;
+  if (fits && total > 0) {
+    if (one_pass) {
 #pragma unroll
-            for (int k = 0; k < REC_INLINE; ++k) {
-              if (k < c) {
-                int rank = 0;
-#pragma unroll
-                for (int m = 0; m < REC_INLINE; ++m) rank += (m < c && es[m] < es[k]) ? 1 : 0;
-                lsrc_l[r][rank] = es[k];
-                lw_l[r][rank] = __uint_as_float(ew[k]);
-              }
-            }
-          }
+      for (int i = 0; i < 4; ++i)
+        if (st_row[i] >= 0) {
+          const int slot = beg[st_row[i]] + st_slot[i];
+          tsrc[slot] = st_src[i];
+          tw[slot] = st_w[i];
+        }
+    } else {
+      for (int e = tid; e < n_ent; e += 256) {
+        const int t = e_tgt[d.ent0 + e];
+        if (t >= tp_lo && t < tp_hi) {
+          const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
+          const int si = S_idx[d.src0 + e / L];
+          tsrc[slot] = si;
+          tw[slot] = e_w[d.ent0 + e];
         }
       }
     }
     __syncthreads();
-    if (!overflow_s || !shared_hubs) break;
-    // the image's hub rows do not fit: this CTA looks after the hub rows among its own rows only
-    __syncthreads();
-    shared_hubs = false;
-    scan_lo = tp_lo;
-    scan_hi = tp_hi;
-    if (tid == 0) { n_hub_s = 0; hub_total_s = 0; overflow_s = 0; }
-    for (int i = tid; i < tp_hi - tp_lo; i += 256) hmap[i] = -1;
-    __syncthreads();
+    // order every list by token index (rank of each entry inside its row)
+    for (int i = tid; i < total; i += 256) {
+      int r = 0;
+      while (i >= beg[r + 1]) ++r;
+      const int my = tsrc[i];
+      int rank = 0;
+      for (int k = beg[r]; k < beg[r + 1]; ++k) rank += tsrc[k] < my ? 1 : 0;
+      lsrc[beg[r] + rank] = my;
+      lw[beg[r] + rank] = tw[i];
+    }
   }
-  const bool fits = overflow_s == 0;
-  const int n_hub = fits ? n_hub_s : 0;
-  // the rest of the hub rows' entries (overflow pool) and their input rows: in flight during the copies
-  uint4 pe[2];
-#pragma unroll
-  for (int j = 0; j < 2; ++j)
-    pe[j] = (n_hub > 0 && tid + 256 * j < np_ent)
-                ? __ldcg(reinterpret_cast<const uint4*>(pool + (size_t)d.ent0 + tid + 256 * j))
-                : make_uint4(0xFFFFFFFFu, 0, 0, 0);
-  const int hub_in = tid < n_hub ? T_idx[d.tgt0 + hub_t[tid]] : 0;
-  FICOCO_PHASE(2, 2);
+  __syncthreads();
 
   // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
   #pragma unroll 1
@@ -225,7 +201,9 @@ __global__ void __launch_bounds__(256, 3) k_merge_rec(
 #pragma unroll
     for (int j = 0; j < MCOPY; ++j) {
       const int r = warp + 8 * j;
-      const bool copy = r < w.nrows && cnt[r] == 0;
+      const int orow = w.r0 + r;
+      const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
       const T* src = tokens + (size_t)(d.row0 + (r < w.nrows ? srow_s[r] : 0)) * D;
 #pragma unroll
       for (int b = 0; b < MVB; ++b) {
@@ -236,8 +214,10 @@ __global__ void __launch_bounds__(256, 3) k_merge_rec(
 #pragma unroll
     for (int j = 0; j < MCOPY; ++j) {
       const int r = warp + 8 * j;
-      const bool copy = r < w.nrows && cnt[r] == 0;
-      T* dst = out + (size_t)(d.out_row0 + w.r0 + r) * D;
+      const int orow = w.r0 + r;
+      const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
+      T* dst = out + (size_t)(d.out_row0 + orow) * D;
 #pragma unroll
       for (int b = 0; b < MVB; ++b) {
         const int v = v0 + 32 * b;
@@ -245,61 +225,49 @@ __global__ void __launch_bounds__(256, 3) k_merge_rec(
       }
     }
   }
-  #pragma unroll 1
-  for (int r = warp + 8 * MCOPY; r < w.nrows; r += 8) {      // rows past the batch (more than 16 rows per CTA)
-    if (cnt[r] != 0) continue;
-    const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
-    T* dst = out + (size_t)(d.out_row0 + w.r0 + r) * D;
-    for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(dst)[v] = ldg16(src + (size_t)v * E);
-  }
-  FICOCO_PHASE(2, 3);
 
   // ---- rows with a few sources: one warp per row --------------------------------------------------
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
-    const int n = cnt[r];
-    if (n == 0 || n > REC_INLINE) continue;
-    T* dst = out + (size_t)(d.out_row0 + w.r0 + r) * D;
+    const int orow = w.r0 + r;
+    T* dst = out + (size_t)(d.out_row0 + orow) * D;
+    const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
+    const int li = is_tgt ? orow - d.n_cls - tp_lo : 0;
+    const int n = is_tgt ? cnt[li] : 0;
     const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
-    float wsum = 0.f;
-    for (int k = 0; k < n; ++k) wsum += lw_l[r][k];
-    const float inv_den = 1.0f / (1.0f + wsum);   // one division per row, then multiplies
-    #pragma unroll 1
-    for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
-      float acc[MVB][E];
+    if (n == 0) {
+      continue;
+    } else if (fits && n <= MHEAVY) {
+      const int b0 = beg[li];
+      float wsum = 0.f;
+      for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
+      const float inv_den = 1.0f / (1.0f + wsum);   // one division per row, then multiplies
+      #pragma unroll 1
+      for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
+        float acc[MVB][E];
 #pragma unroll
-      for (int b = 0; b < MVB; ++b) {
-        const int v = v0 + 32 * b;
-        unpack(v < nvec ? ldg16(src + (size_t)v * E) : make_uint4(0, 0, 0, 0), acc[b], (const T*)nullptr);
-      }
-      merge_accumulate<T>(acc, pbase, D, lsrc_l[r], lw_l[r], 0, n, v0, nvec);
+        for (int b = 0; b < MVB; ++b) {
+          const int v = v0 + 32 * b;
+          unpack(v < nvec ? ldg16(src + (size_t)v * E) : make_uint4(0, 0, 0, 0), acc[b], (const T*)nullptr);
+        }
+        merge_accumulate<T>(acc, pbase, D, lsrc, lw, b0, b0 + n, v0, nvec);
 #pragma unroll
-      for (int b = 0; b < MVB; ++b) {
-        const int v = v0 + 32 * b;
-        if (v < nvec) {
+        for (int b = 0; b < MVB; ++b) {
+          const int v = v0 + 32 * b;
+          if (v < nvec) {
 #pragma unroll
-          for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] * inv_den;
-          reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
+            for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] * inv_den;
+            reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
+          }
         }
       }
-    }
-  }
-  FICOCO_PHASE(2, 4);
-
-  if (!fits) {
-    // too many entries for shared memory: every own hub row walks the image's entries in order
-    // (ascending token index)
-    const int n_ent = d.n_src * L;
-    #pragma unroll 1
-    for (int r = warp; r < w.nrows; r += 8) {
-      if (cnt[r] <= REC_INLINE) continue;
-      const int tp = w.r0 + r - d.n_cls;
-      const T* src = tokens + (size_t)(d.row0 + srow_s[r]) * D;
-      T* dst = out + (size_t)(d.out_row0 + w.r0 + r) * D;
+    } else if (!fits) {
+      // too many sources for shared memory: walk the entries in order (ascending source)
+      const int tp = orow - d.n_cls;
       float wsum = 0.f;
       for (int e = 0; e < n_ent; ++e)
         if (e_tgt[d.ent0 + e] == tp) wsum += e_w[d.ent0 + e];
-      const float inv_den = 1.0f / (1.0f + wsum);
+      const float den = 1.0f + wsum;
       for (int v = lane; v < nvec; v += 32) {
         float acc[E];
         unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
@@ -313,109 +281,53 @@ __global__ void __launch_bounds__(256, 3) k_merge_rec(
           for (int q = 0; q < E; ++q) acc[q] = fmaf(a0, f[q], acc[q]);
         }
 #pragma unroll
-        for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
+        for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
         reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
       }
     }
-    FICOCO_PHASE(2, 5);
-    return;
   }
-  if (n_hub == 0) { FICOCO_PHASE(2, 5); return; }
+  if (!fits) return;
 
-  // ---- hub rows: finish the lists (pool entries), order them, weights ---------------------------
-  {
-    const int span = scan_hi - scan_lo;
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int t = (int)pe[j].x - scan_lo;
-      if (tid + 256 * j < np_ent && t >= 0 && t < span && hmap[t] >= 0) {
-        const int slot = atomicAdd(&hcur[hmap[t]], 1);
-        tsrc[slot] = (int)pe[j].y;
-        tw[slot] = __uint_as_float(pe[j].z);
-      }
-    }
-    #pragma unroll 1
-    for (int e = tid + 512; e < np_ent; e += 256) {
-      const uint4 u = __ldcg(reinterpret_cast<const uint4*>(pool + (size_t)d.ent0 + e));
-      const int t = (int)u.x - scan_lo;
-      if (t >= 0 && t < span && hmap[t] >= 0) {
-        const int slot = atomicAdd(&hcur[hmap[t]], 1);
-        tsrc[slot] = (int)u.y;
-        tw[slot] = __uint_as_float(u.z);
-      }
-    }
-    if (tid < n_hub) hub_srow[tid] = d.n_cls + hub_in;
-  }
-  __syncthreads();
-  #pragma unroll 1
-  for (int h = warp; h < n_hub; h += 8) {
-    const int off = hoff[h], n = hlen[h];
-    for (int k = lane; k < n; k += 32) {
-      const int my = tsrc[off + k];
-      int rank = 0;
-      for (int m = 0; m < n; ++m) rank += tsrc[off + m] < my ? 1 : 0;
-      hsrc[off + rank] = my;
-      hw[off + rank] = tw[off + k];
-    }
-    __syncwarp();
-    // 1 / (1 + sum alpha), the sum in a fixed order: lane l adds entries l, l + 32, ...; then a shuffle tree
-    float wsum = 0.f;
-    for (int k = lane; k < n; k += 32) wsum += hw[off + k];
-    wsum = warp_sum(wsum);
-    if (lane == 0) hub_inv[h] = 1.0f / (1.0f + wsum);
-  }
-  __syncthreads();
-
-  // ---- this CTA's share of the (hub row, block of 32 vectors) items ------------------------------
+  // ---- hub rows: (row, block of 32 vectors) items dealt to the warps; each lane sums all the
+  // sources of its one vector in list order, MHUB source rows in flight ---------------------
+  const int nh = n_heavy;
   const int nblk = (nvec + 31) / 32;
-  int nct = 1, me = 0;                              // CTAs of the image that share its hub rows, this one's index
-  if (shared_hubs) {
-    nct = (d.n_cls + d.n_tgt + d.n_tail + rows_per_cta - 1) / rows_per_cta;
-    me = w.aux;
-  }
   #pragma unroll 1
-  for (int h = warp; h < n_hub; h += 8) {
-    const int b0 = hoff[h], n = hlen[h];
-    // blocks with (position * nblk + block) % nct == me
-    int blk0 = (me - (int)(((long long)hub_t[h] * nblk) % nct)) % nct;
-    if (blk0 < 0) blk0 += nct;
+  for (int it = warp; it < nh * nblk; it += 8) {
+    const int li = heavy_rows[it / nblk];
+    const int v = (it % nblk) * 32 + lane;
+    if (v >= nvec) continue;
+    const int tp = tp_lo + li;
+    const int b0 = beg[li], n = cnt[li];
+    const T* src = tokens + (size_t)(d.row0 + srow_s[tp + d.n_cls - w.r0]) * D;
+    T* dst = out + (size_t)(d.out_row0 + d.n_cls + tp) * D;
+    float wsum = 0.f;
+    for (int k = 0; k < n; ++k) wsum += lw[b0 + k];
+    const float inv_den = 1.0f / (1.0f + wsum);
+    float acc[E];
+    unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
     #pragma unroll 1
-    for (int blk = blk0; blk < nblk; blk += nct) {
-      const int v = blk * 32 + lane;
-      if (v >= nvec) continue;
-      // the target row's vector travels with the first sources
-      const uint4 xt = ldg16(tokens + (size_t)(d.row0 + hub_srow[h]) * D + (size_t)v * E);
-      float acc[E];
+    for (int k = 0; k < n; k += MHUB) {
+      uint4 u[MHUB];
+      float a[MHUB];
 #pragma unroll
-      for (int q = 0; q < E; ++q) acc[q] = 0.f;
-      #pragma unroll 1
-      for (int k0 = 0; k0 < n; k0 += MHUB) {
-        uint4 u[MHUB];
-        float a[MHUB];
-#pragma unroll
-        for (int j = 0; j < MHUB; ++j) {
-          const bool on = k0 + j < n;
-          a[j] = on ? hw[b0 + k0 + j] : 0.f;
-          u[j] = on ? ldg16(pbase + (size_t)hsrc[b0 + k0 + j] * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int j = 0; j < MHUB; ++j) {
-          float f[E];
-          unpack(u[j], f, (const T*)nullptr);
-#pragma unroll
-          for (int q = 0; q < E; ++q) acc[q] = fmaf(a[j], f[q], acc[q]);
-        }
+      for (int j = 0; j < MHUB; ++j) {
+        const bool on = k + j < n;
+        a[j] = on ? lw[b0 + k + j] : 0.f;
+        u[j] = on ? ldg16(pbase + (size_t)lsrc[b0 + k + j] * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
       }
-      T* dst = out + (size_t)(d.out_row0 + d.n_cls + hub_t[h]) * D;
-      float x[E];
-      unpack(xt, x, (const T*)nullptr);
-      const float inv_den = hub_inv[h];
 #pragma unroll
-      for (int q = 0; q < E; ++q) acc[q] = (x[q] + acc[q]) * inv_den;
-      reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
+      for (int j = 0; j < MHUB; ++j) {
+        float f[E];
+        unpack(u[j], f, (const T*)nullptr);
+#pragma unroll
+        for (int q = 0; q < E; ++q) acc[q] = fmaf(a[j], f[q], acc[q]);
+      }
     }
+#pragma unroll
+    for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
+    reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
   }
-  FICOCO_PHASE(2, 5);
 }
 
 }  // namespace ficoco

@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ tile_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c, MergeLists ml) {
+    float* __restrict__ e_w, float* __restrict__ e_c) {
   extern __shared__ int tcol[];              // token index of every column of the split
   __shared__ int is_last;
   const WorkItem w = work[blockIdx.x];
@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
     }
   }
   correlate_tail<LC>(d, w, (int)blockIdx.x - w.aux, tile_done, part_val, part_idx, corr_cnt, tau_out,
-                     e_tgt, e_w, e_c, &is_last, S_idx, ml);
+                     e_tgt, e_w, e_c, &is_last);
 }
 
 }  // namespace ficoco
