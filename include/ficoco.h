@@ -78,6 +78,14 @@ enum ficoco_flags {
                                     the features are averaged directly): every alpha_ij of Eq. 2
                                     is 1, so a preserved token becomes the plain mean of itself
                                     and the discarded tokens sent to it; J_i is unchanged */
+  FICOCO_CONVERGENT = 16u,       /* ablation "convergent correlation" (Sec. "Correlation-based Information
+                                    Recycling" and the ablation tables: all discarded tokens merge into one
+                                    additional token).  The paper gives no weights: the additional token is
+                                    the plain mean of the image's discarded tokens.  Preserved tokens stay as
+                                    they are; an image that discards at least one token gets one more output
+                                    row right after its preserved vision rows (before the text rows of
+                                    FiCoCo-L), with kept_idx -1; out_tokens and kept_idx must have room for
+                                    it.  max_targets and eps are ignored. */
   FICOCO_BACK_TO_BACK = 8u       /* scheduling hint, no effect on results: the caller states that the
                                     work enqueued on the stream right before this call is the
                                     previous reduce step of this library (any context) and nothing

@@ -17,7 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libficoco.so")
 
 FICOCO_FP32, FICOCO_BF16 = 0, 1
-FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY, FICOCO_AVERAGE_COMPRESSION, FICOCO_BACK_TO_BACK = 1, 2, 4, 8
+FICOCO_HAS_CLS, FICOCO_LOCAL_PENALTY, FICOCO_AVERAGE_COMPRESSION, FICOCO_BACK_TO_BACK, FICOCO_CONVERGENT = 1, 2, 4, 8, 16
 KCAP = 16
 
 INSPECT = {
@@ -113,13 +113,13 @@ def ficoco_default_params() -> ficoco_params:
 
 def make_params(lam=0.35, beta=0.6, gamma=0.6, eps=0.998, penalty_coef=2.0, window=2,
                 max_targets=-1, has_cls=True, local_penalty=True, average_compression=False,
-                back_to_back=False) -> ficoco_params:
+                back_to_back=False, convergent=False) -> ficoco_params:
     p = ficoco_params()
     p.lambda_, p.beta, p.gamma, p.eps, p.penalty_coef = lam, beta, gamma, eps, penalty_coef
     p.window, p.max_targets = window, -1 if max_targets is None else max_targets
     p.flags = ((FICOCO_HAS_CLS if has_cls else 0) | (FICOCO_LOCAL_PENALTY if local_penalty else 0) |
                (FICOCO_AVERAGE_COMPRESSION if average_compression else 0) |
-               (FICOCO_BACK_TO_BACK if back_to_back else 0))
+               (FICOCO_BACK_TO_BACK if back_to_back else 0) | (FICOCO_CONVERGENT if convergent else 0))
     return p
 
 
@@ -204,7 +204,9 @@ class Context:
             sl = None
             batch = tokens.shape[0] // n_tokens if n_tokens else 0
         keeps = [int(keep_a[0 if n_keep == 1 else b]) for b in range(batch)]
-        out_rows = [cls + k for k in keeps]
+        ntoks = [int(sl[b]) if sl is not None else n_tokens for b in range(batch)]
+        conv = bool(p.flags & FICOCO_CONVERGENT)        # one more row per image that discards something
+        out_rows = [cls + k + (1 if conv and n - cls - k > 0 else 0) for k, n in zip(keeps, ntoks)]
         dim = tokens.shape[-1]
         dev = tokens.device
         if out_tokens is None:
@@ -241,7 +243,8 @@ class Context:
         keep_a, n_keep = _int_array(keep)
         batch = tokens.shape[0] // (n_vision + n_text)
         keeps = [int(keep_a[0 if n_keep == 1 else b]) for b in range(batch)]
-        out_rows = [k + n_text for k in keeps]
+        conv = bool(p.flags & FICOCO_CONVERGENT)
+        out_rows = [k + n_text + (1 if conv and n_vision - k > 0 else 0) for k in keeps]
         dim = tokens.shape[-1]
         dev = tokens.device
         if out_tokens is None:
@@ -275,7 +278,9 @@ class Context:
         else:
             sl, batch = None, tokens.shape[0] // n_tokens
         keeps = [int(keep_a[0 if n_keep == 1 else b]) for b in range(batch)]
-        out_rows = [cls + k for k in keeps]
+        ntoks = [int(sl[b]) if sl is not None else n_tokens for b in range(batch)]
+        conv = bool(p.flags & FICOCO_CONVERGENT)
+        out_rows = [cls + k + (1 if conv and n - cls - k > 0 else 0) for k, n in zip(keeps, ntoks)]
         dim = tokens.shape[-1]
         if out_tokens is None:
             out_tokens = torch.empty((sum(out_rows), dim), dtype=tokens.dtype).pin_memory()
@@ -300,7 +305,8 @@ class Context:
         keep_a, n_keep = _int_array(keep)
         batch = tokens.shape[0] // (n_vision + n_text)
         keeps = [int(keep_a[0 if n_keep == 1 else b]) for b in range(batch)]
-        out_rows = [k + n_text for k in keeps]
+        conv = bool(p.flags & FICOCO_CONVERGENT)
+        out_rows = [k + n_text + (1 if conv and n_vision - k > 0 else 0) for k in keeps]
         dim = tokens.shape[-1]
         if out_tokens is None:
             out_tokens = torch.empty((sum(out_rows), dim), dtype=tokens.dtype).pin_memory()

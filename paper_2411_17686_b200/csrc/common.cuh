@@ -20,6 +20,7 @@ struct ImgDesc {
   int n_src;       // N^S, discarded
   int n_tgt;       // N^T, preserved
   int n_tail;      // trailing pass-through rows (text)
+  int n_extra;     // 1: one additional output row after the preserved tokens ("convergent correlation" ablation)
   int gh, gw;      // original patch grid
   int patch0;      // offset in per-vision-token arrays
   int out_row0;    // first output row (also offset in kept_idx)

@@ -37,11 +37,12 @@ struct PlanKey {
   int mode;  // 0 = V, 1 = L
   int dtype, batch, dim, n_text, has_cls, max_targets, avg;
   int rel = 0;  // 0: cosine relation of the tokens; 1 / 2: caller-supplied relation, by row / by column
+  int conv = 0; // 1: "convergent correlation" ablation (one additional token per image, no merging)
   double eps;
   std::vector<int> ntok, keep, gh, gw;
   bool operator==(const PlanKey& o) const {
     return mode == o.mode && dtype == o.dtype && batch == o.batch && dim == o.dim &&
-           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets && avg == o.avg && rel == o.rel &&
+           n_text == o.n_text && has_cls == o.has_cls && max_targets == o.max_targets && avg == o.avg && rel == o.rel && conv == o.conv &&
            eps == o.eps && ntok == o.ntok && keep == o.keep && gh == o.gh && gw == o.gw;
   }
 };
@@ -506,6 +507,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     const int keep = key.keep[b];
     if (keep < 0 || keep > np) return FICOCO_ERR_KEEP_RANGE;
     d.n_cls = cls; d.np = np; d.n_tgt = keep; d.n_src = np - keep; d.n_tail = tail;
+    d.n_extra = (key.conv && np - keep > 0) ? 1 : 0;
     d.gh = key.gh[b]; d.gw = key.gw[b];
     if (key.mode == 0) {
       if (d.gh < 1 || d.gw < 1) return FICOCO_ERR_INVALID_ARG;
@@ -610,7 +612,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   {
     auto n_out_ctas = [&](int r) {
       long long n = 0;
-      for (int b = 0; b < B; ++b) n += (cls + key.keep[b] + tail + r - 1) / r;
+      for (int b = 0; b < B; ++b) n += (cls + key.keep[b] + p->h_desc[b].n_extra + tail + r - 1) / r;
       return n;
     };
     while (out_rows_cta > 2 && n_out_ctas(out_rows_cta) < 2LL * c->num_sms &&
@@ -669,7 +671,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       ent0 += (long long)d.n_src * d.list_len;
     }
     // output rows
-    const int orows = d.n_cls + d.n_tgt + d.n_tail;
+    const int orows = d.n_cls + d.n_tgt + d.n_extra + d.n_tail;
     for (int r0 = 0; r0 < orows; r0 += out_rows_cta) {
       WorkItem w; w.img = b; w.r0 = r0; w.nrows = (orows - r0 < out_rows_cta) ? orows - r0 : out_rows_cta;
       w.aux = r0 / out_rows_cta;
@@ -1001,6 +1003,11 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
                    (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
                    (const unsigned*)c->status);
   c->launches += 1;
+  if (p->key.conv) {
+    prof_tick(c, st, "convergent_token");
+    k_convergent_token<T><<<p->key.batch, 256, 0, st>>>(tok, D, p->d_desc, c->S_idx, out_tokens, c->status);
+    c->launches += 1;
+  }
   prof_tick(c, st, nullptr);
   if (c->prof_used > 60000) prof_flush(c);
   cudaError_t e = cudaGetLastError();
@@ -1041,6 +1048,8 @@ int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* pr
   key.has_cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
   key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
   key.avg = (prm->flags & FICOCO_AVERAGE_COMPRESSION) ? 1 : 0;
+  key.conv = (prm->flags & FICOCO_CONVERGENT) ? 1 : 0;
+  if (key.conv) key.max_targets = 0;               // nothing is merged into the preserved tokens
   key.rel = rel_mode;
   key.eps = prm->eps;
   key.ntok.resize(a->batch); key.keep.resize(a->batch); key.gh.resize(a->batch); key.gw.resize(a->batch);
@@ -1096,6 +1105,8 @@ extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const fico
   key.has_cls = 0;
   key.max_targets = prm->max_targets < 0 ? -1 : prm->max_targets;
   key.avg = (prm->flags & FICOCO_AVERAGE_COMPRESSION) ? 1 : 0;
+  key.conv = (prm->flags & FICOCO_CONVERGENT) ? 1 : 0;
+  if (key.conv) key.max_targets = 0;
   key.eps = prm->eps;
   key.ntok.assign(a->batch, a->n_vision + a->n_text);
   key.keep.resize(a->batch);
@@ -1222,7 +1233,7 @@ extern "C" int ficoco_v_reduce_host(ficoco_ctx* c, const ficoco_v_args* h, const
     if (n < cls + 1 || k < 0 || k > n - cls) return FICOCO_ERR_KEEP_RANGE;
     p_rows[b + 1] = p_rows[b] + n;
     p_patch[b + 1] = p_patch[b] + n - cls;
-    p_orow[b + 1] = p_orow[b] + cls + k;
+    p_orow[b + 1] = p_orow[b] + cls + k + (((prm->flags & FICOCO_CONVERGENT) && n - cls - k > 0) ? 1 : 0);
     p_kept[b + 1] = p_kept[b] + k;
   }
   const long long rows = p_rows[B], patches = p_patch[B], orows = p_orow[B], kept = p_kept[B];
@@ -1339,7 +1350,7 @@ extern "C" int ficoco_l_reduce_host(ficoco_ctx* c, const ficoco_l_args* h, const
   for (int b = 0; b < h->batch; ++b) {
     const int k = h->keep[h->n_keep == 1 ? 0 : b];
     if (k < 0 || k > h->n_vision) return FICOCO_ERR_KEEP_RANGE;
-    orows += k + h->n_text;
+    orows += k + h->n_text + (((prm->flags & FICOCO_CONVERGENT) && h->n_vision - k > 0) ? 1 : 0);
   }
   const long long rows = (long long)h->batch * (h->n_vision + h->n_text);
   if (rows > c->max_tokens) return FICOCO_ERR_WORKSPACE;

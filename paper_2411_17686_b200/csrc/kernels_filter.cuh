@@ -424,7 +424,8 @@ __device__ __noinline__ void select_image(
   for (int i = tid; i < d.n_cls; i += nthr) kept_idx[d.out_row0 + i] = i;
   #pragma unroll 1
   for (int i = tid; i < d.n_tail; i += nthr)
-    kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
+    kept_idx[d.out_row0 + d.n_cls + d.n_tgt + d.n_extra + i] = d.n_cls + np + i;
+  if (tid == 0 && d.n_extra) kept_idx[d.out_row0 + d.n_cls + d.n_tgt] = -1;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -691,7 +692,8 @@ __device__ __noinline__ void select_small(
     for (int i = tid; i < d.n_cls; i += NT) kept_idx[d.out_row0 + i] = i;
     #pragma unroll 1
     for (int i = tid; i < d.n_tail; i += NT)
-      kept_idx[d.out_row0 + d.n_cls + d.n_tgt + i] = d.n_cls + np + i;
+      kept_idx[d.out_row0 + d.n_cls + d.n_tgt + d.n_extra + i] = d.n_cls + np + i;
+    if (tid == 0 && d.n_extra) kept_idx[d.out_row0 + d.n_cls + d.n_tgt] = -1;
   }
 }
 

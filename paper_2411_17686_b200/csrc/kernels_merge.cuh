@@ -97,7 +97,8 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     int srow;
     if (orow < d.n_cls) srow = orow;
     else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
-    else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt);
+    else if (orow < d.n_cls + d.n_tgt + d.n_extra) srow = -1;     // the additional token: written by k_convergent_token
+    else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt - d.n_extra);
     if (lane == 0) srow_s[r] = srow;
   }
   if (index_before_wait) grid_dep_wait();
@@ -203,8 +204,8 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       const int r = warp + 8 * j;
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
-      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
-      const T* src = tokens + (size_t)(d.row0 + (r < w.nrows ? srow_s[r] : 0)) * D;
+      const bool copy = r < w.nrows && srow_s[r < w.nrows ? r : 0] >= 0 && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
+      const T* src = tokens + (size_t)(d.row0 + (copy ? srow_s[r] : 0)) * D;
 #pragma unroll
       for (int b = 0; b < MVB; ++b) {
         const int v = v0 + 32 * b;
@@ -216,7 +217,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
       const int r = warp + 8 * j;
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
-      const bool copy = r < w.nrows && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
+      const bool copy = r < w.nrows && srow_s[r < w.nrows ? r : 0] >= 0 && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
       T* dst = out + (size_t)(d.out_row0 + orow) * D;
 #pragma unroll
       for (int b = 0; b < MVB; ++b) {
@@ -327,6 +328,68 @@ __global__ void __launch_bounds__(256) k_merge_scan(
 #pragma unroll
     for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
     reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
+  }
+}
+
+// Ablation "convergent correlation" (Sec. "Correlation-based Information Recycling": all discarded
+// tokens merge into one additional token): the plain mean of an image's discarded rows, written
+// behind the image's preserved rows.  One CTA per image; warp w sums the discarded rows w, w + 8,
+// ... in ascending order, the eight partial sums are added in warp order (fp32, fixed order),
+// scaled by 1 / N^S and rounded once.  Columns are processed in slabs of 128 vectors.
+template <class T>
+__global__ void __launch_bounds__(256) k_convergent_token(
+    const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc, const int* __restrict__ S_idx,
+    T* __restrict__ out, const unsigned* __restrict__ status) {
+  constexpr int E = VecTraits<T>::E;
+  __shared__ float part[8][128 * E];
+  const ImgDesc d = desc[blockIdx.x];
+  if (!d.n_extra || (*status & STATUS_TIMEOUT)) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = D / E;
+  const T* pbase = tokens + (size_t)(d.row0 + d.n_cls) * D;
+  T* dst = out + (size_t)(d.out_row0 + d.n_cls + d.n_tgt) * D;
+  const float inv = 1.0f / (float)d.n_src;
+  #pragma unroll 1
+  for (int c0 = 0; c0 < nvec; c0 += 128) {
+    float acc[4][E];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int q = 0; q < E; ++q) acc[k][q] = 0.f;
+    #pragma unroll 1
+    for (int s = warp; s < d.n_src; s += 8) {
+      const T* row = pbase + (size_t)S_idx[d.src0 + s] * D;
+      uint4 u[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int v = c0 + lane + 32 * k;
+        u[k] = v < nvec ? ldg16(row + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float f[E];
+        unpack(u[k], f, (const T*)nullptr);
+#pragma unroll
+        for (int q = 0; q < E; ++q) acc[k][q] += f[q];
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int q = 0; q < E; ++q) part[warp][(lane + 32 * k) * E + q] = acc[k][q];
+    __syncthreads();
+    if (tid < 128 && c0 + tid < nvec) {
+      float o[E];
+#pragma unroll
+      for (int q = 0; q < E; ++q) {
+        float t = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < 8; ++wv) t += part[wv][tid * E + q];
+        o[q] = t * inv;
+      }
+      reinterpret_cast<uint4*>(dst)[c0 + tid] = pack(o, (const T*)nullptr);
+    }
+    __syncthreads();
   }
 }
 

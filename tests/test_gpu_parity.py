@@ -293,6 +293,31 @@ def test_canaries_around_outputs(ctx):
     assert bool((kidx[pad:pad + rows] >= 0).all())
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_convergent_correlation_variant(ctx, dtype):
+    """Ablation 'convergent correlation': preserved rows bit for bit, one additional row per image
+    (the mean of the discarded rows) with kept index -1, against the checker; uniform and ragged
+    batches, nothing appended where nothing is discarded, and the FiCoCo-L layout."""
+    p = fo.Params(convergent=True)
+    batch = synth.make_v_batch(98, 3, 13, 11, 192, 5, 80, dtype, True, 1.2)
+    gaps.repair_v(batch, p)
+    res, results = parity.run_and_compare_v(ctx, batch, p, DEV, what="convergent")
+    assert res.out_rows == [1 + 80 + 1] * 3
+    kidx = binding.to_numpy(res.kept_idx).reshape(3, -1)
+    assert (kidx[:, -1] == -1).all() and (kidx[:, :-1] >= 0).all()
+    ragged = synth.workload(4, small=True)
+    ragged.keep[0] = ragged.tokens[0].shape[0]          # this image discards nothing: no additional row
+    gaps.repair_v(ragged, p)
+    res, results = parity.run_and_compare_v(ctx, ragged, p, DEV, what="convergent-ragged")
+    assert res.out_rows[0] == ragged.keep[0] and res.out_rows[1] == ragged.keep[1] + 1
+    if dtype == "bf16":
+        lb = synth.make_l_batch(99, 2, 100, 9, 256, 3, 30, "bf16", scale=1.0 / 16)
+        gaps.repair_l(lb, p)
+        res, results = parity.run_and_compare_l(ctx, lb, p, DEV, what="convergent-l")
+        kidx = binding.to_numpy(res.kept_idx).reshape(2, -1)
+        assert (kidx[:, 30] == -1).all() and kidx[0, 31:].tolist() == list(range(100, 109))
+
+
 def test_hand_built_ties_follow_the_lower_index(ctx):
     """The two hand-built tie inputs of tests/golden (bit-identical scores across the selection
     boundary, and inside one local-penalty window), with no margin repair: the library takes the
