@@ -77,6 +77,10 @@ __device__ __forceinline__ uint4 pack(const float (&f)[8], const __nv_bfloat16*)
 }
 
 __device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// Streaming store (st.global.cs) for the output rows.  A step's token rows, read by all three of
+// its kernels, plus its output rows are about as much as L2 keeps; written as ordinary stores the
+// output pushes the token rows out before the next kernel reads them again.
+__device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) { __stcs(p, v); }
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

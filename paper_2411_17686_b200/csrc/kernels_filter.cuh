@@ -1,5 +1,6 @@
 // Filter stage (Eq. 1, local penalty, top-N^S selection).
 #pragma once
+#include "async_ops.cuh"
 #include "common.cuh"
 
 namespace ficoco {
@@ -516,6 +517,7 @@ __device__ __noinline__ void select_small(
     }
   }
   cta_sync(bar, NT);
+  FICOCO_PHASE(0, 9);
 
   // ---- local penalty: one thread per window ------------------------------------------------
   if (penalty) {
@@ -540,6 +542,7 @@ __device__ __noinline__ void select_small(
     cta_sync(bar, NT);
   }
 
+  FICOCO_PHASE(0, 10);
   // ---- keys, their range, dense keys -----------------------------------------------------------
   uint32_t key[2];
   uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
@@ -578,6 +581,7 @@ __device__ __noinline__ void select_small(
     if (on[q]) wk.nk[tid + NT * q] = nk[q];
   }
 
+  FICOCO_PHASE(0, 11);
   // ---- radix select on the dense keys: the n_src-th largest -------------------------------------
   uint32_t thr = 0;      // threshold (dense key)
   int need_eq = 0;       // how many of the keys equal to thr are selected (lowest indices)
@@ -637,6 +641,7 @@ __device__ __noinline__ void select_small(
     need_eq = remaining;
   }
 
+  FICOCO_PHASE(0, 12);
   // ---- membership ---------------------------------------------------------------------------------
   bool sel[2];
 #pragma unroll
@@ -687,6 +692,7 @@ __device__ __noinline__ void select_small(
       }
     }
   }
+  FICOCO_PHASE(0, 13);
   if (w_lo == 0) {
     #pragma unroll 1
     for (int i = tid; i < d.n_cls; i += NT) kept_idx[d.out_row0 + i] = i;

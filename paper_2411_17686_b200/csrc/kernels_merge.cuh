@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
 #pragma unroll
       for (int b = 0; b < MVB; ++b) {
         const int v = v0 + 32 * b;
-        if (copy && v < nvec) reinterpret_cast<uint4*>(dst)[v] = u[j][b];
+        if (copy && v < nvec) st_stream16(reinterpret_cast<uint4*>(dst) + v, u[j][b]);
       }
     }
   }
@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
           if (v < nvec) {
 #pragma unroll
             for (int q = 0; q < E; ++q) acc[b][q] = acc[b][q] * inv_den;
-            reinterpret_cast<uint4*>(dst)[v] = pack(acc[b], (const T*)nullptr);
+            st_stream16(reinterpret_cast<uint4*>(dst) + v, pack(acc[b], (const T*)nullptr));
           }
         }
       }
@@ -283,7 +283,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
         }
 #pragma unroll
         for (int q = 0; q < E; ++q) acc[q] = acc[q] / den;
-        reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
+        st_stream16(reinterpret_cast<uint4*>(dst) + v, pack(acc, (const T*)nullptr));
       }
     }
   }
@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     }
 #pragma unroll
     for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
-    reinterpret_cast<uint4*>(dst)[v] = pack(acc, (const T*)nullptr);
+    st_stream16(reinterpret_cast<uint4*>(dst) + v, pack(acc, (const T*)nullptr));
   }
 }
 
