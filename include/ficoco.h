@@ -190,6 +190,31 @@ int ficoco_v_reduce_relation(ficoco_ctx* ctx, const ficoco_v_args* args, const f
                              int by_column, const ficoco_params* params, void* cuda_stream);
 
 /*
+ * A progressive FiCoCo-V schedule in one call: the reduce step applied n_steps times, every step
+ * on the output of the one before (the paper reduces at successive encoder layers, Sec.
+ * "Implementation Details"; between two steps the host model would run its layers, so this entry
+ * point is the reduction part of such a schedule on its own, as the multi-step workloads use it).
+ *   first     : the arguments of step 0 (tokens, pos, grid, dtype, batch, n_tokens, dim, heads) and
+ *               the buffers of the LAST step's results: out_tokens [B, c + keep[n_steps-1], dim],
+ *               kept_idx (row indices into the ORIGINAL input of step 0, the chain of the steps
+ *               composed), pos_out [B, keep[n_steps-1]].  first->attn, first->keep and
+ *               first->scores_out are ignored; batches must be uniform (seqlens NULL).
+ *   n_steps   : 1 .. 8.
+ *   keep      : host int32[n_steps], patch tokens preserved by each step (the same for every
+ *               image), non-increasing.
+ *   attn      : host array of n_steps device pointers; attn[s] holds step s's CLS->patch weights
+ *               [B, H, Np_s] over the patch tokens alive at that step (Np_0 = n_tokens - c,
+ *               Np_s = keep[s-1]).
+ * Intermediate tokens, kept indices and positions live in the context; they are allocated (and
+ * grown) by the first call that needs them, which synchronises and must therefore happen outside
+ * stream capture; later calls of the same or a smaller size allocate nothing.  Every step but the
+ * first is launched while the step before is still finishing and reads its input only once that
+ * step is complete.  Errors and the status word are those of ficoco_v_reduce.
+ */
+int ficoco_v_reduce_schedule(ficoco_ctx* ctx, const ficoco_v_args* first, int n_steps, const int* keep,
+                             const float* const* attn, const ficoco_params* params, void* cuda_stream);
+
+/*
  * FiCoCo-L reduce step (Algorithm 2) for a batch of decoder sequences of equal shape.
  * Each sequence has n_vision vision rows followed by n_text text rows.  Vision rows are
  * reduced to `keep`; text rows pass through unchanged after them.
@@ -319,7 +344,8 @@ int ficoco_equivalent_token(const void* keys, int dtype, int batch, int n_tokens
  *     every word a call reads it has written itself first, so nothing needs clearing, but two
  *     calls that overlap on the GPU (different streams, no ordering) race on it;
  *   - the first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *     outside any stream capture (a first call under capture returns FICOCO_ERR_CAPTURE and
+ *     launches nothing).
  * The device that owns `tokens`, `v_out` and `cuda_stream` must be the calling thread's
  * current device.  tokens: device, [batch, n_tokens, dim] (n_tokens includes the CLS row when
  * flags has FICOCO_HAS_CLS), 16-byte aligned rows; v_out: device fp32 [batch, Np].  Work is

@@ -32,7 +32,7 @@ EXPORTS = [
     "ficoco_default_params", "ficoco_v_reduce", "ficoco_l_reduce", "ficoco_v_reduce_host",
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
     "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
-    "ficoco_equivalent_token", "ficoco_v_reduce_relation", "ficoco_debug_waits",
+    "ficoco_equivalent_token", "ficoco_v_reduce_relation", "ficoco_debug_waits", "ficoco_v_reduce_schedule",
 ]
 
 
@@ -94,6 +94,8 @@ def load_library() -> C.CDLL:
     lib.ficoco_l_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params)]
     lib.ficoco_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
     lib.ficoco_debug_waits.argtypes = [C.c_void_p, C.c_longlong, C.c_int]
+    lib.ficoco_v_reduce_schedule.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.c_int, C.c_void_p, C.c_void_p,
+                                             C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_inspect.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
     lib.ficoco_last_launch_count.argtypes = [C.c_void_p]
     lib.ficoco_profile.argtypes = [C.c_void_p, C.c_int]
@@ -233,6 +235,40 @@ class Context:
         else:
             _check(self.h, self.lib.ficoco_v_reduce(self.h, C.byref(a), C.byref(p), C.c_void_p(stream)))
         return VResult(out_tokens, kept_idx, pos_out, scores_out, out_rows)
+
+    def ficoco_v_reduce_schedule(self, tokens, attns, keeps, grid_h: int, grid_w: int, heads: int, *, n_tokens: int,
+                                 pos=None, params: Optional[ficoco_params] = None, out_tokens=None, kept_idx=None,
+                                 pos_out=None, stream: Optional[int] = None) -> VResult:
+        """A progressive schedule in one call.  attns: list of cuda fp32 tensors, one per step
+        ([B, H, Np_s] over the patch tokens alive at that step); keeps: patch tokens preserved by
+        each step.  Returns the last step's tokens, kept_idx (into the original rows) and pos."""
+        import torch
+        p = params or ficoco_default_params()
+        cls = 1 if (p.flags & FICOCO_HAS_CLS) else 0
+        batch = tokens.shape[0] // n_tokens
+        keep_a = np.ascontiguousarray(np.asarray(keeps, dtype=np.int32))
+        n_steps = int(keep_a.shape[0])
+        rows = cls + int(keep_a[-1])
+        dim, dev = tokens.shape[-1], tokens.device
+        if out_tokens is None:
+            out_tokens = torch.empty((batch * rows, dim), dtype=tokens.dtype, device=dev)
+        if kept_idx is None:
+            kept_idx = torch.empty((batch * rows,), dtype=torch.int32, device=dev)
+        if pos_out is None:
+            pos_out = torch.empty((max(batch * int(keep_a[-1]), 1),), dtype=torch.int32, device=dev)
+        gh_a, gw_a = _int_array(grid_h)[0], _int_array(grid_w)[0]
+        a = ficoco_v_args()
+        a.tokens, a.pos = _ptr(tokens), _ptr(pos)
+        a.grid_h, a.grid_w = gh_a.ctypes.data, gw_a.ctypes.data
+        a.out_tokens, a.kept_idx, a.pos_out = _ptr(out_tokens), _ptr(kept_idx), _ptr(pos_out)
+        a.dtype, a.batch, a.n_tokens, a.dim, a.heads = _dtype_code(tokens), batch, n_tokens, dim, heads
+        a.n_grid, a.n_keep = 1, 1
+        ptrs = (C.c_void_p * n_steps)(*[t.data_ptr() for t in attns])
+        if stream is None:
+            stream = torch.cuda.current_stream(dev).cuda_stream
+        _check(self.h, self.lib.ficoco_v_reduce_schedule(self.h, C.byref(a), n_steps, keep_a.ctypes.data, ptrs,
+                                                         C.byref(p), C.c_void_p(stream)))
+        return VResult(out_tokens, kept_idx, pos_out, None, [rows] * batch)
 
     def ficoco_l_reduce(self, tokens, attn_t2v, keep, n_vision: int, n_text: int, heads: int, *,
                         params: Optional[ficoco_params] = None, out_tokens=None, kept_idx=None,

@@ -22,7 +22,7 @@ using namespace ficoco;
 
 namespace {
 
-constexpr int N_PLANS = 8;
+constexpr int N_PLANS = 16;
 constexpr int PART_PER_TOKEN = 64;   // partial top-list entries budgeted per token row
 constexpr int OUT_ROWS_PER_CTA = MROWS_CTA;  // the merge kernel's copy batches are sized for it
 constexpr int NSPLIT_MAX = 16;
@@ -193,6 +193,10 @@ struct ficoco_ctx {
   std::vector<int> prof_name;            // per recorded event: index into prof_acc, -1 = end of call
   struct ProfAcc { const char* name; double ms; long long launches; };
   std::vector<ProfAcc> prof_acc;
+
+  // grow-only intermediates of ficoco_v_reduce_schedule: tokens / positions ping-pong, kept indices per step
+  char* sch_base = nullptr;
+  size_t sch_bytes = 0;
 
   // grow-only staging for the host-buffer entry points
   char* hs_dev = nullptr;
@@ -453,6 +457,7 @@ extern "C" int ficoco_destroy(ficoco_ctx* c) {
   if (c->d_base) cudaFree(c->d_base);
   if (c->h_stage) cudaFreeHost(c->h_stage);
   if (c->hs_dev) cudaFree(c->hs_dev);
+  if (c->sch_base) cudaFree(c->sch_base);
   if (c->hs_stream) cudaStreamDestroy(c->hs_stream);
   if (c->hs_run) cudaStreamDestroy(c->hs_run);
   if (c->hs_out) cudaStreamDestroy(c->hs_out);
@@ -837,7 +842,7 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size
 template <class T, int VPL>
 cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* attn,
                                 int attn_rows, float cA, const int* pos, int window, float coef, int penalty,
-                                int* kept_idx, int* pos_out, float* scores_out, bool overlap_prev,
+                                int* kept_idx, int* pos_out, float* scores_out, int overlap_prev,
                                 cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p->f_grid);
@@ -850,13 +855,13 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
   at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = (c->coop_pdl_ok && overlap_prev) ? 2 : 1;
+  cfg.numAttrs = (c->coop_pdl_ok && overlap_prev) ? 2 : 1;   // 1: inputs independent of the step before; 2: fed by it
   return cudaLaunchKernelEx(&cfg, k_filter_fused<T, VPL>, tok, D, (const ImgDesc*)p->d_desc,
                             (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
                             p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), c->wait_ns,
-                            c->dbg_extra_arrivals);
+                            c->dbg_extra_arrivals, (c->coop_pdl_ok && overlap_prev == 2) ? 1 : 0);
 }
 
 template <class T, int VPL>
@@ -891,7 +896,9 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     if (spans_overlap(out_spans[o], rel_span)) return FICOCO_ERR_INVALID_ARG;
   }
   // the early start is taken only when the caller vouches for what sits in front of this step
-  const bool overlap_prev = back_to_back && inputs_clear_of_last_outputs(c->device, st, in_spans, 3);
+  // 0: plain stream order; 1: the filter grid may read its inputs under the tail of the step before;
+  // 2: it is fed by that step: launched early all the same, reads only once that step is complete
+  const int overlap_prev = !back_to_back ? 0 : inputs_clear_of_last_outputs(c->device, st, in_spans, 3) ? 1 : 2;
   record_last_outputs(c->device, st, out_spans, N_SPANS);
   if (p->fused) {
     prof_tick(c, st, "filter_fused");
@@ -1086,6 +1093,107 @@ extern "C" int ficoco_v_reduce_relation(ficoco_ctx* c, const ficoco_v_args* a, c
                                         int by_column, const ficoco_params* prm, void* cuda_stream) {
   if (!relation || ((uintptr_t)relation & 3)) return FICOCO_ERR_INVALID_ARG;
   return v_reduce_impl(c, a, prm, cuda_stream, relation, by_column ? 2 : 1);
+}
+
+// kept_idx of a schedule: the chain of the steps' kept indices, last step first.
+// kidx[s] : [B, rows_s] row indices into step s's input rows (rows_s = c + keep[s]).
+struct ComposeArgs {
+  const int* kidx[8];
+  int rows[8];
+  int n_steps;
+};
+__global__ void k_compose_kept(ComposeArgs a, int batch, int* __restrict__ out) {
+  const int rows_last = a.rows[a.n_steps - 1];
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= batch * rows_last) return;
+  const int b = i / rows_last;
+  int idx = a.kidx[a.n_steps - 1][i];
+  for (int s = a.n_steps - 2; s >= 0 && idx >= 0; --s) idx = a.kidx[s][(size_t)b * a.rows[s] + idx];
+  out[i] = idx;
+}
+
+extern "C" int ficoco_v_reduce_schedule(ficoco_ctx* c, const ficoco_v_args* first, int n_steps, const int* keep,
+                                        const float* const* attn, const ficoco_params* prm, void* cuda_stream) {
+  if (!c || !first || !keep || !attn || !prm) return FICOCO_ERR_INVALID_ARG;
+  if (n_steps < 1 || n_steps > 8) return FICOCO_ERR_INVALID_ARG;
+  if (first->seqlens || (prm->flags & FICOCO_CONVERGENT)) return FICOCO_ERR_UNSUPPORTED;
+  if (first->batch < 1 || first->n_tokens < 1 || first->dim < 1 || !first->out_tokens || !first->kept_idx)
+    return FICOCO_ERR_INVALID_ARG;
+  if (first->dtype != FICOCO_FP32 && first->dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
+  const int cls = (prm->flags & FICOCO_HAS_CLS) ? 1 : 0;
+  const size_t es = first->dtype == FICOCO_BF16 ? 2 : 4;
+  const int B = first->batch;
+  int np = first->n_tokens - cls;
+  for (int s = 0; s < n_steps; ++s) {
+    if (!attn[s]) return FICOCO_ERR_INVALID_ARG;
+    if (keep[s] < 0 || keep[s] > np) return FICOCO_ERR_KEEP_RANGE;
+    np = keep[s];
+  }
+  if (n_steps == 1) {
+    ficoco_v_args a = *first;
+    a.attn = attn[0]; a.keep = keep; a.n_keep = 1; a.scores_out = nullptr;
+    return ficoco_v_reduce(c, &a, prm, cuda_stream);
+  }
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  CUDA_TRY(c, cudaSetDevice(c->device));
+  // intermediates: tokens and positions ping-pong (A holds the outputs of even steps, B of odd
+  // ones), kept indices of every step
+  const size_t rows0 = (size_t)B * (cls + keep[0]), rows1 = (size_t)B * (cls + keep[1 < n_steps ? 1 : 0]);
+  const size_t tokA = align_up(rows0 * first->dim * es, 256), tokB = align_up(rows1 * first->dim * es, 256);
+  const size_t posA = align_up((size_t)B * keep[0] * 4 + 4, 256), posB = align_up((size_t)B * keep[1] * 4 + 4, 256);
+  size_t kid_bytes = 0;
+  for (int s = 0; s < n_steps; ++s) kid_bytes += align_up((size_t)B * (cls + keep[s]) * 4, 256);
+  const size_t need = tokA + tokB + posA + posB + kid_bytes;
+  if (need > c->sch_bytes) {
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    CUDA_TRY(c, cudaStreamIsCapturing(st, &cs));
+    if (cs != cudaStreamCaptureStatusNone) return FICOCO_ERR_CAPTURE;
+    CUDA_TRY(c, cudaDeviceSynchronize());
+    if (c->sch_base) { cudaFree(c->sch_base); c->sch_base = nullptr; c->sch_bytes = 0; }
+    CUDA_TRY(c, cudaMalloc((void**)&c->sch_base, need));
+    c->sch_bytes = need;
+  }
+  char* tok_buf[2] = {c->sch_base, c->sch_base + tokA};
+  int* pos_buf[2] = {(int*)(c->sch_base + tokA + tokB), (int*)(c->sch_base + tokA + tokB + posA)};
+  ComposeArgs ca = {};
+  ca.n_steps = n_steps;
+  char* kp = c->sch_base + tokA + tokB + posA + posB;
+  for (int s = 0; s < n_steps; ++s) {
+    ca.kidx[s] = (const int*)kp;
+    ca.rows[s] = cls + keep[s];
+    kp += align_up((size_t)B * (cls + keep[s]) * 4, 256);
+  }
+  ficoco_params ps = *prm;
+  int total_launches = 0;
+  np = first->n_tokens - cls;
+  for (int s = 0; s < n_steps; ++s) {
+    const bool last = s + 1 == n_steps;
+    ficoco_v_args a = *first;
+    a.seqlens = nullptr;
+    a.n_tokens = cls + np;
+    a.attn = attn[s];
+    a.keep = &keep[s];
+    a.n_keep = 1;
+    a.scores_out = nullptr;
+    if (s > 0) {
+      a.tokens = tok_buf[(s - 1) & 1];
+      a.pos = pos_buf[(s - 1) & 1];
+      ps.flags |= FICOCO_BACK_TO_BACK;              // the kernel in front of this step is the library's own
+    }
+    a.out_tokens = last ? first->out_tokens : (void*)tok_buf[s & 1];
+    a.pos_out = last ? first->pos_out : pos_buf[s & 1];
+    a.kept_idx = (int*)ca.kidx[s];
+    const int rc = ficoco_v_reduce(c, &a, &ps, cuda_stream);
+    if (rc) return rc;
+    total_launches += c->launches;
+    np = keep[s];
+  }
+  const int n_out = B * (cls + keep[n_steps - 1]);
+  k_compose_kept<<<(n_out + 255) / 256, 256, 0, st>>>(ca, B, first->kept_idx);
+  c->launches = total_launches + 1;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { c->last_cuda = (int)e; return FICOCO_ERR_CUDA; }
+  return FICOCO_OK;
 }
 
 extern "C" int ficoco_l_reduce(ficoco_ctx* c, const ficoco_l_args* a, const ficoco_params* prm,

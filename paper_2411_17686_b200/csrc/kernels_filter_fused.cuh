@@ -104,7 +104,8 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     const int* __restrict__ pos, int window, float coef, int penalty, float* __restrict__ s_pen,
     float* __restrict__ scores_out, int* __restrict__ S_idx, int* __restrict__ T_idx,
     int* __restrict__ kept_idx, int* __restrict__ pos_out, unsigned* __restrict__ status,
-    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals) {
+    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals,
+    int dep_wait_first) {
   constexpr int E = VecTraits<T>::E;
   constexpr int F_P2B = VPL <= 4 ? 2 : 1;   // rows a warp scores together in pass 2 (and has in flight from L2)
   extern __shared__ __align__(128) unsigned char fs_raw[];
@@ -142,6 +143,10 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // A step fed from the outputs of the step before it on the stream (a progressive schedule) is
+  // still launched early, so that its blocks are in place and set up when that step ends, but
+  // must not touch the tokens before then.
+  if (dep_wait_first) grid_dep_wait();
 
   if (warp == FWARPS) {
     // ------------------------------- producer (pass 1 only) -------------------------------

@@ -139,7 +139,12 @@ extern "C" int ficoco_vision_redundancy_noalloc(const void* tokens, int dtype, i
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES) return FICOCO_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
   if (g_scratch_addr[dev] == nullptr) {
+    // The address lookup may load the module: it must not run under stream capture.
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return FICOCO_ERR_CUDA; }
+    if (cs != cudaStreamCaptureStatusNone) return FICOCO_ERR_CAPTURE;
     // The array's name is only a handle on the host; the kernels need its device address.
     float* p = nullptr;
     if (cudaGetSymbolAddress((void**)&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) {
@@ -150,16 +155,18 @@ extern "C" int ficoco_vision_redundancy_noalloc(const void* tokens, int dtype, i
   }
   float* rn = g_scratch_addr[dev];
   float* partial = rn + NA_RN_FLOATS;
-  cudaStream_t st = (cudaStream_t)cuda_stream;
   const int grid = batch * chunks;
+  cudaGetLastError();                       // an error left over from earlier work is not this call's
   if (dtype == FICOCO_BF16) {
     const __nv_bfloat16* t = (const __nv_bfloat16*)tokens;
     k_na_colsum<__nv_bfloat16><<<grid, 256, 0, st>>>(t, n_tokens, n_cls, dim, chunks, rn, partial);
+    if (cudaGetLastError() != cudaSuccess) return FICOCO_ERR_CUDA;      // the second kernel needs the first
     k_na_rowdot<__nv_bfloat16><<<grid, 256, dim * sizeof(float), st>>>(t, n_tokens, n_cls, dim, chunks, rn,
                                                                          partial, v_out);
   } else {
     const float* t = (const float*)tokens;
     k_na_colsum<float><<<grid, 256, 0, st>>>(t, n_tokens, n_cls, dim, chunks, rn, partial);
+    if (cudaGetLastError() != cudaSuccess) return FICOCO_ERR_CUDA;
     k_na_rowdot<float><<<grid, 256, dim * sizeof(float), st>>>(t, n_tokens, n_cls, dim, chunks, rn, partial,
                                                               v_out);
   }

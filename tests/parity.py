@@ -16,6 +16,10 @@ SCORE_RTOL = 1e-5
 BF16_ATOL, BF16_RTOL = 2e-2, 1e-2
 FP32_ATOL, FP32_RTOL = 1e-5, 1e-5
 ALPHA_ATOL = 1e-4
+# Largest plain relative score error |got - exp| / |exp| seen by compare_stages (the tolerance is
+# measured against max(|s_i|, mean |s|) of the image because lambda v - (1 - lambda) a cancels for
+# some tokens); the full-size tests print it.
+WORST_PLAIN_REL = {}
 
 
 def params_to_abi(p: fo.Params, has_cls: bool):
@@ -78,7 +82,10 @@ def compare_stages(ctx: binding.Context, results: List[fo.StepResult], n_cls: in
                              (s_pen[p0:p0 + npatch], r.score, "score")):
             err = np.abs(got.astype(np.float64) - exp)
             tol = SCORE_RTOL * np.maximum(np.abs(exp), scale)
-            assert (err <= tol).all(), f"{tag} {nm}: max rel err {np.max(err / np.maximum(np.abs(exp), scale)):.3e}"
+            plain = float(np.max(err / np.maximum(np.abs(exp), 1e-300)))      # plain relative error, no scale floor
+            WORST_PLAIN_REL[nm] = max(WORST_PLAIN_REL.get(nm, 0.0), plain)
+            assert (err <= tol).all(), (f"{tag} {nm}: max rel err {np.max(err / np.maximum(np.abs(exp), scale)):.3e} "
+                                        f"(plain relative, where the two terms of the score cancel: {plain:.3e})")
         # index work: bit exact
         assert np.array_equal(S[s0:s0 + ns], np.sort(r.S)), tag + " S"
         assert np.array_equal(T[t0:t0 + nt], r.T), tag + " T"

@@ -475,10 +475,16 @@ def test_error_codes_and_status(ctx):
 # ---------------------------------------------------------------------------------------
 # full-size workloads, in the launch configuration the benchmark times
 # ---------------------------------------------------------------------------------------
+def _report_plain_score_error(what):
+    print(f"\n[{what}] worst plain relative score error so far: "
+          + ", ".join(f"{k} {v:.2e}" for k, v in sorted(parity.WORST_PLAIN_REL.items())))
+
+
 def test_full_c1(ctx):
     batch = synth.workload(1)
     gaps.repair_v(batch)
     parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="c1")
+    _report_plain_score_error("c1")
 
 
 def test_full_c2_schedule(ctx):
@@ -492,6 +498,7 @@ def test_full_c2_schedule(ctx):
         batch.pos = [r.pos_out for r in results]
         if step + 1 < 3:
             synth.regenerate_attention(batch, 2000, step + 1, 1.5)
+    _report_plain_score_error("c2 schedule")
 
 
 @pytest.mark.parametrize("by_column", [True, False], ids=["by-column", "by-row"])
@@ -503,10 +510,85 @@ def test_full_c2_shape_relation_mode(ctx, by_column):
     parity.run_and_compare_v_relation(ctx, batch, rels, by_column, fo.Params(), DEV, what="c2-relation")
 
 
-def test_full_c3_first_step(ctx):
+def test_full_c3_schedule(ctx):
+    """2880 -> 1440 -> 720 -> 320 at full size (8 images x 2881 tokens), every step on the checker's
+    previous output; the later steps reach top lists of three and two entries."""
     batch = synth.workload(3)
-    gaps.repair_v(batch)
-    parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="c3")
+    p = fo.Params()
+    for step, keep in enumerate(synth.SCHEDULES[3]):
+        batch.keep = [keep] * batch.batch
+        gaps.repair_v(batch)
+        _, results = parity.run_and_compare_v(ctx, batch, p, DEV, what=f"c3 step {step}")
+        batch.tokens = [r.out for r in results]
+        batch.pos = [r.pos_out for r in results]
+        if step + 1 < 3:
+            synth.regenerate_attention(batch, 3000, step + 1, 1.0)
+    _report_plain_score_error("c3 schedule")
+
+
+def _checker_chain(batch, sched, seed, sigma):
+    """The checker's chained run of a schedule: per step the (margin-repaired) attention it used,
+    and at the end the tokens, the composed kept indices and the positions."""
+    p = fo.Params()
+    attns, chain = [], None
+    for step, keep in enumerate(sched):
+        batch.keep = [keep] * batch.batch
+        gaps.repair_v(batch)
+        attns.append(np.stack(batch.attn, axis=0).astype(np.float32))
+        results = fo.v_reduce_batch(batch, p)
+        chain = [r.kept_idx if chain is None else c[r.kept_idx] for r, c in zip(results, chain or results)]
+        batch.tokens = [r.out for r in results]
+        batch.pos = [r.pos_out for r in results]
+        if step + 1 < len(sched):
+            synth.regenerate_attention(batch, seed, step + 1, sigma)
+    return attns, results, chain
+
+
+@pytest.mark.parametrize("idx,small", [(2, True), (3, True), (2, False)], ids=["c2-small", "c3-small", "c2-full"])
+def test_schedule_entry_point_chains_its_own_outputs(ctx, idx, small):
+    """ficoco_v_reduce_schedule runs all steps on the GPU's own intermediate outputs; the result is
+    compared with the checker's chained run of the same schedule: the composed kept indices and
+    the final positions exactly, the final tokens within the bf16 tolerance once per step (a
+    merged row may be rounded differently by one ulp in one step and feed the next).  The margins
+    that make a step's decisions unambiguous were established on the checker's intermediates; on
+    intermediates that differ by an ulp here and there a discarded token whose two best targets are
+    nearly tied can go to the other one, which moves two output rows: at most 1 % of the rows may
+    be off for that reason (what is kept, and where, must still agree exactly)."""
+    batch = synth.workload(idx, small=small)
+    sched = (synth.SCHEDULES_SMALL if small else synth.SCHEDULES)[idx]
+    pk = packing.pack_v(batch, DEV)
+    gh, gw = batch.grid[0]
+    attns, results, chain = _checker_chain(batch, sched, 1000 * idx, 1.5 if idx == 2 else 1.0)
+    attn_d = [torch.from_numpy(a.reshape(-1)).to(DEV) for a in attns]
+    pk.attn = attn_d[0]
+    prm = parity.params_to_abi(fo.Params(), True)
+    for rep in range(2):                                   # the second call allocates nothing
+        res = ctx.ficoco_v_reduce_schedule(pk.tokens, attn_d, sched, gh, gw, pk.heads, n_tokens=pk.n_tokens,
+                                           pos=pk.pos, params=prm)
+        torch.cuda.synchronize()
+        assert ctx.ficoco_status() == 0
+        out = binding.to_numpy(res.out_tokens).reshape(batch.batch, 1 + sched[-1], -1)
+        kidx = binding.to_numpy(res.kept_idx).reshape(batch.batch, -1)
+        pout = binding.to_numpy(res.pos_out).reshape(batch.batch, -1)
+        n_steps = len(sched)
+        rows_off = rows_all = 0
+        for b, r in enumerate(results):
+            assert np.array_equal(kidx[b], chain[b]), f"image {b}: composed kept indices"
+            assert np.array_equal(pout[b], r.pos_out), f"image {b}: positions"
+            g, e = fo.widen(out[b]), fo.widen(r.out)
+            tol = n_steps * (parity.BF16_ATOL + parity.BF16_RTOL * np.abs(e))
+            rows_off += int(np.any(np.abs(g - e) > tol, axis=1).sum())
+            rows_all += g.shape[0]
+            assert np.array_equal(out[b][0], r.out[0])   # CLS passes through every step untouched
+        assert rows_off <= 0.01 * rows_all, f"{rows_off} of {rows_all} final rows off"
+    # the same chain as separate calls gives the same bytes
+    cur_tok, cur_pos, n_tok = pk.tokens, pk.pos, pk.n_tokens
+    for s, keep in enumerate(sched):
+        r1 = ctx.ficoco_v_reduce(cur_tok, attn_d[s], keep, gh, gw, pk.heads, n_tokens=n_tok, pos=cur_pos, params=prm)
+        cur_tok, cur_pos, n_tok = r1.out_tokens, r1.pos_out, 1 + keep
+    torch.cuda.synchronize()
+    assert np.array_equal(binding.to_numpy(cur_tok), binding.to_numpy(res.out_tokens))
+    assert np.array_equal(binding.to_numpy(cur_pos), binding.to_numpy(res.pos_out))
 
 
 def test_full_c4(ctx):

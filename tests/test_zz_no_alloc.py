@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import ficoco_oracle as fo
 from paper_2411_17686_b200 import binding, packing, synth
 
 pytestmark = pytest.mark.gpu
@@ -39,6 +40,12 @@ def test_noalloc_matches_context_entry_point_twice():
         got = got.cpu().numpy().astype(np.float64)
         scale = float(np.mean(np.abs(want)))
         assert np.all(np.abs(got - want) <= 1e-5 * np.maximum(np.abs(want), scale))
+        # and against the float64 checker: the first term of Eq. 1 from the literal N x N relation
+        np_ = n_tokens - 1
+        for b in range(batch.batch):
+            P = fo.widen(batch.tokens[b])[1:]
+            exact = fo.vision_redundancy(fo.cosine_relation(P))
+            assert np.all(np.abs(got[b * np_:(b + 1) * np_] - exact) <= 1e-5 * np.abs(exact) + 1e-7)
     ctx.close()
 
 
