@@ -31,7 +31,9 @@
  *     synchronising.  A context must be used from one stream at a time.
  *   - The first call with a new combination of shapes builds and uploads a small plan
  *     (per-image descriptors); that first call may synchronise the stream and must happen
- *     outside stream capture.  Up to 8 plans are cached per context.
+ *     outside stream capture (or be replaced by ficoco_v_plan).  Up to 16 plans are cached per
+ *     context.  The per-image sizes come from host arrays (seqlens, keep, grids): the library
+ *     sizes its grids from them without reading anything back from the device.
  *   - Every function returns FICOCO_OK (0) or a negative ficoco_error; nothing is launched
  *     when argument validation fails.  Problems only the device can see (a `pos` entry
  *     outside the grid) set bits in a status word read by ficoco_status.
@@ -166,10 +168,21 @@ typedef struct ficoco_v_args {
   int n_grid;              /* 1 (same grid for all images) or B */
   int n_keep;              /* 1 or B */
   int reserved;
+  int* out_cu_seqlens;     /* device int32[B + 1] or NULL: receives the first output row of every
+                              image and, last, the total number of output rows (the cu_seqlens of
+                              the packed output, for the layers behind) */
 } ficoco_v_args;
 
 int ficoco_v_reduce(ficoco_ctx* ctx, const ficoco_v_args* args, const ficoco_params* params,
                     void* cuda_stream);
+
+/* Build and upload the plan for the shapes of `args` (batch, n_tokens or seqlens, dim, heads,
+ * dtype, grids, keep counts) and the settings of `params` ahead of time.  Only the host arrays of
+ * `args` are read; its device pointers may be NULL.  This call may synchronise the stream and must
+ * happen outside stream capture; afterwards ficoco_v_reduce with the same shapes and settings
+ * neither synchronises nor fails under capture (16 plans are cached per context, least recently
+ * used first out). */
+int ficoco_v_plan(ficoco_ctx* ctx, const ficoco_v_args* args, const ficoco_params* params, void* cuda_stream);
 
 /* FiCoCo-V reduce step on a caller-supplied relation matrix: the paper's own formulation, in
  * which every token-token quantity is read from the self-attention map A^v (Sec.

@@ -33,6 +33,7 @@ EXPORTS = [
     "ficoco_l_reduce_host", "ficoco_status", "ficoco_inspect", "ficoco_last_launch_count",
     "ficoco_profile", "ficoco_profile_read", "ficoco_vision_redundancy_noalloc",
     "ficoco_equivalent_token", "ficoco_v_reduce_relation", "ficoco_debug_waits", "ficoco_v_reduce_schedule",
+    "ficoco_v_plan",
 ]
 
 
@@ -48,7 +49,8 @@ class ficoco_v_args(C.Structure):
                 ("keep", C.c_void_p), ("out_tokens", C.c_void_p), ("kept_idx", C.c_void_p),
                 ("pos_out", C.c_void_p), ("scores_out", C.c_void_p),
                 ("dtype", C.c_int), ("batch", C.c_int), ("n_tokens", C.c_int), ("dim", C.c_int),
-                ("heads", C.c_int), ("n_grid", C.c_int), ("n_keep", C.c_int), ("reserved", C.c_int)]
+                ("heads", C.c_int), ("n_grid", C.c_int), ("n_keep", C.c_int), ("reserved", C.c_int),
+                ("out_cu_seqlens", C.c_void_p)]
 
 
 class ficoco_l_args(C.Structure):
@@ -94,6 +96,7 @@ def load_library() -> C.CDLL:
     lib.ficoco_l_reduce_host.argtypes = [C.c_void_p, C.POINTER(ficoco_l_args), C.POINTER(ficoco_params)]
     lib.ficoco_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int)]
     lib.ficoco_debug_waits.argtypes = [C.c_void_p, C.c_longlong, C.c_int]
+    lib.ficoco_v_plan.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_v_reduce_schedule.argtypes = [C.c_void_p, C.POINTER(ficoco_v_args), C.c_int, C.c_void_p, C.c_void_p,
                                              C.POINTER(ficoco_params), C.c_void_p]
     lib.ficoco_inspect.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]
@@ -187,7 +190,8 @@ class Context:
                         seqlens=None, pos=None, params: Optional[ficoco_params] = None,
                         out_tokens=None, kept_idx=None, pos_out=None, scores_out=None,
                         want_scores: bool = False, stream: Optional[int] = None,
-                        relation=None, by_column: bool = False) -> VResult:
+                        relation=None, by_column: bool = False, out_cu_seqlens=None,
+                        plan_only: bool = False) -> VResult:
         """tokens: cuda tensor [rows, D]; attn: cuda fp32 tensor (packed per image [H, Np]);
         keep / grid_h / grid_w: int or per-image list; seqlens: per-image rows incl. CLS or
         None with n_tokens given.  Output tensors are allocated with torch when not passed.
@@ -211,6 +215,16 @@ class Context:
         out_rows = [cls + k + (1 if conv and n - cls - k > 0 else 0) for k, n in zip(keeps, ntoks)]
         dim = tokens.shape[-1]
         dev = tokens.device
+        if plan_only:               # ficoco_v_plan: shapes only
+            a = ficoco_v_args()
+            a.seqlens = sl.ctypes.data if sl is not None else None
+            a.grid_h, a.grid_w, a.keep = gh_a.ctypes.data, gw_a.ctypes.data, keep_a.ctypes.data
+            a.dtype, a.batch, a.n_tokens, a.dim, a.heads = _dtype_code(tokens), batch, n_tokens, dim, heads
+            a.n_grid, a.n_keep = n_gh, n_keep
+            if stream is None:
+                stream = torch.cuda.current_stream(dev).cuda_stream
+            _check(self.h, self.lib.ficoco_v_plan(self.h, C.byref(a), C.byref(p), C.c_void_p(stream)))
+            return VResult(None, None, None, None, out_rows)
         if out_tokens is None:
             out_tokens = torch.empty((sum(out_rows), dim), dtype=tokens.dtype, device=dev)
         if kept_idx is None:
@@ -227,6 +241,7 @@ class Context:
         a.pos_out, a.scores_out = _ptr(pos_out), _ptr(scores_out)
         a.dtype, a.batch, a.n_tokens, a.dim, a.heads = _dtype_code(tokens), batch, n_tokens, dim, heads
         a.n_grid, a.n_keep = n_gh, n_keep
+        a.out_cu_seqlens = _ptr(out_cu_seqlens)
         if stream is None:
             stream = torch.cuda.current_stream(dev).cuda_stream
         if relation is not None:

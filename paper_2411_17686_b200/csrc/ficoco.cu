@@ -64,6 +64,7 @@ struct Plan {
   // fused persistent filter kernel
   bool fused = false;
   int* d_ctafirst = nullptr;
+  int* d_out_cu = nullptr;      // device int32[batch + 1]: first output row of every image, then the total
   int f_grid = 0, f_nstage = 0, f_max_piece = 0, f_vpl = 0;
   size_t f_smem = 0;
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
@@ -178,7 +179,7 @@ struct ficoco_ctx {
   bool coop_pdl_ok = false;  // a cooperative grid may also be a programmatic dependent
   char* plan_slots = nullptr;
   size_t slot_bytes = 0;
-  size_t off_rows = 0, off_corr = 0, off_out = 0, off_ctaf = 0;
+  size_t off_rows = 0, off_corr = 0, off_out = 0, off_ctaf = 0, off_ocu = 0;
   int cap_rows = 0, cap_corr = 0, cap_out = 0;
   long long cap_part = 0;
 
@@ -377,7 +378,8 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   c->off_corr = c->off_rows + align_up((size_t)c->cap_rows * sizeof(WorkItem), 256);
   c->off_out = c->off_corr + align_up((size_t)c->cap_corr * sizeof(WorkItem), 256);
   c->off_ctaf = c->off_out + align_up((size_t)c->cap_out * sizeof(WorkItem), 256);
-  c->slot_bytes = c->off_ctaf + align_up((size_t)(c->num_sms + 2) * sizeof(int), 256);
+  c->off_ocu = c->off_ctaf + align_up((size_t)(c->num_sms + 2) * sizeof(int), 256);
+  c->slot_bytes = c->off_ocu + align_up((B + 1) * sizeof(int), 256);
 
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
@@ -769,6 +771,12 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   p->d_corr = (WorkItem*)(slot_dev + c->off_corr);
   p->d_out = (WorkItem*)(slot_dev + c->off_out);
   p->d_ctafirst = (int*)(slot_dev + c->off_ctaf);
+  p->d_out_cu = (int*)(slot_dev + c->off_ocu);
+  {
+    int* ocu = (int*)(c->h_stage + c->off_ocu);
+    for (int b = 0; b < B; ++b) ocu[b] = p->h_desc[b].out_row0;
+    ocu[B] = p->tot_out_rows;
+  }
   p->key = key;
   if (p->fused) memcpy(c->h_stage + c->off_ctaf, cta_first.data(), cta_first.size() * sizeof(int));
   memcpy(c->h_stage + c->off_rows, rows.data(), rows.size() * sizeof(WorkItem));
@@ -1038,11 +1046,15 @@ int check_common(const ficoco_params* prm, int dtype, int batch, int dim, int he
 
 namespace {
 int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm, void* cuda_stream,
-                  const float* rel, int rel_mode) {
+                  const float* rel, int rel_mode, bool plan_only = false) {
   if (!c || !a) return FICOCO_ERR_INVALID_ARG;
-  int rc = check_common(prm, a->dtype, a->batch, a->dim, a->heads, a->tokens, a->out_tokens);
+  // planning needs the shapes only: stand-ins for the data pointers pass the checks
+  static const long long dummy[2] = {0, 0};
+  int rc = check_common(prm, a->dtype, a->batch, a->dim, a->heads, plan_only ? (const void*)dummy : a->tokens,
+                        plan_only ? (const void*)dummy : (const void*)a->out_tokens);
   if (rc) return rc;
-  if (!a->attn || !a->grid_h || !a->grid_w || !a->keep || !a->kept_idx) return FICOCO_ERR_INVALID_ARG;
+  if (!a->grid_h || !a->grid_w || !a->keep) return FICOCO_ERR_INVALID_ARG;
+  if (!plan_only && (!a->attn || !a->kept_idx)) return FICOCO_ERR_INVALID_ARG;
   if ((a->n_grid != 1 && a->n_grid != a->batch) || (a->n_keep != 1 && a->n_keep != a->batch))
     return FICOCO_ERR_INVALID_ARG;
   if (!a->seqlens && a->n_tokens < 1) return FICOCO_ERR_INVALID_ARG;
@@ -1069,8 +1081,12 @@ int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* pr
   Plan* p = nullptr;
   rc = get_plan(c, key, a->heads, st, &p);
   if (rc) return rc;
+  if (plan_only) return FICOCO_OK;
   c->last_plan = p;
   c->launches = 0;
+  if (a->out_cu_seqlens)       // prefix of the output rows per image, from the plan's device copy
+    CUDA_TRY(c, cudaMemcpyAsync(a->out_cu_seqlens, p->d_out_cu, (size_t)(a->batch + 1) * sizeof(int),
+                                cudaMemcpyDeviceToDevice, st));
   const int penalty = (prm->flags & FICOCO_LOCAL_PENALTY) ? 1 : 0;
   const bool b2b = (prm->flags & FICOCO_BACK_TO_BACK) != 0;
   if (a->dtype == FICOCO_BF16)
@@ -1087,6 +1103,10 @@ int v_reduce_impl(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* pr
 extern "C" int ficoco_v_reduce(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm,
                                void* cuda_stream) {
   return v_reduce_impl(c, a, prm, cuda_stream, nullptr, 0);
+}
+
+extern "C" int ficoco_v_plan(ficoco_ctx* c, const ficoco_v_args* a, const ficoco_params* prm, void* cuda_stream) {
+  return v_reduce_impl(c, a, prm, cuda_stream, nullptr, 0, true);
 }
 
 extern "C" int ficoco_v_reduce_relation(ficoco_ctx* c, const ficoco_v_args* a, const float* relation,

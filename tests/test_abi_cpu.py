@@ -29,7 +29,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_struct_layouts_match_header():
     # pointers first, then ints: no padding surprises between C and ctypes
     assert C.sizeof(binding.ficoco_params) == 5 * 8 + 4 * 4
-    assert C.sizeof(binding.ficoco_v_args) == 11 * 8 + 8 * 4
+    assert C.sizeof(binding.ficoco_v_args) == 11 * 8 + 8 * 4 + 8     # out_cu_seqlens last
     assert C.sizeof(binding.ficoco_l_args) == 6 * 8 + 8 * 4
 
 

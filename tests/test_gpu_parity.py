@@ -422,6 +422,50 @@ def test_step_behind_a_foreign_producer_kernel(ctx):
             assert np.array_equal(a, binding.to_numpy(b))
 
 
+def test_planned_ragged_shape_is_captured_into_a_graph():
+    """A ragged shape the context has never seen: ficoco_v_plan builds its plan ahead of time, after
+    which the reduce step is captured into a CUDA graph (no synchronisation, no allocation inside
+    the call) and the replay gives the bytes of an ordinary call; out_cu_seqlens holds the prefix of
+    the output rows.  Without the plan the captured call is refused with FICOCO_ERR_CAPTURE."""
+    c = binding.Context(max_tokens=8192, max_dim=256, max_batch=8, device=0)
+    batch = synth.make_v_batch(85, 5, 9, 7, 256, 4, 20, "bf16", False, 1.0)
+    for b, cut in enumerate((0, 5, 11, 2, 30)):          # five different lengths
+        if cut:
+            batch.tokens[b] = batch.tokens[b][:-cut]; batch.attn[b] = batch.attn[b][:, :-cut].copy()
+            batch.pos[b] = batch.pos[b][:-cut]
+    batch.keep = [20, 25, 17, 30, 9]
+    pk = packing.pack_v(batch, DEV)
+    prm = binding.make_params(has_cls=False)
+    rows = sum(batch.keep)
+    out = torch.zeros((rows, 256), dtype=torch.bfloat16, device=DEV)
+    kidx = torch.zeros((rows,), dtype=torch.int32, device=DEV)
+    pout = torch.zeros((rows,), dtype=torch.int32, device=DEV)
+    ocu = torch.zeros((6,), dtype=torch.int32, device=DEV)
+    st = torch.cuda.Stream()
+    kw = dict(params=prm, out_tokens=out, kept_idx=kidx, pos_out=pout, out_cu_seqlens=ocu, stream=st.cuda_stream,
+              **pk.call_kwargs())
+    g = torch.cuda.CUDAGraph()
+    with pytest.raises(binding.FicocoError) as e:
+        with torch.cuda.graph(g, stream=st):
+            c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **kw)
+    assert e.value.code == -7
+    torch.cuda.synchronize()
+    c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, plan_only=True, **kw)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, **kw)
+    g.replay()
+    torch.cuda.synchronize()
+    got = [binding.to_numpy(t) for t in (out, kidx, pout)]
+    assert ocu.cpu().tolist() == [0, 20, 45, 62, 92, 101]
+    ref = c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm, **pk.call_kwargs())
+    torch.cuda.synchronize()
+    for a, b in zip(got, (ref.out_tokens, ref.kept_idx, ref.pos_out)):
+        assert np.array_equal(a, binding.to_numpy(b))
+    assert c.ficoco_status() == 0
+    c.close()
+
+
 def test_error_codes_and_status(ctx):
     batch = synth.make_v_batch(84, 2, 6, 6, 64, 2, 20, "bf16", True, 1.0)
     pk = packing.pack_v(batch, DEV)
