@@ -1123,6 +1123,8 @@ struct ComposeArgs {
   int n_steps;
 };
 __global__ void k_compose_kept(ComposeArgs a, int batch, int* __restrict__ out) {
+  grid_dep_wait();        // launched under the tail of the last step's merge grid
+  grid_dep_launch();
   const int rows_last = a.rows[a.n_steps - 1];
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= batch * rows_last) return;
@@ -1209,7 +1211,7 @@ extern "C" int ficoco_v_reduce_schedule(ficoco_ctx* c, const ficoco_v_args* firs
     np = keep[s];
   }
   const int n_out = B * (cls + keep[n_steps - 1]);
-  k_compose_kept<<<(n_out + 255) / 256, 256, 0, st>>>(ca, B, first->kept_idx);
+  launch_dependent(k_compose_kept, (n_out + 255) / 256, 256, 0, st, ca, B, first->kept_idx);
   c->launches = total_launches + 1;
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { c->last_cuda = (int)e; return FICOCO_ERR_CUDA; }
