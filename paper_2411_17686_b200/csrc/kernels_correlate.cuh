@@ -10,6 +10,15 @@ namespace ficoco {
 constexpr int CBM = 64;   // source rows per CTA
 constexpr int CBN = 64;   // target columns per tile
 constexpr int CKC = 16;   // reduction chunk
+constexpr int CPG = 4;    // reduction chunks fetched together (one group in flight ahead of the multiply)
+
+// Four consecutive elements of a token row as fp32 (16-byte / 8-byte aligned).
+__device__ __forceinline__ float4 load4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
+  return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xFFFF0000u), __uint_as_float(v.y << 16),
+                     __uint_as_float(v.y & 0xFFFF0000u));
+}
 
 template <int LC>
 __device__ __forceinline__ void correlate_tail(
@@ -82,52 +91,46 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
       for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
     const int lr = tid >> 2, lq = tid & 3;
-    for (int k0 = 0; k0 < D; k0 += CKC) {
-      {
-        float fa[4] = {0.f, 0.f, 0.f, 0.f}, fb[4] = {0.f, 0.f, 0.f, 0.f};
-        const int kk = k0 + lq * 4;
-        if (kk < D) {
-          const int pa = rowS[lr], pb = rowT[lr];
-          if (sizeof(T) == 4) {
-            if (pa >= 0) {
-              float4 v = __ldg(reinterpret_cast<const float4*>(tokens + (tok0 + pa) * D + kk));
-              fa[0] = v.x; fa[1] = v.y; fa[2] = v.z; fa[3] = v.w;
-            }
-            if (pb >= 0) {
-              float4 v = __ldg(reinterpret_cast<const float4*>(tokens + (tok0 + pb) * D + kk));
-              fb[0] = v.x; fb[1] = v.y; fb[2] = v.z; fb[3] = v.w;
-            }
-          } else {
-            if (pa >= 0) {
-              uint2 v = __ldg(reinterpret_cast<const uint2*>(tokens + (tok0 + pa) * D + kk));
-              fa[0] = __uint_as_float(v.x << 16); fa[1] = __uint_as_float(v.x & 0xFFFF0000u);
-              fa[2] = __uint_as_float(v.y << 16); fa[3] = __uint_as_float(v.y & 0xFFFF0000u);
-            }
-            if (pb >= 0) {
-              uint2 v = __ldg(reinterpret_cast<const uint2*>(tokens + (tok0 + pb) * D + kk));
-              fb[0] = __uint_as_float(v.x << 16); fb[1] = __uint_as_float(v.x & 0xFFFF0000u);
-              fb[2] = __uint_as_float(v.y << 16); fb[3] = __uint_as_float(v.y & 0xFFFF0000u);
-            }
+    // Operands are fetched CPG reduction chunks at a time, one group ahead of the one being
+    // multiplied: a chunk per round trip to L2 made the loop pure latency (64 round trips for
+    // D = 1024).
+    const int pa = rowS[lr], pb = rowT[lr];
+    const T* rowA = tokens + (tok0 + (pa >= 0 ? pa : 0)) * D;
+    const T* rowB = tokens + (tok0 + (pb >= 0 ? pb : 0)) * D;
+    auto load_group = [&](int k0, float4 (&fa)[CPG], float4 (&fb)[CPG]) {
+#pragma unroll
+      for (int g = 0; g < CPG; ++g) {
+        const int kk = k0 + g * CKC + lq * 4;
+        fa[g] = (kk < D && pa >= 0) ? load4(rowA + kk) : make_float4(0.f, 0.f, 0.f, 0.f);
+        fb[g] = (kk < D && pb >= 0) ? load4(rowB + kk) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    };
+    float4 ca[CPG], cb[CPG], na[CPG], nb[CPG];
+    load_group(0, ca, cb);
+    #pragma unroll 1
+    for (int k0 = 0; k0 < D; k0 += CPG * CKC) {
+      if (k0 + CPG * CKC < D) load_group(k0 + CPG * CKC, na, nb);
+#pragma unroll
+      for (int g = 0; g < CPG; ++g) {
+        if (k0 + g * CKC < D) {
+          As[lq * 4 + 0][lr] = ca[g].x; As[lq * 4 + 1][lr] = ca[g].y; As[lq * 4 + 2][lr] = ca[g].z; As[lq * 4 + 3][lr] = ca[g].w;
+          Bs[lq * 4 + 0][lr] = cb[g].x; Bs[lq * 4 + 1][lr] = cb[g].y; Bs[lq * 4 + 2][lr] = cb[g].z; Bs[lq * 4 + 3][lr] = cb[g].w;
+          __syncthreads();
+#pragma unroll
+          for (int kk = 0; kk < CKC; ++kk) {
+            const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
           }
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          As[lq * 4 + e][lr] = fa[e];
-          Bs[lq * 4 + e][lr] = fb[e];
+          __syncthreads();
         }
       }
-      __syncthreads();
 #pragma unroll
-      for (int kk = 0; kk < CKC; ++kk) {
-        const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-        const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-      }
-      __syncthreads();
+      for (int g = 0; g < CPG; ++g) { ca[g] = na[g]; cb[g] = nb[g]; }
     }
 
     float cval[4][4];
