@@ -928,13 +928,14 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
         rel, p->d_desc, p->d_rows, attn, attn_rows, cA, p->key.rel == 2 ? 1 : 0, c->s_raw);
     c->launches += 1;
   } else {
-  prof_tick(c, st, vpl <= 8 ? "colsum" : "rownorm");
-  if (vpl <= 8) {
+  prof_tick(c, st, vpl <= 16 ? "colsum" : "rownorm");
+  if (vpl <= 16) {
     if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
     else if (vpl <= 2) launch_colsum_fused<T, 2>(c, p, tok, D, st);
     else if (vpl <= 4) launch_colsum_fused<T, 4>(c, p, tok, D, st);
     else if (vpl <= 5) launch_colsum_fused<T, 5>(c, p, tok, D, st);
-    else launch_colsum_fused<T, 8>(c, p, tok, D, st);
+    else if (vpl <= 8) launch_colsum_fused<T, 8>(c, p, tok, D, st);
+    else launch_colsum_fused<T, 16>(c, p, tok, D, st);      // rows of up to 4096 bf16 / 2048 fp32: one row per warp at a time
     c->launches += 1;
   } else {
     k_rownorm<T><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn);

@@ -75,21 +75,25 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
   const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D + c0;
   float* rn_out = rn + d.patch0 + w.r0;
 
-  for (int r = warp; r < w.nrows; r += 16) {
+  // rows in pairs (r, r + 8) while two rows fit in registers, one row at a time for very wide rows
+  constexpr bool PAIR = VPL <= 8;
+  for (int r = warp; r < w.nrows; r += PAIR ? 16 : 8) {
     const int r2 = r + 8;
-    const bool has2 = r2 < w.nrows;
-    uint4 u[VPL], u2[VPL];
+    const bool has2 = PAIR && r2 < w.nrows;
+    uint4 u[VPL], u2[PAIR ? VPL : 1];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
       const int v = lane + 32 * k;
       u[k] = (v < nvec) ? ldg16(base + (size_t)r * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
     }
+    if (PAIR) {
 #pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-      const int v = lane + 32 * k;
-      u2[k] = (has2 && v < nvec) ? ldg16(base + (size_t)r2 * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      for (int k = 0; k < VPL; ++k) {
+        const int v = lane + 32 * k;
+        u2[PAIR ? k : 0] = (has2 && v < nvec) ? ldg16(base + (size_t)r2 * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+      }
     }
-    float s1, s2;
+    float s1, s2 = 0.f;
     if (FUSED) {
       float ss = 0.f, ss2 = 0.f;
 #pragma unroll
@@ -98,14 +102,18 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
         unpack(u[k], f, (const T*)nullptr);
 #pragma unroll
         for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
-        unpack(u2[k], f, (const T*)nullptr);
+        if (PAIR) {
+          unpack(u2[PAIR ? k : 0], f, (const T*)nullptr);
 #pragma unroll
-        for (int e = 0; e < E; ++e) ss2 = fmaf(f[e], f[e], ss2);
+          for (int e = 0; e < E; ++e) ss2 = fmaf(f[e], f[e], ss2);
+        }
       }
       ss = warp_sum(ss);
-      ss2 = warp_sum(ss2);
       s1 = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-      s2 = ss2 > 0.f ? 1.0f / sqrtf(ss2) : 0.f;
+      if (PAIR) {
+        ss2 = warp_sum(ss2);
+        s2 = ss2 > 0.f ? 1.0f / sqrtf(ss2) : 0.f;
+      }
       if (lane == 0) {
         rn_out[r] = s1;
         if (has2) rn_out[r2] = s2;
@@ -120,9 +128,11 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
       unpack(u[k], f, (const T*)nullptr);
 #pragma unroll
       for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s1, acc[k][e]);
-      unpack(u2[k], f, (const T*)nullptr);
+      if (PAIR) {
+        unpack(u2[PAIR ? k : 0], f, (const T*)nullptr);
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s2, acc[k][e]);
+        for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s2, acc[k][e]);
+      }
     }
   }
 
