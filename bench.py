@@ -259,6 +259,14 @@ def other_workloads(binding, packing, ctx, insts, prm, stream, dev) -> dict:
             torch.cuda.synchronize()
             assert c2.ficoco_status(stream.cuda_stream) == 0
             out[label] = {"us_per_step": e0.elapsed_time(e1) * 1e3 / 20, "images": len(wl.tokens), "token_rows": rows}
+            # the library's own events between its launches (serialises them: shares, not a sum to compare)
+            c2.ficoco_profile(True)
+            with torch.cuda.stream(stream):
+                for _ in range(5):
+                    step()
+            torch.cuda.synchronize()
+            out[label]["kernels_us"] = {nm: round(1e3 * t / max(cnt, 1), 2) for nm, t, cnt in c2.ficoco_profile_read()}
+            c2.ficoco_profile(False)
         finally:
             c2.close()
     return out

@@ -17,19 +17,29 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Optional phase timestamps (compile with -DFICOCO_PHASE_TIMERS): thread 0 of a CTA notes the SM
-// clock at named points of a kernel; phase 0 also notes the global timer, so that the CTAs of a
-// grid can be laid on one time line.  Compiled out by default.
+// clock at named points of a kernel, in a record of its own that it draws from a per-kernel counter
+// (so that the records of several launches in a row can be told apart by their order); the record
+// also keeps the CTA's index and the global timer at its first and last mark, so that the CTAs of
+// all grids can be laid on one time line.  Compiled out by default.
 #ifdef FICOCO_PHASE_TIMERS
-constexpr int PH_KERNELS = 4, PH_CTAS = 1024, PH_SLOTS = 16;
+constexpr int PH_KERNELS = 4, PH_CTAS = 4096, PH_SLOTS = 16;
 __device__ unsigned long long g_phase_ts[PH_KERNELS][PH_CTAS][PH_SLOTS];
+__device__ unsigned g_phase_n[PH_KERNELS];
+#define FICOCO_PHASE_BEGIN(k)                                                          \
+  unsigned ph_rec = 0;                                                                 \
+  if (threadIdx.x == 0) {                                                              \
+    const unsigned long long c0 = (unsigned long long)clock64(), g0 = ficoco::global_ns(); \
+    ph_rec = atomicAdd(&ficoco::g_phase_n[k], 1u) % ficoco::PH_CTAS;                   \
+    ficoco::g_phase_ts[k][ph_rec][0] = c0;                                             \
+    ficoco::g_phase_ts[k][ph_rec][ficoco::PH_SLOTS - 1] = g0;                          \
+    ficoco::g_phase_ts[k][ph_rec][ficoco::PH_SLOTS - 2] = blockIdx.x;                  \
+  }
 #define FICOCO_PHASE(k, p)                                                             \
   do {                                                                                 \
-    if (threadIdx.x == 0 && blockIdx.x < ficoco::PH_CTAS) {                            \
-      ficoco::g_phase_ts[k][blockIdx.x][p] = (unsigned long long)clock64();            \
-      if ((p) == 0) ficoco::g_phase_ts[k][blockIdx.x][ficoco::PH_SLOTS - 1] = ficoco::global_ns(); \
-    }                                                                                  \
+    if (threadIdx.x == 0) ficoco::g_phase_ts[k][ph_rec][p] = (unsigned long long)clock64(); \
   } while (0)
 #else
+#define FICOCO_PHASE_BEGIN(k) do { } while (0)
 #define FICOCO_PHASE(k, p) do { } while (0)
 #endif
 

@@ -7,7 +7,7 @@
 namespace ficoco {
 
 constexpr int KCAP = 16;            // longest per-token top list (targets + 1 order statistic)
-constexpr int MAX_CHUNKS = 16;      // row chunks per image for the column-sum partials
+constexpr int MAX_CHUNKS = 64;      // row chunks per image for the column-sum partials
 constexpr int MAX_IMG_TOKENS = 8192;
 constexpr unsigned STATUS_POS_RANGE = 1u;
 

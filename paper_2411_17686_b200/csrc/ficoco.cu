@@ -155,6 +155,7 @@ struct ficoco_ctx {
   // scratch arrays
   float* rn = nullptr;
   float* partial = nullptr;
+  float* msum = nullptr;     // [B][max_dim] column sums of the unfused filter
   float* s_raw = nullptr;
   float* s_pen = nullptr;
   int* S_idx = nullptr;
@@ -169,7 +170,8 @@ struct ficoco_ctx {
   float* tmean = nullptr;
   unsigned* status = nullptr;
   int* tile_cnt = nullptr;  // per source tile: column splits of the correlate kernel that are done
-  int merge_ctas_per_sm = 1;    // resident CTAs of the merge kernel per SM
+  int merge_ctas_per_sm = 1;    // resident CTAs of the merge kernel per SM (register cap for 3)
+  int merge_ctas_per_sm_dense = 1;   // the same with the register cap for 4 (plans without the fused filter)
   int* img_cnt = nullptr;   // two sets of 3 * max_batch per-image counters of the fused filter kernel
   unsigned long long epoch = 0;          // fused filter launches so far (its parity picks the counter set)
   unsigned long long wait_ns = WAIT_NS_DEFAULT;   // bound of every device-side wait
@@ -314,7 +316,13 @@ extern "C" void ficoco_default_params(ficoco_params* p) {
 extern "C" int ficoco_phase_read(void* host_dst, size_t bytes) {
   if (cudaDeviceSynchronize() != cudaSuccess) return FICOCO_ERR_CUDA;
   const size_t n = sizeof(unsigned long long) * PH_KERNELS * PH_CTAS * PH_SLOTS;
-  return cudaMemcpyFromSymbol(host_dst, g_phase_ts, bytes < n ? bytes : n) == cudaSuccess ? FICOCO_OK : FICOCO_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(host_dst, g_phase_ts, bytes < n ? bytes : n) != cudaSuccess) return FICOCO_ERR_CUDA;
+  // start the next run from empty records
+  static const unsigned long long zeros[PH_SLOTS * 64] = {0};
+  for (size_t o = 0; o < n; o += sizeof(zeros))
+    if (cudaMemcpyToSymbol(g_phase_ts, zeros, sizeof(zeros), o) != cudaSuccess) return FICOCO_ERR_CUDA;
+  const unsigned zn[PH_KERNELS] = {0};
+  return cudaMemcpyToSymbol(g_phase_n, zn, sizeof(zn)) == cudaSuccess ? FICOCO_OK : FICOCO_ERR_CUDA;
 }
 #endif
 
@@ -384,6 +392,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   size_t off = 0;
   auto carve = [&](size_t bytes) { size_t o = off; off += align_up(bytes, 256); return o; };
   const size_t o_rn = carve(T * 4), o_partial = carve((size_t)c->cap_rows * max_dim * 4);
+  const size_t o_msum = carve((size_t)B * max_dim * 4);
   const size_t o_icnt = carve(6 * B * 4);
   const size_t o_tcnt = carve((size_t)c->cap_corr * 4);
 
@@ -402,7 +411,7 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   if (e == cudaSuccess) e = cudaMallocHost((void**)&c->h_stage, c->slot_bytes);
   if (e != cudaSuccess) { cudaFree(c->d_base); delete c; return FICOCO_ERR_CUDA; }
   char* b = c->d_base;
-  c->rn = (float*)(b + o_rn); c->partial = (float*)(b + o_partial);
+  c->rn = (float*)(b + o_rn); c->partial = (float*)(b + o_partial); c->msum = (float*)(b + o_msum);
   c->s_raw = (float*)(b + o_sraw); c->s_pen = (float*)(b + o_spen);
   c->S_idx = (int*)(b + o_S); c->T_idx = (int*)(b + o_T);
   c->part_val = (float*)(b + o_pv); c->part_idx = (int*)(b + o_pi);
@@ -442,8 +451,10 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
   }
   {
     int nb = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_scan<__nv_bfloat16>, 256, 0) == cudaSuccess && nb > 0)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_scan<__nv_bfloat16, 3>, 256, 0) == cudaSuccess && nb > 0)
       c->merge_ctas_per_sm = nb;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, k_merge_scan<__nv_bfloat16, 4>, 256, 0) == cudaSuccess && nb > 0)
+      c->merge_ctas_per_sm_dense = nb;
   }
   cudaFuncSetAttribute(k_score<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
   cudaFuncSetAttribute(k_score<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
@@ -625,6 +636,12 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     while (out_rows_cta > 2 && n_out_ctas(out_rows_cta) < 2LL * c->num_sms &&
            n_out_ctas(out_rows_cta / 2) <= c->cap_out)
       out_rows_cta /= 2;
+    // 24 rows per CTA when the grid then fits the SMs in one go and did not before.  Not ahead of the
+    // persistent filter: the next step's filter grid starts only once every SM has drained, and longer
+    // merge CTAs delay that by more than the saved wave gains (measured: +2.4 us per step with, -4.5 us
+    // per step on a supplied relation map, whose score kernel is an ordinary grid).
+    const long long slots = (long long)c->num_sms * (p->fused ? c->merge_ctas_per_sm : c->merge_ctas_per_sm_dense);
+    if (out_rows_cta == OUT_ROWS_PER_CTA && n_out_ctas(16) > slots && n_out_ctas(24) <= slots && !p->fused) out_rows_cta = 24;
     p->out_rows_cta = out_rows_cta;
   }
   for (int b = 0; b < B; ++b) {
@@ -637,7 +654,11 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     // row chunks (fused filter: equal pieces of at most f_rc rows)
     int rc = (d.np + MAX_CHUNKS - 1) / MAX_CHUNKS;
     rc = (rc + 7) / 8 * 8;
-    if (rc < 64) rc = 64;
+    // unfused filter: chunks of about 256 KB of token rows (at most 64 rows; 32 rows of 4096 bf16), so
+    // that wide rows still give every SM several CTAs
+    int rc_floor = (int)(262144 / ((size_t)key.dim * (key.dtype == FICOCO_BF16 ? 2 : 4))) / 8 * 8;
+    rc_floor = rc_floor < 8 ? 8 : (rc_floor > 64 ? 64 : rc_floor);
+    if (rc < rc_floor) rc = rc_floor;
     if (p->fused) {
       const int npc = (d.np + f_rc - 1) / f_rc;
       rc = ((d.np + npc - 1) / npc + 7) / 8 * 8;
@@ -928,14 +949,18 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
         rel, p->d_desc, p->d_rows, attn, attn_rows, cA, p->key.rel == 2 ? 1 : 0, c->s_raw);
     c->launches += 1;
   } else {
-  prof_tick(c, st, vpl <= 16 ? "colsum" : "rownorm");
-  if (vpl <= 16) {
+  const bool wide = vpl > 8 && nvec <= 1024;   // rows of 257 .. 1024 16-byte vectors: CTA-wide rows
+  prof_tick(c, st, (vpl <= 8 || wide) ? "colsum" : "rownorm");
+  if (vpl <= 8) {
     if (vpl <= 1) launch_colsum_fused<T, 1>(c, p, tok, D, st);
     else if (vpl <= 2) launch_colsum_fused<T, 2>(c, p, tok, D, st);
     else if (vpl <= 4) launch_colsum_fused<T, 4>(c, p, tok, D, st);
     else if (vpl <= 5) launch_colsum_fused<T, 5>(c, p, tok, D, st);
-    else if (vpl <= 8) launch_colsum_fused<T, 8>(c, p, tok, D, st);
-    else launch_colsum_fused<T, 16>(c, p, tok, D, st);      // rows of up to 4096 bf16 / 2048 fp32: one row per warp at a time
+    else launch_colsum_fused<T, 8>(c, p, tok, D, st);
+    c->launches += 1;
+  } else if (wide) {
+    if (nvec <= 512) k_colsum_wide<T, 2, 8><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn, c->partial);
+    else k_colsum_wide<T, 4, 4><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn, c->partial);
     c->launches += 1;
   } else {
     k_rownorm<T><<<p->n_rows, 256, 0, st>>>(tok, D, p->d_desc, p->d_rows, c->rn);
@@ -946,9 +971,17 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     c->launches += 2;
   }
   prof_tick(c, st, "score");
-  k_score<T><<<p->n_rows, 256, (size_t)(D + p->max_rc) * sizeof(float), st>>>(
-      tok, D, p->d_desc, p->d_rows, c->rn, c->partial, attn, attn_rows, cA, c->s_raw);
-  c->launches += 1;
+  k_msum<<<dim3(p->key.batch, (D + 255) / 256), 256, 0, st>>>(D, p->d_desc, c->partial, c->msum);
+  if (wide && nvec <= 512)
+    k_score_wide<T, 2, 8><<<p->n_rows, 256, (size_t)9 * p->max_rc * sizeof(float), st>>>(
+        tok, D, p->d_desc, p->d_rows, c->rn, c->msum, attn, attn_rows, cA, c->s_raw);
+  else if (wide)
+    k_score_wide<T, 4, 4><<<p->n_rows, 256, (size_t)9 * p->max_rc * sizeof(float), st>>>(
+        tok, D, p->d_desc, p->d_rows, c->rn, c->msum, attn, attn_rows, cA, c->s_raw);
+  else
+    k_score<T><<<p->n_rows, 256, (size_t)(D + 9 * p->max_rc) * sizeof(float), st>>>(
+        tok, D, p->d_desc, p->d_rows, c->rn, c->msum, attn, attn_rows, cA, c->s_raw);
+  c->launches += 2;
   }
   size_t sel_smem = select_work_bytes(p->max_np, penalty ? p->max_nwin_cells : 0) + 16;
   if (p->max_np <= SEL_SMALL_MAX) {
@@ -1014,10 +1047,16 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
   }
   prof_tick(c, st, "merge_compact");
   const int after_correlate = p->n_corr > 0 ? 1 : 0;   // else the grid before may be the filter itself
-  launch_dependent(k_merge_scan<T>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
-                   (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
-                   (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
-                   (const unsigned*)c->status);
+  if (p->fused)
+    launch_dependent(k_merge_scan<T, 3>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+                     (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
+                     (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
+                     (const unsigned*)c->status);
+  else
+    launch_dependent(k_merge_scan<T, 4>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
+                     (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
+                     (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
+                     (const unsigned*)c->status);
   c->launches += 1;
   if (p->key.conv) {
     prof_tick(c, st, "convergent_token");

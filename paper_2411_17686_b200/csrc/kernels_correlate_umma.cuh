@@ -177,7 +177,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   __shared__ float rnT[UN_MAX];
   __shared__ int failed, acc_committed, is_last, dead;
 
-  FICOCO_PHASE(1, 0);
+  FICOCO_PHASE_BEGIN(1);
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int L = d.list_len;
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
   const uint32_t ring = (smem_u32(um_raw) + 1023u) & ~1023u;
 
   if (tid == 0) {
-    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full_bar[s], 256); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < NSTAGE; ++s) { mbar_init(&full_bar[s], 8); mbar_init(&empty_bar[s], 1); }
     mbar_init(&acc_bar, 1);
     failed = 0;
     acc_committed = 0;
@@ -284,7 +284,9 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       if (done >= 0) {
         cp_async_wait<LAG>();
         fence_proxy_async();
-        mbar_arrive(&full_bar[done % NSTAGE]);
+        // one arrival per producer warp: 256 arrivals per stage queue up on the barrier word
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full_bar[done % NSTAGE]);
       }
     }
     cp_async_wait<0>();

@@ -75,25 +75,21 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
   const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D + c0;
   float* rn_out = rn + d.patch0 + w.r0;
 
-  // rows in pairs (r, r + 8) while two rows fit in registers, one row at a time for very wide rows
-  constexpr bool PAIR = VPL <= 8;
-  for (int r = warp; r < w.nrows; r += PAIR ? 16 : 8) {
+  for (int r = warp; r < w.nrows; r += 16) {
     const int r2 = r + 8;
-    const bool has2 = PAIR && r2 < w.nrows;
-    uint4 u[VPL], u2[PAIR ? VPL : 1];
+    const bool has2 = r2 < w.nrows;
+    uint4 u[VPL], u2[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
       const int v = lane + 32 * k;
       u[k] = (v < nvec) ? ldg16(base + (size_t)r * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
     }
-    if (PAIR) {
 #pragma unroll
-      for (int k = 0; k < VPL; ++k) {
-        const int v = lane + 32 * k;
-        u2[PAIR ? k : 0] = (has2 && v < nvec) ? ldg16(base + (size_t)r2 * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
-      }
+    for (int k = 0; k < VPL; ++k) {
+      const int v = lane + 32 * k;
+      u2[k] = (has2 && v < nvec) ? ldg16(base + (size_t)r2 * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
     }
-    float s1, s2 = 0.f;
+    float s1, s2;
     if (FUSED) {
       float ss = 0.f, ss2 = 0.f;
 #pragma unroll
@@ -102,18 +98,14 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
         unpack(u[k], f, (const T*)nullptr);
 #pragma unroll
         for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
-        if (PAIR) {
-          unpack(u2[PAIR ? k : 0], f, (const T*)nullptr);
+        unpack(u2[k], f, (const T*)nullptr);
 #pragma unroll
-          for (int e = 0; e < E; ++e) ss2 = fmaf(f[e], f[e], ss2);
-        }
+        for (int e = 0; e < E; ++e) ss2 = fmaf(f[e], f[e], ss2);
       }
       ss = warp_sum(ss);
+      ss2 = warp_sum(ss2);
       s1 = ss > 0.f ? 1.0f / sqrtf(ss) : 0.f;
-      if (PAIR) {
-        ss2 = warp_sum(ss2);
-        s2 = ss2 > 0.f ? 1.0f / sqrtf(ss2) : 0.f;
-      }
+      s2 = ss2 > 0.f ? 1.0f / sqrtf(ss2) : 0.f;
       if (lane == 0) {
         rn_out[r] = s1;
         if (has2) rn_out[r2] = s2;
@@ -128,11 +120,9 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
       unpack(u[k], f, (const T*)nullptr);
 #pragma unroll
       for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s1, acc[k][e]);
-      if (PAIR) {
-        unpack(u2[PAIR ? k : 0], f, (const T*)nullptr);
+      unpack(u2[k], f, (const T*)nullptr);
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s2, acc[k][e]);
-      }
+      for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], s2, acc[k][e]);
     }
   }
 
@@ -155,31 +145,57 @@ __global__ void __launch_bounds__(256) k_colsum(const T* __restrict__ tokens, in
 
 // ---------------------------------------------------------------------------------------
 // Eq. 1 (and the FiCoCo-L score): s_i = cA * v_i - (1 - cA) * a_i with
-//   v_i = rn_i * (x_i . msum) / Np,   msum = sum of the image's column-sum partials,
+//   v_i = rn_i * (x_i . msum) / Np,   msum = the image's column sums (k_msum),
 //   a_i = (1/H) sum_h attn[h, i]      (FiCoCo-L: H = M rows of the head-mean block t).
 // One CTA per row chunk, one warp per token for the dot product.
 // ---------------------------------------------------------------------------------------
+// Column sums of every image: msum[b, c] = sum over the image's row chunks, in chunk order.
+__global__ void __launch_bounds__(256) k_msum(int D, const ImgDesc* __restrict__ desc,
+                                              const float* __restrict__ partial, float* __restrict__ msum) {
+  const ImgDesc d = desc[blockIdx.x];
+  const int c = blockIdx.y * 256 + threadIdx.x;
+  if (c >= D) return;
+  float s = 0.f;
+  for (int k = 0; k < d.n_chunks; ++k) s += partial[(size_t)(d.chunk0 + k) * D + c];
+  msum[(size_t)blockIdx.x * D + c] = s;
+}
+
+// Mean over the H attention rows of the chunk's tokens, a_i = (1/H) sum_h attn[h, i], by all 256 threads:
+// warp q adds rows q, q + 8, ... for 32 tokens per lane trip (eight loads in flight), the eight partial sums
+// of a token are then added in warp order.  `part` holds 8 * nrows floats.
+__device__ __forceinline__ void attn_mean_rows(const float* __restrict__ a0, int H, int np, int nrows,
+                                               float* part, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  for (int r = lane; r < nrows; r += 32) {
+    float s = 0.f;
+    for (int h0 = warp; h0 < H; h0 += 64) {
+      float q[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) q[j] = h0 + 8 * j < H ? __ldg(a0 + (size_t)(h0 + 8 * j) * np + r) : 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) s += q[j];
+    }
+    part[warp * nrows + r] = s;
+  }
+}
+
 template <class T>
 __global__ void __launch_bounds__(256) k_score(const T* __restrict__ tokens, int D,
                                                const ImgDesc* __restrict__ desc,
                                                const WorkItem* __restrict__ work,
                                                const float* __restrict__ rn,
-                                               const float* __restrict__ partial,
+                                               const float* __restrict__ msum_all,
                                                const float* __restrict__ attn, int H, float cA,
                                                float* __restrict__ s_raw) {
   constexpr int E = VecTraits<T>::E;
-  extern __shared__ float sm[];  // msum[D], v[nrows]
+  extern __shared__ float sm[];  // msum[D], v[nrows], attention partial sums [8][nrows]
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   float* msum = sm;
   float* vrow = sm + D;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-  for (int c = threadIdx.x; c < D; c += 256) {
-    float s = 0.f;
-    for (int k = 0; k < d.n_chunks; ++k) s += partial[(size_t)(d.chunk0 + k) * D + c];
-    msum[c] = s;
-  }
+  for (int c = threadIdx.x; c < D; c += 256) msum[c] = msum_all[(size_t)w.img * D + c];
   __syncthreads();
 
   const int nvec = D / E;
@@ -212,10 +228,167 @@ __global__ void __launch_bounds__(256) k_score(const T* __restrict__ tokens, int
   __syncthreads();
 
   const float inv_h = 1.0f / (float)H;
+  float* part = vrow + w.nrows;
+  attn_mean_rows(attn + d.attn0 + w.r0, H, d.np, w.nrows, part, threadIdx.x);
+  __syncthreads();
   for (int r = threadIdx.x; r < w.nrows; r += 256) {
-    const float* a = attn + d.attn0 + w.r0 + r;
     float s = 0.f;
-    for (int h = 0; h < H; ++h) s += __ldg(a + (size_t)h * d.np);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) s += part[q * w.nrows + r];
+    s_raw[d.patch0 + w.r0 + r] = cA * vrow[r] - (1.0f - cA) * (s * inv_h);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Wide rows (more than 256 16-byte vectors: hidden 4096 in bf16): a row no longer fits one
+// warp's registers, so the CTA's 256 threads own the row's column vectors (NV each) and rows
+// go through in batches of RB.  A per-row sum is folded lane -> warp -> the 8 warps in order.
+//   k_colsum_wide: row norms and the chunk's column sums of the normalised rows in one read;
+//                  every thread keeps the sums of its own columns, so there is no fold at the end
+//   k_score_wide:  Eq. 1 with the image's column sums held in registers
+// ---------------------------------------------------------------------------------------
+template <class T, int NV, int RB>
+__device__ __forceinline__ void wide_load(const T* __restrict__ base, int D, int nvec, int r0, int nrows, int tid,
+                                          uint4 (&u)[RB][NV]) {
+  constexpr int E = VecTraits<T>::E;
+#pragma unroll
+  for (int j = 0; j < RB; ++j)
+#pragma unroll
+    for (int k = 0; k < NV; ++k) {
+      const int v = tid + 256 * k;
+      u[j][k] = (r0 + j < nrows && v < nvec) ? ldg16(base + (size_t)(r0 + j) * D + (size_t)v * E) : make_uint4(0, 0, 0, 0);
+    }
+}
+
+__device__ __forceinline__ float fold8(const float* r) {
+  const float4 a = *reinterpret_cast<const float4*>(r), b = *reinterpret_cast<const float4*>(r + 4);
+  return ((((((a.x + a.y) + a.z) + a.w) + b.x) + b.y) + b.z) + b.w;
+}
+
+template <class T, int NV, int RB>
+__global__ void __launch_bounds__(256, 2) k_colsum_wide(const T* __restrict__ tokens, int D,
+                                                     const ImgDesc* __restrict__ desc,
+                                                     const WorkItem* __restrict__ work,
+                                                     float* __restrict__ rn_out, float* __restrict__ partial) {
+  constexpr int E = VecTraits<T>::E;
+  __shared__ __align__(16) float red[2][RB][8];
+  const WorkItem w = work[blockIdx.x];
+  const ImgDesc d = desc[w.img];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = D / E;
+  const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D;
+  float* rn = rn_out + d.patch0 + w.r0;
+  float acc[NV][E];
+#pragma unroll
+  for (int k = 0; k < NV; ++k)
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[k][e] = 0.f;
+
+  int par = 0;
+  for (int r0 = 0; r0 < w.nrows; r0 += RB, par ^= 1) {
+    uint4 u[RB][NV];
+    wide_load<T, NV, RB>(base, D, nvec, r0, w.nrows, tid, u);
+#pragma unroll
+    for (int j = 0; j < RB; ++j) {
+      float ss = 0.f;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        float f[E];
+        unpack(u[j][k], f, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
+      }
+      ss = warp_sum(ss);
+      if (lane == 0) red[par][j][warp] = ss;
+    }
+    __syncthreads();   // one barrier per batch: the next batch writes the other half of `red`
+#pragma unroll
+    for (int j = 0; j < RB; ++j) {
+      const float tot = fold8(red[par][j]);
+      const float sc = tot > 0.f ? 1.0f / sqrtf(tot) : 0.f;
+      if (tid == j && r0 + j < w.nrows) rn[r0 + j] = sc;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        float f[E];
+        // unpack again rather than keep the batch's converted values in registers across the barrier
+        asm volatile("" : "+r"(u[j][k].x), "+r"(u[j][k].y), "+r"(u[j][k].z), "+r"(u[j][k].w));
+        unpack(u[j][k], f, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[k][e] = fmaf(f[e], sc, acc[k][e]);
+      }
+    }
+  }
+  float* out = partial + (size_t)(d.chunk0 + w.aux) * D;
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int v = tid + 256 * k;
+    if (v < nvec) {
+#pragma unroll
+      for (int e = 0; e < E; e += 4)
+        *reinterpret_cast<float4*>(out + (size_t)v * E + e) = make_float4(acc[k][e], acc[k][e + 1], acc[k][e + 2], acc[k][e + 3]);
+    }
+  }
+}
+
+template <class T, int NV, int RB>
+__global__ void __launch_bounds__(256) k_score_wide(const T* __restrict__ tokens, int D,
+                                                    const ImgDesc* __restrict__ desc,
+                                                    const WorkItem* __restrict__ work,
+                                                    const float* __restrict__ rn,
+                                                    const float* __restrict__ msum_all,
+                                                    const float* __restrict__ attn, int H, float cA,
+                                                    float* __restrict__ s_raw) {
+  constexpr int E = VecTraits<T>::E;
+  extern __shared__ float vrow[];  // v[nrows], attention partial sums [8][nrows]
+  __shared__ __align__(16) float red[2][RB][8];
+  const WorkItem w = work[blockIdx.x];
+  const ImgDesc d = desc[w.img];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = D / E;
+  const T* base = tokens + (size_t)(d.row0 + d.n_cls + w.r0) * D;
+  float m[NV][E];
+#pragma unroll
+  for (int k = 0; k < NV; ++k) {
+    const int v = tid + 256 * k;
+#pragma unroll
+    for (int e = 0; e < E; e += 4) {
+      const float4 q = v < nvec ? __ldg(reinterpret_cast<const float4*>(msum_all + (size_t)w.img * D + (size_t)v * E + e))
+                                : make_float4(0.f, 0.f, 0.f, 0.f);
+      m[k][e] = q.x; m[k][e + 1] = q.y; m[k][e + 2] = q.z; m[k][e + 3] = q.w;
+    }
+  }
+  const float inv_np = 1.0f / (float)d.np;
+  int par = 0;
+  for (int r0 = 0; r0 < w.nrows; r0 += RB, par ^= 1) {
+    uint4 u[RB][NV];
+    wide_load<T, NV, RB>(base, D, nvec, r0, w.nrows, tid, u);
+#pragma unroll
+    for (int j = 0; j < RB; ++j) {
+      float dot = 0.f;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        float f[E];
+        unpack(u[j][k], f, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < E; ++e) dot = fmaf(f[e], m[k][e], dot);
+      }
+      dot = warp_sum(dot);
+      if (lane == 0) red[par][j][warp] = dot;
+    }
+    __syncthreads();
+    if (tid < RB && r0 + tid < w.nrows)
+      vrow[r0 + tid] = fold8(red[par][tid]) * rn[d.patch0 + w.r0 + r0 + tid] * inv_np;
+  }
+  __syncthreads();
+
+  const float inv_h = 1.0f / (float)H;
+  float* part = vrow + w.nrows;
+  attn_mean_rows(attn + d.attn0 + w.r0, H, d.np, w.nrows, part, tid);
+  __syncthreads();
+  for (int r = tid; r < w.nrows; r += 256) {
+    float s = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) s += part[q * w.nrows + r];
     s_raw[d.patch0 + w.r0 + r] = cA * vrow[r] - (1.0f - cA) * (s * inv_h);
   }
 }
@@ -230,6 +403,23 @@ __global__ void __launch_bounds__(256) k_head_mean(const float* __restrict__ att
   const float inv_h = 1.0f / (float)H;
   const float* src = attn + ((size_t)b * H * M + k) * N;
   float* dst = t + ((size_t)b * M + k) * N;
+  if ((N & 3) == 0 && (reinterpret_cast<uintptr_t>(attn) & 15) == 0 && (reinterpret_cast<uintptr_t>(t) & 15) == 0) {
+    // four tokens per thread, eight heads in flight, added in head order
+    for (int i = threadIdx.x * 4; i < N; i += 1024) {
+      float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int h0 = 0; h0 < H; h0 += 8) {
+        float4 a[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          a[q] = h0 + q < H ? __ldg(reinterpret_cast<const float4*>(src + (size_t)(h0 + q) * M * N + i))
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) { s.x += a[q].x; s.y += a[q].y; s.z += a[q].z; s.w += a[q].w; }
+      }
+      *reinterpret_cast<float4*>(dst + i) = make_float4(s.x * inv_h, s.y * inv_h, s.z * inv_h, s.w * inv_h);
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < N; i += 256) {
     float s = 0.f;
     for (int h0 = 0; h0 < H; h0 += 8) {      // eight heads in flight, added in head order
@@ -527,7 +717,6 @@ __device__ __noinline__ void select_small(
     }
   }
   cta_sync(bar, NT);
-  FICOCO_PHASE(0, 9);
 
   // ---- local penalty: one thread per window ------------------------------------------------
   if (penalty) {
@@ -552,7 +741,6 @@ __device__ __noinline__ void select_small(
     cta_sync(bar, NT);
   }
 
-  FICOCO_PHASE(0, 10);
   // ---- keys, their range, dense keys -----------------------------------------------------------
   uint32_t key[2];
   uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
@@ -591,7 +779,6 @@ __device__ __noinline__ void select_small(
     if (on[q]) wk.nk[tid + NT * q] = nk[q];
   }
 
-  FICOCO_PHASE(0, 11);
   // ---- radix select on the dense keys: the n_src-th largest -------------------------------------
   uint32_t thr = 0;      // threshold (dense key)
   int need_eq = 0;       // how many of the keys equal to thr are selected (lowest indices)
@@ -651,7 +838,6 @@ __device__ __noinline__ void select_small(
     need_eq = remaining;
   }
 
-  FICOCO_PHASE(0, 12);
   // ---- membership ---------------------------------------------------------------------------------
   bool sel[2];
 #pragma unroll
@@ -702,7 +888,6 @@ __device__ __noinline__ void select_small(
       }
     }
   }
-  FICOCO_PHASE(0, 13);
   if (w_lo == 0) {
     #pragma unroll 1
     for (int i = tid; i < d.n_cls; i += NT) kept_idx[d.out_row0 + i] = i;

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   // All CTAs of this grid are co-resident, so the next grid may be staged right away: its blocks
   // take over SMs as blocks of this grid exit and park until this grid has completed.
   grid_dep_launch();
-  FICOCO_PHASE(0, 0);
+  FICOCO_PHASE_BEGIN(0);
   __shared__ int won[F_MAXWON];
   __shared__ int nwon, failed;
 

@@ -7,7 +7,7 @@ namespace ficoco {
 
 constexpr int MHUB = 4;        // source rows a lane has in flight for a hub row
 constexpr int MROWS = 32;      // most output rows a CTA can take (sizes of the per-row arrays)
-constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp)
+constexpr int MROWS_CTA = 16;  // output rows per CTA the host plans (two per warp); 24 when that saves a wave
 constexpr int MCOPY = MROWS_CTA / 8;   // rows a warp copies in one batch
 constexpr int MLIST = 1024;    // (source, alpha) entries a CTA can hold in shared memory
 constexpr int MHEAVY = 2;      // rows with more sources than this are split into 32-vector blocks over the warps
@@ -59,8 +59,11 @@ __device__ __forceinline__ void merge_accumulate(float (&acc)[MVB][VecTraits<T>:
 //      rows with few sources by their own warp; hub rows are cut into blocks of 32 vectors that
 //      are dealt to the warps, every lane summing the sources of its vector in list order.
 // If the CTA's rows receive more than MLIST sources in total, a slow in-order rescan is used.
-template <class T>
-__global__ void __launch_bounds__(256) k_merge_scan(
+// MINB (resident CTAs per SM the registers are capped for): 4 fills the SMs better when the merge
+// grid runs between ordinary grids; 3 (no spills, fewer and shorter waves of CTAs draining) is
+// faster when the next step's persistent filter grid is waiting for every SM to drain.
+template <class T, int MINB>
+__global__ void __launch_bounds__(256, MINB) k_merge_scan(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out,
@@ -73,7 +76,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   __shared__ float tw[MLIST];
   __shared__ int heavy_rows[MROWS];
   __shared__ int n_heavy, dead;
-  FICOCO_PHASE(2, 0);
+  FICOCO_PHASE_BEGIN(2);
   const WorkItem w = work[blockIdx.x];
   const ImgDesc d = desc[w.img];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -195,13 +198,16 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   }
   __syncthreads();
 
+  FICOCO_PHASE(2, 2);
   // ---- rows without sources: plain copies, all of a warp's rows in flight together --------------
+  #pragma unroll 1
+  for (int j0 = 0; 8 * j0 < w.nrows; j0 += MCOPY)
   #pragma unroll 1
   for (int v0 = lane; v0 < nvec; v0 += 32 * MVB) {
     uint4 u[MCOPY][MVB];
 #pragma unroll
     for (int j = 0; j < MCOPY; ++j) {
-      const int r = warp + 8 * j;
+      const int r = warp + 8 * (j0 + j);
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
       const bool copy = r < w.nrows && srow_s[r < w.nrows ? r : 0] >= 0 && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
@@ -214,7 +220,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     }
 #pragma unroll
     for (int j = 0; j < MCOPY; ++j) {
-      const int r = warp + 8 * j;
+      const int r = warp + 8 * (j0 + j);
       const int orow = w.r0 + r;
       const bool is_tgt = orow >= d.n_cls && orow < d.n_cls + d.n_tgt;
       const bool copy = r < w.nrows && srow_s[r < w.nrows ? r : 0] >= 0 && (!is_tgt || cnt[orow - d.n_cls - tp_lo] == 0);
@@ -227,6 +233,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     }
   }
 
+  FICOCO_PHASE(2, 3);
   // ---- rows with a few sources: one warp per row --------------------------------------------------
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
@@ -289,6 +296,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
   }
   if (!fits) return;
 
+  FICOCO_PHASE(2, 4);
   // ---- hub rows: (row, block of 32 vectors) items dealt to the warps; each lane sums all the
   // sources of its one vector in list order, MHUB source rows in flight ---------------------
   const int nh = n_heavy;
@@ -329,6 +337,7 @@ __global__ void __launch_bounds__(256) k_merge_scan(
     for (int q = 0; q < E; ++q) acc[q] = acc[q] * inv_den;
     st_stream16(reinterpret_cast<uint4*>(dst) + v, pack(acc, (const T*)nullptr));
   }
+  FICOCO_PHASE(2, 5);
 }
 
 // Ablation "convergent correlation" (Sec. "Correlation-based Information Recycling": all discarded
