@@ -783,6 +783,7 @@ __device__ __noinline__ void select_small(
   uint32_t thr = 0;      // threshold (dense key)
   int need_eq = 0;       // how many of the keys equal to thr are selected (lowest indices)
   int c_eq = 0;          // how many keys equal thr
+  uint32_t thr_mask = 0xFFFFFFFFu;   // digits of the dense keys the passes have looked at
   if (k > 0 && k < np) {
     const int npass = range ? (32 - sh_l + 7) / 8 : 1;   // the low sh_l bits of every dense key are zero
     uint32_t prefix = 0, mask = 0;
@@ -833,9 +834,11 @@ __device__ __noinline__ void select_small(
       c_eq = __shfl_sync(0xFFFFFFFFu, ceq_new, src);
       prefix |= (uint32_t)digit << shift;
       mask |= 0xFFu << shift;
+      if (remaining == c_eq) break;    // every key that shares these digits is selected: no need to tell them apart
     }
     thr = prefix;
     need_eq = remaining;
+    thr_mask = mask;
   }
 
   // ---- membership ---------------------------------------------------------------------------------
@@ -846,10 +849,11 @@ __device__ __noinline__ void select_small(
     if (!on[q]) sel[q] = false;
     else if (k <= 0) sel[q] = false;
     else if (k >= np) sel[q] = true;
-    else if (nk[q] != thr) sel[q] = nk[q] > thr;
+    else if ((nk[q] & thr_mask) != thr) sel[q] = (nk[q] & thr_mask) > thr;
     else if (need_eq >= c_eq) sel[q] = true;
     else {
       // equal scores straddle the boundary: the lowest indices among them are taken
+      // (all passes were made, so the mask covers every bit that is set in any key)
       int before = 0;
       #pragma unroll 1
       for (int j = 0; j < i; ++j) before += wk.nk[j] == thr ? 1 : 0;

@@ -177,6 +177,19 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   FICOCO_PHASE(0, 1);
   int seq = 0;
   bool ok = true;
+  // The attention term of the first piece's rows depends on nothing this kernel computes: it is
+  // fetched now, while the ring fills, instead of between the two passes.
+  if (p_begin < p_end) {
+    const WorkItem w = pieces[p_begin];
+    const ImgDesc d = desc[w.img];
+    const float inv_h = 1.0f / (float)H;
+    for (int r = tid; r < w.nrows; r += F_NCONS) {
+      const float* a = attn + d.attn0 + w.r0 + r;
+      float t = 0.f;
+      for (int h = 0; h < H; ++h) t += __ldg(a + (size_t)h * d.np);
+      a_s[r] = t * inv_h;
+    }
+  }
   // pass 1: norms and column sums
   for (int pi = p_begin; pi < p_end; ++pi) {
     const WorkItem w = pieces[pi];
@@ -286,7 +299,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     }
     if (pi == p_begin) FICOCO_PHASE(0, 3);
     const float inv_h = 1.0f / (float)H;
-    for (int r = tid; r < w.nrows; r += F_NCONS) {     // attention term, does not depend on the wait
+    for (int r = tid; pi > p_begin && r < w.nrows; r += F_NCONS) {     // attention term of a further piece
       const float* a = attn + d.attn0 + w.r0 + r;
       float t = 0.f;
       for (int h = 0; h < H; ++h) t += __ldg(a + (size_t)h * d.np);
