@@ -13,6 +13,7 @@
 #include "common.cuh"
 #include "kernels_correlate.cuh"
 #include "kernels_correlate_umma.cuh"
+#include "kernels_correlate_umma_f32.cuh"
 #include "kernels_filter.cuh"
 #include "kernels_filter_fused.cuh"
 #include "kernels_merge.cuh"
@@ -70,6 +71,8 @@ struct Plan {
   // tensor-core correlate (bf16, hidden size a multiple of 64, FiCoCo-V)
   bool need_finalize = false;   // some image merges nothing: its per-token counts are zeroed by a kernel
   bool umma = false;
+  bool um_f32 = false;          // fp32 tokens split into three bf16 terms (k_correlate_umma_f32)
+  int um_b_bytes = 0;
   int um_stage_bytes = 0, um_a_bytes = 0, um_tmem_cols = 0, um_nstage = 0;
   size_t um_smem = 0;
   std::vector<ImgDesc> h_desc;
@@ -439,6 +442,9 @@ extern "C" int ficoco_create(ficoco_ctx** out, int device, long long max_tokens,
     cudaFuncSetAttribute(k_correlate_umma<6, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<6, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
     cudaFuncSetAttribute(k_correlate_umma<6, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma_f32<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma_f32<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
+    cudaFuncSetAttribute(k_correlate_umma_f32<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, um_smem_max);
   }
   {
     const int fmax = 221 * 1024;
@@ -499,7 +505,11 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   // in the epilogue from weights staged in shared memory, 2 KB per text token for the largest tile.
   p->umma = key.dtype == FICOCO_BF16 && key.dim % UKB == 0 &&
             (key.mode == 0 || (size_t)key.n_text * 2048 + 1024 + (size_t)UM * KCAP * 8 <= 220 * 1024);
-  if (key.rel) p->umma = false;                       // C is read from the supplied matrix, not contracted
+  // fp32 tokens (FiCoCo-V): the same tiling with narrower column tiles, operands split into bf16 terms
+  p->um_f32 = key.dtype == FICOCO_FP32 && key.dim % UKB == 0 && key.mode == 0;
+  if (p->um_f32) p->umma = true;
+  if (key.rel) p->umma = p->um_f32 = false;           // C is read from the supplied matrix, not contracted
+  const int un_max = p->um_f32 ? UF_COLS : UN_MAX;    // accumulator columns per CTA
   int tile_rows_max = p->umma ? UM : CBM;             // source rows per correlate CTA (decided below)
   if (key.rel) {
     // a warp of the relation correlate takes one discarded token at a time and is bound by the
@@ -591,7 +601,9 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     const long long slots = (long long)c->num_sms * ctas_per_sm;
     long long ws = slots / strips;
     if (ws < 1) ws = 1;
-    if (ws > NSPLIT_MAX) ws = NSPLIT_MAX;
+    // (fp32 tiles: the CTA that completes a tile merges nsplit * L entries per token, one thread each)
+    const int split_max = p->um_f32 ? 8 : NSPLIT_MAX;
+    if (ws > split_max) ws = split_max;
     ch.want_split = (int)ws;
     long long n_ctas = 0, max_rows = 0;
     for (int b = 0; b < B; ++b) {
@@ -601,7 +613,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       const int max_by_cols = (d.n_tgt + col_granule - 1) / col_granule;
       if (ns > max_by_cols) ns = max_by_cols;
       int cps = ((d.n_tgt + ns - 1) / ns + col_granule - 1) / col_granule * col_granule;
-      if (p->umma && cps > UN_MAX) cps = UN_MAX;
+      if (p->umma && cps > un_max) cps = un_max;
       ns = (d.n_tgt + cps - 1) / cps;
       const int ntile = (d.n_src + rows_max - 1) / rows_max;
       const int trows = ((d.n_src + ntile - 1) / ntile + 7) / 8 * 8;
@@ -616,7 +628,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
   int want_split = 1;
   {
     CorrChoice best = cost_corr(tile_rows_max, 2);
-    if (p->umma) {
+    if (p->umma && !p->um_f32) {
       const CorrChoice wide = cost_corr(UM * UM_SUB, 1);
       if (wide.load > 0 && wide.load * 10 <= best.load * 7) best = wide;
     }
@@ -679,7 +691,7 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
       if (ns > max_by_cols) ns = max_by_cols;
       int cps = (d.n_tgt + ns - 1) / ns;
       cps = (cps + col_granule - 1) / col_granule * col_granule;
-      if (p->umma && cps > UN_MAX) cps = UN_MAX;
+      if (p->umma && cps > un_max) cps = un_max;
       ns = (d.n_tgt + cps - 1) / cps;
       d.nsplit = ns; d.cols_per_split = cps;
       const size_t corr_before = corr.size();
@@ -759,7 +771,16 @@ int build_plan(ficoco_ctx* c, Plan* p, const PlanKey& key, int slot) {
     return FICOCO_ERR_WORKSPACE;
   p->tot_patch = (int)patch0; p->tot_src = (int)src0; p->tot_tgt = (int)tgt0; p->tot_out_rows = (int)out0;
   p->n_rows = (int)rows.size(); p->n_corr = (int)corr.size(); p->n_out = (int)outw.size();
-  if (p->umma) {
+  if (p->um_f32) {
+    // two stages of three bf16 tiles per operand, 16 KB behind them for the 128-row reads of the last A tile
+    p->um_a_bytes = um_a_rows * 128;
+    p->um_b_bytes = (um_cols + 15) / 16 * 16 * 128;
+    p->um_tmem_cols = 32;
+    while (p->um_tmem_cols < 6 * (p->um_b_bytes / 128)) p->um_tmem_cols *= 2;   // six partial products per entry
+    p->um_nstage = UF_STAGES;
+    p->um_smem = (size_t)UF_STAGES * 3 * (p->um_a_bytes + p->um_b_bytes) + (size_t)UM * 128 + 2048;
+    if (um_a_rows > UM || um_cols > UF_COLS || p->um_smem > 220 * 1024) return FICOCO_ERR_UNSUPPORTED;
+  } else if (p->umma) {
     // shared-memory ring of the tensor-core correlate: prefer a size that lets two CTAs share an SM
     p->um_a_bytes = um_a_rows * 128;
     p->um_stage_bytes = p->um_a_bytes + um_cols * 128;
@@ -1009,6 +1030,19 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       else if (p->max_list <= 4) FICOCO_REL_GO(4);
       else FICOCO_REL_GO(16);
 #undef FICOCO_REL_GO
+    } else if (p->um_f32 && sizeof(T) == 4) {
+      prof_tick(c, st, "correlate_umma_f32");
+      const float* tk = reinterpret_cast<const float*>(tok);
+#define FICOCO_UF32_LAUNCH(LC)                                                                         \
+  launch_dependent(k_correlate_umma_f32<LC>, p->n_corr, UTHREADS, p->um_smem, st, tk, D,               \
+      (const ImgDesc*)p->d_desc, (const WorkItem*)p->d_corr, (const float*)c->rn,                       \
+      (const int*)c->S_idx, (const int*)c->T_idx, c->part_val, c->part_idx, c->status,                 \
+      p->um_a_bytes, p->um_b_bytes, p->um_tmem_cols, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,        \
+      c->e_w, c->e_c, c->wait_ns)
+      if (p->max_list <= 2) FICOCO_UF32_LAUNCH(2);
+      else if (p->max_list <= 4) FICOCO_UF32_LAUNCH(4);
+      else FICOCO_UF32_LAUNCH(16);
+#undef FICOCO_UF32_LAUNCH
     } else if (p->umma && sizeof(T) == 2) {
       prof_tick(c, st, "correlate_umma");
       const __nv_bfloat16* tk = reinterpret_cast<const __nv_bfloat16*>(tok);
