@@ -111,6 +111,22 @@ def test_fp32_wide_rows(ctx):
     parity.run_and_compare_v(ctx, batch, fo.Params(), DEV, what="fp32-wide")
 
 
+@pytest.mark.parametrize("keep", [130, 30])
+def test_fp32_tensor_core_correlate_tiles(ctx, keep):
+    """fp32 tokens whose hidden size is a multiple of 64 take the tensor-core correlate that splits
+    every value into three bf16 terms: several tiles of discarded tokens, column splits with a ragged
+    last one, ragged images, fixed K and pruning, all at the fp32 tolerances."""
+    batch = synth.make_v_batch(85, 3, 20, 20, 128, 4, keep, "fp32", True, 1.2)
+    # ragged: the second image loses a fifth of its cells
+    alive = np.sort(synth.rng_for(85, 1, 8).permutation(400)[:320]).astype(np.int32)
+    batch.tokens[1] = np.concatenate([batch.tokens[1][:1], batch.tokens[1][1:][alive]], axis=0)
+    batch.attn[1] = batch.attn[1][:, alive].copy()
+    batch.pos[1] = alive
+    for p in (fo.Params(), fo.Params(eps=0.9), fo.Params(max_targets=2), fo.Params(max_targets=0)):
+        gaps.repair_v(batch, p)
+        parity.run_and_compare_v(ctx, batch, p, DEV, what=f"fp32-umma-keep{keep}")
+
+
 def _relations(batch, seed, stochastic=True, times_n=False):
     c = 1 if batch.has_cls else 0
     rels = []
