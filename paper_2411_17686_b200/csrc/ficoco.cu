@@ -910,7 +910,7 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
                             (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
-                            p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), c->wait_ns,
+                            p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), 3 * c->max_batch, c->wait_ns,
                             c->dbg_extra_arrivals, (c->coop_pdl_ok && overlap_prev == 2) ? 1 : 0);
 }
 

@@ -12,7 +12,7 @@
 //   select  images of up to 1024 tokens: every CTA that scored a piece waits until all of the
 //           image's scores are in, runs the (short) selection on the whole image and writes the
 //           outputs of its own tokens; larger images: the CTA that finishes the last piece runs
-//           the selection alone.  The last CTA to leave an image resets its counters.
+//           the selection alone.
 // The inter-CTA waits are polls of per-image counters, bounded by elapsed time (wait_ns).  The
 // counters exist twice; a launch uses the set of its parity and zeroes the other one, so a step
 // that gave up half-way cannot leave counts behind for the step after the next.
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
     const int* __restrict__ pos, int window, float coef, int penalty, float* __restrict__ s_pen,
     float* __restrict__ scores_out, int* __restrict__ S_idx, int* __restrict__ T_idx,
     int* __restrict__ kept_idx, int* __restrict__ pos_out, unsigned* __restrict__ status,
-    int nstage, int max_piece, int parity, unsigned long long wait_ns, int dbg_extra_arrivals,
+    int nstage, int max_piece, int parity, int set_stride, unsigned long long wait_ns, int dbg_extra_arrivals,
     int dep_wait_first) {
   constexpr int E = VecTraits<T>::E;
   constexpr int F_P2B = VPL <= 4 ? 2 : 1;   // rows a warp scores together in pass 2 (and has in flight from L2)
@@ -127,13 +127,16 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
   float* fold = reinterpret_cast<float*>(fs_raw + (size_t)nstage * stage_bytes);   // [FFOLD][D], msum aliases fold[0]
   float* a_s = fold + (size_t)FFOLD * D;                                            // [max_piece]
   const int p_begin = cta_first[blockIdx.x], p_end = cta_first[blockIdx.x + 1];
-  // counters of this launch: [0, B) pieces through pass 1, [B, 2B) pieces scored, [2B, 3B) pieces
-  // whose CTA has left the selection.  The other set belongs to the launch before and the one after.
+  // counters of this launch: [0, B) pieces through pass 1, [B, 2B) pieces scored ([2B, 3B) unused).
+  // The other set belongs to the launch before and the one after: it is zeroed here for the latter
+  // (the launch before is complete: the correlate grid between the two waited for it).
   {
-    int* other = cnt + (parity ? 0 : 3 * B);
+    // (the sets lie set_stride apart whatever the batch of this launch, so that launches of
+    // different plans find and clear each other's counters)
+    int* other = cnt + (parity ? 0 : set_stride);
     if (blockIdx.x == 0)
-      for (int i = tid; i < 3 * B; i += F_THREADS) other[i] = 0;
-    cnt += parity ? 3 * B : 0;
+      for (int i = tid; i < set_stride; i += F_THREADS) other[i] = 0;
+    cnt += parity ? set_stride : 0;
   }
 
   if (tid == 0) {
@@ -416,20 +419,15 @@ __global__ void __launch_bounds__(F_THREADS, 1) k_filter_fused(
       FICOCO_PHASE(0, 7);
       select_small(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
                    status, ring, sel_small_sh, tid, 1, w0.r0, hi);
-      cta_sync(1, F_NCONS);
-      if (tid == 0) {
-        // the last pieces to leave reset the image's counters (everybody is past its polls by then)
-        const int old = atomicAdd(&cnt[2 * B + w0.img], pj - pi);
-        if (old + (pj - pi) == d.n_chunks) { cnt[w0.img] = 0; cnt[B + w0.img] = 0; cnt[2 * B + w0.img] = 0; }
-      }
+      // (the counters are not reset here: the next launch zeroes this launch's set, see the top)
+      if (pj < p_end) cta_sync(1, F_NCONS);     // the work area is reused by the next image
     } else {
       bool mine = false;
       for (int k = 0; k < nwon; ++k) mine = mine || won[k] == w0.img;
       if (mine) {
         select_image(d, s_raw, pos, window, coef, penalty, s_pen, scores_out, S_idx, T_idx, kept_idx, pos_out,
                      status, ring, sel_sh, tid, F_NCONS, 1);
-        cta_sync(1, F_NCONS);
-        if (tid == 0) { cnt[w0.img] = 0; cnt[B + w0.img] = 0; }
+        if (pj < p_end) cta_sync(1, F_NCONS);
       }
     }
     pi = pj;
