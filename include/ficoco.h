@@ -257,7 +257,9 @@ int ficoco_l_reduce(ficoco_ctx* ctx, const ficoco_l_args* args, const ficoco_par
  * HOST pointer here.  The call copies the inputs to the device, runs the same kernels,
  * copies the outputs back and returns after the results are in host memory.  Staging
  * buffers are allocated inside the context on the first host call (sized by the maxima
- * given to ficoco_create) and reused.
+ * given to ficoco_create) and reused.  Large batches go through in groups of images (V) or
+ * sequences (L) whose uploads, kernels and downloads overlap on three internal streams; the
+ * results are the same bytes as those of one device-buffer call on the whole batch.
  */
 int ficoco_v_reduce_host(ficoco_ctx* ctx, const ficoco_v_args* host_args,
                          const ficoco_params* params);

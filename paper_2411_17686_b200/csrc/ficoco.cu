@@ -1550,19 +1550,24 @@ extern "C" int ficoco_l_reduce_host(ficoco_ctx* c, const ficoco_l_args* h, const
     return FICOCO_ERR_INVALID_ARG;
   if (h->dtype != FICOCO_FP32 && h->dtype != FICOCO_BF16) return FICOCO_ERR_UNSUPPORTED;
   const size_t es = h->dtype == FICOCO_BF16 ? 2 : 4;
-  long long orows = 0;
-  for (int b = 0; b < h->batch; ++b) {
+  const int B = h->batch;
+  std::vector<long long> p_orow(B + 1, 0);
+  for (int b = 0; b < B; ++b) {
     const int k = h->keep[h->n_keep == 1 ? 0 : b];
     if (k < 0 || k > h->n_vision) return FICOCO_ERR_KEEP_RANGE;
-    orows += k + h->n_text + (((prm->flags & FICOCO_CONVERGENT) && h->n_vision - k > 0) ? 1 : 0);
+    p_orow[b + 1] = p_orow[b] + k + h->n_text + (((prm->flags & FICOCO_CONVERGENT) && h->n_vision - k > 0) ? 1 : 0);
   }
-  const long long rows = (long long)h->batch * (h->n_vision + h->n_text);
+  const long long orows = p_orow[B];
+  const long long rows = (long long)B * (h->n_vision + h->n_text);
   if (rows > c->max_tokens) return FICOCO_ERR_WORKSPACE;
   CUDA_TRY(c, cudaSetDevice(c->device));
-  const size_t b_tok = (size_t)rows * h->dim * es;
-  const size_t b_attn = (size_t)h->batch * h->heads * h->n_text * h->n_vision * 4;
-  const size_t b_out = (size_t)orows * h->dim * es, b_kidx = (size_t)orows * 4;
-  const size_t b_sc = h->scores_out ? (size_t)h->batch * h->n_vision * 4 : 0;
+  const size_t seq_tok = (size_t)(h->n_vision + h->n_text) * h->dim * es;      // bytes per sequence
+  const size_t seq_attn = (size_t)h->heads * h->n_text * h->n_vision * 4;
+  const size_t seq_sc = (size_t)h->n_vision * 4;
+  const size_t row_b = (size_t)h->dim * es;
+  const size_t b_tok = seq_tok * B, b_attn = seq_attn * B;
+  const size_t b_out = (size_t)orows * row_b, b_kidx = (size_t)orows * 4;
+  const size_t b_sc = h->scores_out ? seq_sc * B : 0;
   const size_t total = align_up(b_tok, 256) + align_up(b_attn, 256) + align_up(b_out, 256) +
                        align_up(b_kidx, 256) + align_up(b_sc, 256) + 256;
   int rc = ensure_staging(c, total);
@@ -1573,17 +1578,67 @@ extern "C" int ficoco_l_reduce_host(ficoco_ctx* c, const ficoco_l_args* h, const
   char* d_out = dv.take<char>(b_out);
   char* d_kidx = dv.take<char>(b_kidx);
   char* d_sc = dv.take<char>(b_sc);
-  cudaStream_t st = c->hs_stream;
-  CUDA_TRY(c, cudaMemcpyAsync(d_tok, h->tokens, b_tok, cudaMemcpyHostToDevice, st));
-  CUDA_TRY(c, cudaMemcpyAsync(d_attn, h->attn_t2v, b_attn, cudaMemcpyHostToDevice, st));
-  ficoco_l_args a = *h;
-  a.tokens = d_tok; a.attn_t2v = (const float*)d_attn; a.out_tokens = d_out; a.kept_idx = (int*)d_kidx;
-  a.scores_out = h->scores_out ? (float*)d_sc : nullptr;
-  rc = ficoco_l_reduce(c, &a, prm, st);
+
+  // Sequences are independent: groups of sequences go through upload, kernels and download on three
+  // streams, as in ficoco_v_reduce_host (every group has its own slice of the staging area).
+  int n_groups = (int)((b_tok + b_attn) / HOST_GROUP_BYTES);
+  if (n_groups > HOST_MAX_GROUPS) n_groups = HOST_MAX_GROUPS;
+  if (n_groups > B) n_groups = B;
+  if (n_groups < 1) n_groups = 1;
+  cudaStream_t s_in = c->hs_stream, s_run = c->hs_run, s_out = c->hs_out;
+  if (n_groups == 1) s_run = s_out = s_in;
+  int launches = 0;
+  rc = FICOCO_OK;
+  auto group_begin = [&](int g) { return (int)((long long)B * g / n_groups); };
+  for (int g = 0; g < n_groups && rc == FICOCO_OK; ++g) {
+    const int b0 = group_begin(g), b1 = group_begin(g + 1);
+    cudaError_t e = cudaMemcpyAsync(d_tok + seq_tok * b0, (const char*)h->tokens + seq_tok * b0, seq_tok * (b1 - b0),
+                                    cudaMemcpyHostToDevice, s_in);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(d_attn + seq_attn * b0, (const char*)h->attn_t2v + seq_attn * b0, seq_attn * (b1 - b0),
+                          cudaMemcpyHostToDevice, s_in);
+    if (e == cudaSuccess && n_groups > 1) e = cudaEventRecord(c->hs_ev[2 * g], s_in);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; }
+  }
+  for (int g = 0; g < n_groups && rc == FICOCO_OK; ++g) {
+    const int b0 = group_begin(g), b1 = group_begin(g + 1);
+    const size_t o_out = (size_t)p_orow[b0] * row_b, n_out = (size_t)(p_orow[b1] - p_orow[b0]) * row_b;
+    const size_t o_ki = (size_t)p_orow[b0] * 4, n_ki = (size_t)(p_orow[b1] - p_orow[b0]) * 4;
+    cudaError_t e = cudaSuccess;
+    if (n_groups > 1) e = cudaStreamWaitEvent(s_run, c->hs_ev[2 * g], 0);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; break; }
+    ficoco_l_args a = *h;
+    a.batch = b1 - b0;
+    a.tokens = d_tok + seq_tok * b0;
+    a.attn_t2v = (const float*)(d_attn + seq_attn * b0);
+    if (h->n_keep != 1) { a.keep = h->keep + b0; a.n_keep = b1 - b0; }
+    a.out_tokens = d_out + o_out;
+    a.kept_idx = (int*)(d_kidx + o_ki);
+    a.scores_out = h->scores_out ? (float*)(d_sc + seq_sc * b0) : nullptr;
+    rc = ficoco_l_reduce(c, &a, prm, s_run);
+    if (rc) break;
+    launches += c->launches;
+    if (n_groups > 1) {
+      e = cudaEventRecord(c->hs_ev[2 * g + 1], s_run);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, c->hs_ev[2 * g + 1], 0);
+    }
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync((char*)h->out_tokens + o_out, d_out + o_out, n_out, cudaMemcpyDeviceToHost, s_out);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync((char*)h->kept_idx + o_ki, d_kidx + o_ki, n_ki, cudaMemcpyDeviceToHost, s_out);
+    if (e == cudaSuccess && h->scores_out)
+      e = cudaMemcpyAsync((char*)h->scores_out + seq_sc * b0, d_sc + seq_sc * b0, seq_sc * (b1 - b0),
+                          cudaMemcpyDeviceToHost, s_out);
+    if (e != cudaSuccess) { c->last_cuda = (int)e; rc = FICOCO_ERR_CUDA; }
+  }
+  // drain all three streams whatever happened, so that no copy outlives the call
+  const cudaError_t e1 = cudaStreamSynchronize(s_in), e2 = cudaStreamSynchronize(s_run),
+                    e3 = cudaStreamSynchronize(s_out);
   if (rc) return rc;
-  CUDA_TRY(c, cudaMemcpyAsync(h->out_tokens, d_out, b_out, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(c, cudaMemcpyAsync(h->kept_idx, d_kidx, b_kidx, cudaMemcpyDeviceToHost, st));
-  if (h->scores_out) CUDA_TRY(c, cudaMemcpyAsync(h->scores_out, d_sc, b_sc, cudaMemcpyDeviceToHost, st));
-  CUDA_TRY(c, cudaStreamSynchronize(st));
+  if (e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess) {
+    c->last_cuda = (int)(e1 != cudaSuccess ? e1 : e2 != cudaSuccess ? e2 : e3);
+    return FICOCO_ERR_CUDA;
+  }
+  c->launches = launches;
   return FICOCO_OK;
 }

@@ -208,6 +208,27 @@ def test_run_to_run_determinism_and_host_entry_point(ctx):
     assert np.array_equal(binding.to_numpy(d.kept_idx), binding.to_numpy(hh.kept_idx))
 
 
+def test_l_host_entry_point_in_sequence_groups(ctx):
+    """FiCoCo-L host-buffer call on the full-size workload (cut into groups of sequences whose uploads,
+    kernels and downloads overlap), with per-sequence keep counts: every output equals the
+    device-buffer call on the same bytes."""
+    lb = synth.workload(5)
+    pl = packing.pack_l(lb, DEV)
+    nseq = len(lb.tokens)
+    keep = np.array([64 + 3 * (b % 5) for b in range(nseq)], dtype=np.int32)
+    scores_d = torch.empty((nseq * pl.n_vision,), dtype=torch.float32, device=DEV)
+    d = ctx.ficoco_l_reduce(pl.tokens, pl.attn_t2v, keep, pl.n_vision, pl.n_text, pl.heads, scores_out=scores_d)
+    torch.cuda.synchronize()
+    plh = packing.pack_l(lb, None, pin=True)
+    scores_h = torch.empty((nseq * pl.n_vision,), dtype=torch.float32).pin_memory()
+    hh = ctx.ficoco_l_reduce_host(plh.tokens, plh.attn_t2v, keep, plh.n_vision, plh.n_text, plh.heads,
+                                  scores_out=scores_h)
+    assert np.array_equal(binding.to_numpy(d.out_tokens), binding.to_numpy(hh.out_tokens))
+    assert np.array_equal(binding.to_numpy(d.kept_idx), binding.to_numpy(hh.kept_idx))
+    assert np.array_equal(scores_d.cpu().numpy(), scores_h.numpy())
+    assert ctx.ficoco_status() == 0
+
+
 def test_back_to_back_steps_without_sync(ctx):
     """Steps queued on one stream with no host synchronisation between them: a step fed
     straight from the outputs of the step before it, and an independent step right behind
