@@ -307,13 +307,32 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       tT = reinterpret_cast<float*>(um_raw + (ring - smem_u32(um_raw)) + (size_t)UM * LCAP * 8);
       tSb = tT + (size_t)M * n_pad;
       const float* tb = tmean + (size_t)w.img * M * NV;
-      for (int i = pt; i < M * n_pad; i += 256) {
-        const int k = i / n_pad, cc = i - k * n_pad;
-        tT[i] = cc < ncols ? __ldg(tb + (size_t)k * NV + rowT[cc]) : 0.f;
+      // eight gathers in flight per thread (one at a time cost a round trip each: 13 us per CTA)
+      #pragma unroll 1
+      for (int i0 = pt; i0 < M * n_pad; i0 += 8 * 256) {
+        float q[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int i = i0 + 256 * j;
+          const int k = i / n_pad, cc = i - k * n_pad;
+          q[j] = (i < M * n_pad && cc < ncols) ? __ldg(tb + (size_t)k * NV + rowT[cc]) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (i0 + 256 * j < M * n_pad) tT[i0 + 256 * j] = q[j];
       }
-      for (int i = pt; i < M * rows_pad; i += 256) {
-        const int k = i / rows_pad, rr = i - k * rows_pad;
-        tSb[i] = rr < w.nrows ? __ldg(tb + (size_t)k * NV + rowS[rr]) : 0.f;
+      #pragma unroll 1
+      for (int i0 = pt; i0 < M * rows_pad; i0 += 8 * 256) {
+        float q[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int i = i0 + 256 * j;
+          const int k = i / rows_pad, rr = i - k * rows_pad;
+          q[j] = (i < M * rows_pad && rr < w.nrows) ? __ldg(tb + (size_t)k * NV + rowS[rr]) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (i0 + 256 * j < M * rows_pad) tSb[i0 + 256 * j] = q[j];
       }
       cta_sync(1, 256);
     }
