@@ -269,8 +269,9 @@ int ficoco_l_reduce_host(ficoco_ctx* ctx, const ficoco_l_args* host_args,
 /* Synchronise `cuda_stream`, read and clear the device status word into *device_status
  * (0 = clean; bit 0 (1): a pos entry outside grid_h*grid_w was ignored by the local penalty;
  * bit 2 (4): a bounded device-side wait ran out: the outputs of that step and of every step
- * enqueued after it are invalid).  Returns FICOCO_OK when the word could be read, whatever it
- * holds. */
+ * enqueued after it are invalid; bit 3 (8): an internal index list held a token index outside
+ * its image, which was replaced by 0 instead of being followed: the outputs of that step are
+ * invalid).  Returns FICOCO_OK when the word could be read, whatever it holds. */
 int ficoco_status(ficoco_ctx* ctx, void* cuda_stream, int* device_status);
 
 /* Testing hook for the bounded waits.  wait_ns > 0 sets the time after which a device-side wait

@@ -8,6 +8,7 @@
 namespace ficoco {
 
 constexpr unsigned STATUS_TIMEOUT = 4u;
+constexpr unsigned STATUS_INDEX = 8u;     // an index list held a token index outside its image (replaced by 0)
 constexpr unsigned long long WAIT_NS_DEFAULT = 20ull * 1000 * 1000;   // 20 ms: far beyond any wait of a healthy step
 
 __device__ __forceinline__ unsigned long long global_ns() {

@@ -82,6 +82,17 @@ __device__ __forceinline__ uint4 ldg16(const void* p) { return __ldg(reinterpret
 // output pushes the token rows out before the next kernel reads them again.
 __device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) { __stcs(p, v); }
 
+// A token index read from an index list of the step, as a row offset inside its image: anything
+// outside [0, np) (lists left behind by a step that went wrong) raises STATUS_INDEX and becomes 0,
+// so that no gather leaves the image.
+__device__ __forceinline__ int checked_index(int idx, int np, unsigned* status) {
+  if ((unsigned)idx >= (unsigned)np) {
+    atomicOr(status, 8u);
+    return 0;
+  }
+  return idx;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);

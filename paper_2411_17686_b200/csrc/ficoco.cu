@@ -177,6 +177,7 @@ struct ficoco_ctx {
   int merge_ctas_per_sm_dense = 1;   // the same with the register cap for 4 (plans without the fused filter)
   int* img_cnt = nullptr;   // two sets of 3 * max_batch per-image counters of the fused filter kernel
   unsigned long long epoch = 0;          // fused filter launches so far (its parity picks the counter set)
+  int last_parity = 0;                   // counter set of the latest fused filter launch
   unsigned long long wait_ns = WAIT_NS_DEFAULT;   // bound of every device-side wait
   int dbg_extra_arrivals = 0;            // testing hook: arrivals the fused filter waits for that never come
   int num_sms = 0;
@@ -917,11 +918,12 @@ cudaError_t launch_filter_fused(ficoco_ctx* c, const Plan* p, const T* tok, int 
   at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
   cfg.numAttrs = (c->coop_pdl_ok && overlap_prev) ? 2 : 1;   // 1: inputs independent of the step before; 2: fed by it
+  c->last_parity = (int)(c->epoch++ & 1);
   return cudaLaunchKernelEx(&cfg, k_filter_fused<T, VPL>, tok, D, (const ImgDesc*)p->d_desc,
                             (const WorkItem*)p->d_rows, (const int*)p->d_ctafirst, c->rn, c->partial, attn,
                             attn_rows, cA, c->s_raw, c->img_cnt, p->key.batch, pos, window, coef, penalty,
                             c->s_pen, scores_out, c->S_idx, c->T_idx, kept_idx, pos_out, c->status,
-                            p->f_nstage, p->f_max_piece, (int)(c->epoch++ & 1), 3 * c->max_batch, c->wait_ns,
+                            p->f_nstage, p->f_max_piece, c->last_parity, 3 * c->max_batch, c->wait_ns,
                             c->dbg_extra_arrivals, (c->coop_pdl_ok && overlap_prev == 2) ? 1 : 0);
 }
 
@@ -1096,12 +1098,12 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
     launch_dependent(k_merge_scan<T, 3>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
                      (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
                      (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
-                     (const unsigned*)c->status);
+                     c->status, c->img_cnt + (size_t)c->last_parity * 3 * c->max_batch, 3 * c->max_batch);
   else
     launch_dependent(k_merge_scan<T, 4>, p->n_out, 256, 0, st, tok, D, (const ImgDesc*)p->d_desc,
                      (const WorkItem*)p->d_out, (const int*)c->S_idx, (const int*)c->T_idx,
                      (const int*)c->e_tgt, (const float*)c->e_w, out_tokens, after_correlate,
-                     (const unsigned*)c->status);
+                     c->status, (int*)nullptr, 0);
   c->launches += 1;
   if (p->key.conv) {
     prof_tick(c, st, "convergent_token");

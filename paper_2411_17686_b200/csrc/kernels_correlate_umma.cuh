@@ -220,9 +220,9 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
                    : "memory");
     return;
   }
-  if (tid < UM * UM_SUB) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
+  if (tid < UM * UM_SUB) rowS[tid] = tid < w.nrows ? checked_index(S_idx[d.src0 + w.r0 + tid], d.np, status) : -1;
   for (int c = tid; c < UN_MAX; c += UTHREADS) {
-    const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
+    const int p = c < ncols ? checked_index(T_idx[d.tgt0 + col_begin + c], d.np, status) : -1;
     rowT[c] = p;
     rnT[c] = p >= 0 ? rn[d.patch0 + p] : 0.f;
   }

@@ -161,10 +161,10 @@ __global__ void __launch_bounds__(UTHREADS, 1) k_correlate_umma_f32(
                    : "memory");
     return;
   }
-  if (tid < UM) rowS[tid] = tid < w.nrows ? S_idx[d.src0 + w.r0 + tid] : -1;
+  if (tid < UM) rowS[tid] = tid < w.nrows ? checked_index(S_idx[d.src0 + w.r0 + tid], d.np, status) : -1;
   if (tid >= UM && tid < UM + UF_COLS) {
     const int c = tid - UM;
-    const int p = c < ncols ? T_idx[d.tgt0 + col_begin + c] : -1;
+    const int p = c < ncols ? checked_index(T_idx[d.tgt0 + col_begin + c], d.np, status) : -1;
     rowT[c] = p;
     rnT[c] = p >= 0 ? rn[d.patch0 + p] : 0.f;
   }

@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(256, MINB) k_merge_scan(
     const T* __restrict__ tokens, int D, const ImgDesc* __restrict__ desc,
     const WorkItem* __restrict__ work, const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     const int* __restrict__ e_tgt, const float* __restrict__ e_w, T* __restrict__ out,
-    int index_before_wait, const unsigned* __restrict__ status) {
+    int index_before_wait, unsigned* __restrict__ status, int* __restrict__ filter_cnt, int n_filter_cnt) {
   constexpr int E = VecTraits<T>::E;
   __shared__ int cnt[MROWS], beg[MROWS + 1], cur[MROWS], srow_s[MROWS];
   __shared__ int lsrc[MLIST];
@@ -99,12 +99,20 @@ __global__ void __launch_bounds__(256, MINB) k_merge_scan(
     const int orow = w.r0 + r;
     int srow;
     if (orow < d.n_cls) srow = orow;
-    else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + T_idx[d.tgt0 + orow - d.n_cls];
+    else if (orow < d.n_cls + d.n_tgt) srow = d.n_cls + checked_index(T_idx[d.tgt0 + orow - d.n_cls], d.np, status);
     else if (orow < d.n_cls + d.n_tgt + d.n_extra) srow = -1;     // the additional token: written by k_convergent_token
     else srow = d.n_cls + d.np + (orow - d.n_cls - d.n_tgt - d.n_extra);
     if (lane == 0) srow_s[r] = srow;
   }
   if (index_before_wait) grid_dep_wait();
+  // The filter grid of this step is complete: its per-image counters are cleared for whichever launch
+  // uses that set next (launches replayed from graphs need not alternate between the two sets).  The
+  // stores are fenced and the CTA synchronised before it releases the dependent grid.
+  if (filter_cnt != nullptr && blockIdx.x == 0) {
+    for (int i = tid; i < n_filter_cnt; i += 256) filter_cnt[i] = 0;
+    __threadfence();
+    __syncthreads();
+  }
   grid_dep_launch();   // correlate is complete: the next step's filter may stream its rows under our tail
   FICOCO_PHASE(2, 1);
   // a step whose filter or correlate grid gave up has no valid index lists: write nothing
@@ -129,7 +137,7 @@ __global__ void __launch_bounds__(256, MINB) k_merge_scan(
         const int e = tid + 256 * i;
         const bool on = e < n_ent;
         t4[i] = on ? e_tgt[d.ent0 + e] : -1;
-        st_src[i] = on ? S_idx[d.src0 + e / L] : 0;
+        st_src[i] = on ? checked_index(S_idx[d.src0 + e / L], d.np, status) : 0;
         st_w[i] = on ? e_w[d.ent0 + e] : 0.f;
       }
 #pragma unroll
@@ -178,7 +186,7 @@ __global__ void __launch_bounds__(256, MINB) k_merge_scan(
         const int t = e_tgt[d.ent0 + e];
         if (t >= tp_lo && t < tp_hi) {
           const int slot = beg[t - tp_lo] + atomicAdd(&cur[t - tp_lo], 1);
-          const int si = S_idx[d.src0 + e / L];
+          const int si = checked_index(S_idx[d.src0 + e / L], d.np, status);
           tsrc[slot] = si;
           tw[slot] = e_w[d.ent0 + e];
         }
@@ -281,7 +289,7 @@ __global__ void __launch_bounds__(256, MINB) k_merge_scan(
         unpack(ldg16(src + (size_t)v * E), acc, (const T*)nullptr);
         for (int e = 0; e < n_ent; ++e) {
           if (e_tgt[d.ent0 + e] != tp) continue;
-          const T* x0 = pbase + (size_t)S_idx[d.src0 + e / L] * D;
+          const T* x0 = pbase + (size_t)checked_index(S_idx[d.src0 + e / L], d.np, status) * D;
           float f[E];
           unpack(ldg16(x0 + (size_t)v * E), f, (const T*)nullptr);
           const float a0 = e_w[d.ent0 + e];

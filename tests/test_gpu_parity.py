@@ -1,5 +1,6 @@
 """GPU parity: the CUDA library (through its C ABI) against the float64 checker, element by
 element, on seeded inputs whose discrete decisions were made unambiguous beforehand."""
+import collections
 import copy
 import json
 import os
@@ -13,6 +14,7 @@ from paper_2411_17686_b200 import binding, packing, synth
 from tests import parity
 
 pytestmark = pytest.mark.gpu
+VResultLike = collections.namedtuple("VResultLike", "out_tokens kept_idx pos_out")
 DEV = "cuda:0"
 
 
@@ -500,6 +502,56 @@ def test_planned_ragged_shape_is_captured_into_a_graph():
     for a, b in zip(got, (ref.out_tokens, ref.kept_idx, ref.pos_out)):
         assert np.array_equal(a, binding.to_numpy(b))
     assert c.ficoco_status() == 0
+    c.close()
+
+
+def test_graph_of_an_odd_number_of_steps_replayed():
+    """Three back-to-back steps captured into one graph and replayed several times, then followed by
+    ordinary calls: launches replayed from a graph do not alternate between the fused filter's two
+    sets of per-image counters the way consecutive calls do, and every launch must still find its
+    set clean.  Every replay reproduces the bytes of an ordinary call."""
+    c = binding.Context(max_tokens=8 * 145, max_dim=256, max_batch=8, device=0)
+    prm = binding.make_params(has_cls=True, back_to_back=True)
+    sets = []
+    for i in range(3):
+        batch = synth.make_v_batch(120 + i, 8, 12, 12, 256, 4, 64, "bf16", True, 1.0)
+        pk = packing.pack_v(batch, DEV)
+        ref = c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads,
+                                params=binding.make_params(has_cls=True), **pk.call_kwargs())
+        torch.cuda.synchronize()
+        res = VResultLike(torch.zeros_like(ref.out_tokens), torch.zeros_like(ref.kept_idx), torch.zeros_like(ref.pos_out))
+        sets.append((pk, ref, res))
+    st = torch.cuda.Stream()
+
+    def step(i):
+        pk, _, res = sets[i]
+        c.ficoco_v_reduce(pk.tokens, pk.attn, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm,
+                          out_tokens=res.out_tokens, kept_idx=res.kept_idx, pos_out=res.pos_out,
+                          stream=st.cuda_stream, **pk.call_kwargs())
+
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        for i in range(3):
+            step(i)
+    for rep in range(5):
+        for _, _, res in sets:
+            res.out_tokens.zero_(); res.kept_idx.zero_(); res.pos_out.zero_()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(st):
+            g.replay()
+            if rep == 2:
+                g.replay()            # two replays with nothing in between
+        torch.cuda.synchronize()
+        for _, ref, res in sets:
+            assert np.array_equal(binding.to_numpy(ref.out_tokens), binding.to_numpy(res.out_tokens)), rep
+            assert np.array_equal(binding.to_numpy(ref.kept_idx), binding.to_numpy(res.kept_idx)), rep
+            assert np.array_equal(binding.to_numpy(ref.pos_out), binding.to_numpy(res.pos_out)), rep
+    with torch.cuda.stream(st):           # an ordinary call right behind a replay
+        g.replay()
+        step(0)
+    torch.cuda.synchronize()
+    assert np.array_equal(binding.to_numpy(sets[0][1].out_tokens), binding.to_numpy(sets[0][2].out_tokens))
+    assert c.ficoco_status(st.cuda_stream) == 0
     c.close()
 
 
