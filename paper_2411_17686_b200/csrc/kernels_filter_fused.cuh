@@ -15,7 +15,10 @@
 //           the selection alone.
 // The inter-CTA waits are polls of per-image counters, bounded by elapsed time (wait_ns).  The
 // counters exist twice; a launch uses the set of its parity and zeroes the other one, so a step
-// that gave up half-way cannot leave counts behind for the step after the next.
+// that gave up half-way cannot leave counts behind for the step after the next.  The set a launch
+// used is cleared by the merge grid of the same step (which runs once the filter grid is complete
+// and before a later filter grid can start), so launches replayed from CUDA graphs, whose
+// parities are fixed at capture, find their set clean in whatever order they run.
 #pragma once
 #include "async_ops.cuh"
 #include "common.cuh"
