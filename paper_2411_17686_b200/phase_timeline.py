@@ -115,6 +115,7 @@ def main() -> None:
         ctx.ficoco_v_reduce(tok, att, pk.keep, pk.grid_h, pk.grid_w, pk.heads, params=prm, out_tokens=res.out_tokens,
                             kept_idx=res.kept_idx, pos_out=res.pos_out, **pk.call_kwargs())
 
+    torch.cuda.synchronize()                             # a context serves one stream at a time
     stream = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.stream(stream):
