@@ -33,7 +33,7 @@ MIN_TIMED_MS = 50.0   # device time the timed repetitions add up to, at least
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}   # vendor figures, reported beside the measured peaks
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised under
 # profiles/ (bytes); an entry is removed when its kernel changes after the capture.
-NCU_TRAFFIC = {"filter_fused": 39091200 + 10240, "correlate_umma": 37960192 + 256, "merge_compact": 37890048 + 61184}
+NCU_TRAFFIC = {"filter_fused": 39088384 + 12800, "correlate_umma": 37963264 + 7680, "merge_compact": 37894912 + 30720}
 
 
 def algorithmic_bytes() -> dict:
