@@ -1038,7 +1038,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
 #define FICOCO_REL_GO(LC)                                                                              \
   k_correlate_rel<LC><<<p->n_corr, 256, (size_t)rel_cols * sizeof(int), st>>>(rel, p->d_desc, p->d_corr, c->S_idx, c->T_idx, c->part_val, \
                                                  c->part_idx, c->tile_cnt, c->corr_cnt, c->tau, c->e_tgt,    \
-                                                 c->e_w, c->e_c)
+                                                 c->e_w, c->e_c, c->status)
       if (p->max_list <= 2) FICOCO_REL_GO(2);
       else if (p->max_list <= 4) FICOCO_REL_GO(4);
       else FICOCO_REL_GO(16);
@@ -1082,7 +1082,7 @@ int run_step(ficoco_ctx* c, const Plan* p, const T* tok, int D, const float* att
       k_correlate_simt<T><<<p->n_corr, 256, 0, st>>>(tok, D, p->d_desc, p->d_corr, c->rn, c->S_idx,
                                                      c->T_idx, tmean, M, gamma, c->part_val, c->part_idx,
                                                      c->tile_cnt, c->corr_cnt, c->tau,
-                                                     c->e_tgt, c->e_w, c->e_c);
+                                                     c->e_tgt, c->e_w, c->e_c, c->status);
     }
     c->launches += 1;
   }

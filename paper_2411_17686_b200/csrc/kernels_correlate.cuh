@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     const float* __restrict__ tmean, int M, float gamma,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ img_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c) {
+    float* __restrict__ e_w, float* __restrict__ e_c, unsigned* __restrict__ status) {
   __shared__ int is_last;
   __shared__ __align__(16) float As[CKC][CBM + 4];
   __shared__ __align__(16) float Bs[CKC][CBN + 4];
@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
   }
   if (tid < CBM) {
     const bool ok = tid < w.nrows;
-    const int p = ok ? S_idx[d.src0 + w.r0 + tid] : -1;
+    const int p = ok ? checked_index(S_idx[d.src0 + w.r0 + tid], d.np, status) : -1;
     rowS[tid] = p;
     rnS[tid] = ok ? rn[d.patch0 + p] : 0.f;
   }
@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(256) k_correlate_simt(
     if (tid < CBN) {
       const int c = c0 + tid;
       const bool ok = c < col_end;
-      const int p = ok ? T_idx[d.tgt0 + c] : -1;
+      const int p = ok ? checked_index(T_idx[d.tgt0 + c], d.np, status) : -1;
       rowT[tid] = p;
       rnT[tid] = ok ? rn[d.patch0 + p] : 0.f;
     }

@@ -168,7 +168,7 @@ __global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
     const int* __restrict__ S_idx, const int* __restrict__ T_idx,
     float* __restrict__ part_val, int* __restrict__ part_idx, int* __restrict__ tile_done,
     int* __restrict__ corr_cnt, float* __restrict__ tau_out, int* __restrict__ e_tgt,
-    float* __restrict__ e_w, float* __restrict__ e_c) {
+    float* __restrict__ e_w, float* __restrict__ e_c, unsigned* __restrict__ status) {
   extern __shared__ int tcol[];              // token index of every column of the split
   __shared__ int is_last;
   const WorkItem w = work[blockIdx.x];
@@ -180,12 +180,12 @@ __global__ void __launch_bounds__(256, LC <= 4 ? 4 : 2) k_correlate_rel(
   const int ncol = min(d.n_tgt, col_begin + d.cols_per_split) - col_begin;
   // the rows of this warp (two at most with the planned tiles of 16) are looked up while the
   // column indices arrive
-  const int r_first = warp < w.nrows ? S_idx[d.src0 + w.r0 + warp] : 0;
-  for (int c = threadIdx.x; c < ncol; c += 256) tcol[c] = T_idx[d.tgt0 + col_begin + c];
+  const int r_first = warp < w.nrows ? checked_index(S_idx[d.src0 + w.r0 + warp], np, status) : 0;
+  for (int c = threadIdx.x; c < ncol; c += 256) tcol[c] = checked_index(T_idx[d.tgt0 + col_begin + c], np, status);
   __syncthreads();
   #pragma unroll 1
   for (int r = warp; r < w.nrows; r += 8) {
-    const float* row = A + (size_t)(r == warp ? r_first : S_idx[d.src0 + w.r0 + r]) * np;
+    const float* row = A + (size_t)(r == warp ? r_first : checked_index(S_idx[d.src0 + w.r0 + r], np, status)) * np;
     float v[LC];
     int ix[LC];
 #pragma unroll
