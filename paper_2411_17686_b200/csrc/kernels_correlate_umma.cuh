@@ -360,9 +360,9 @@ __global__ void __launch_bounds__(UTHREADS, 2) k_correlate_umma(
       {
         const float* hv = reinterpret_cast<const float*>(um_raw + (ring - smem_u32(um_raw)));
         const int* hi = reinterpret_cast<const int*>(hv + UM * LCAP);
-#pragma unroll
-        for (int e = 0; e < LCAP; ++e) {
-          if (e < L) {
+        #pragma unroll 1                               // rolled: the body is a full insertion
+        for (int e = 0; e < L; ++e) {
+          {
             float cv = hv[tid * LCAP + e];
             int ci = hi[tid * LCAP + e];
             bool shift = ci == INT_MAX;                // empty helper slot: nothing to insert

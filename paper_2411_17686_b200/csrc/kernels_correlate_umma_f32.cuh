@@ -277,9 +277,9 @@ __global__ void __launch_bounds__(UTHREADS, 1) k_correlate_umma_f32(
         for (int k = 0; k < LCAP; ++k) { v[k] = -CUDART_INF_F; ix[k] = INT_MAX; }
       }
       cta_sync(1, 256);                                // the helpers' lists are in shared memory
-#pragma unroll
-      for (int e = 0; e < LCAP; ++e) {
-        if (e < L) {
+      #pragma unroll 1                                 // rolled: the body is a full insertion
+      for (int e = 0; e < L; ++e) {
+        {
           float cv = hv[tid * LCAP + e];
           int ci = hi[tid * LCAP + e];
           if (ci != INT_MAX) {
